@@ -1,0 +1,509 @@
+"""Pins for the CPU oracle: each check ties one oracle function to something other than itself --
+a closed form, a hand-worked fixture under tests/golden/, a brute-force library routine, or an
+invariant the paper states (degree bound, exact reverse graph, no edge to a deleted node)."""
+import os
+
+import numpy as np
+import pytest
+
+from oracle import grand_oracle as go
+from paper_2608_21163_b200 import synth
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+INV = go.INVALID
+
+
+def mk(dim, dtype=go.U8, metric=go.L2, R=4, L=8, alpha=1.2, cap=16, **kw):
+    return go.Oracle(dim, dtype, metric, R, L, alpha, cap, nthreads=kw.pop("nthreads", 2), **kw)
+
+
+def load_graph(o, vecs, rows, entry, live=None):
+    cap, R = o.capacity, o.R
+    adj = np.full((cap, R), INV, np.uint32)
+    deg = np.zeros(cap, np.uint32)
+    for v, r in rows.items():
+        adj[v, :len(r)] = r
+        deg[v] = len(r)
+    if live is None:
+        live = np.zeros(cap, bool)
+        live[:len(vecs)] = True
+    full = np.zeros((cap, o.dim), o.np_dtype)
+    full[:len(vecs)] = vecs
+    o.import_graph(adj, deg, go.pack_bitmap(live), entry, full)
+
+
+def brute_knn(base, ids, q, k, metric=go.L2):
+    b = base[ids].astype(np.float64)
+    if metric == go.L2:
+        d = ((b - q.astype(np.float64)[None, :]) ** 2).sum(1)
+    else:
+        d = -(b @ q.astype(np.float64))
+    order = np.lexsort((ids, d))[:k]
+    return ids[order], d[order]
+
+
+# ------------------------------------------------------------------ distance
+def test_dist_closed_forms():
+    o = mk(4)
+    assert o.dist([0, 0, 0, 0], [255, 255, 255, 255]) == 4 * 255 * 255
+    assert o.dist([1, 2, 3, 4], [4, 2, 0, 9]) == 9 + 0 + 9 + 25
+    oi = mk(4, dtype=go.I8)
+    assert oi.dist([-128, 127, 0, 5], [127, -128, 0, 5]) == 2 * 255 * 255
+    oip = mk(4, dtype=go.U8, metric=go.IP, mode=go.FIXED_DEGREE)
+    assert oip.dist([1, 2, 3, 4], [5, 6, 7, 8]) == -(5 + 12 + 21 + 32)
+    of = mk(3, dtype=go.F32)
+    assert of.dist([0.5, 0.25, 0.0], [0.0, 0.0, 2.0]) == 0.25 + 0.0625 + 4.0
+    ofi = mk(3, dtype=go.F32, metric=go.IP, mode=go.FIXED_DEGREE)
+    assert ofi.dist([0.5, 0.25, 1.0], [2.0, 4.0, -1.0]) == -(1.0 + 1.0 - 1.0)
+
+
+def test_dist_symmetry_and_range():
+    rng = np.random.default_rng(1)
+    o = mk(960)
+    a = rng.integers(0, 256, 960).astype(np.uint8)
+    b = rng.integers(0, 256, 960).astype(np.uint8)
+    assert o.dist(a, b) == o.dist(b, a) == float(((a.astype(np.int64) - b.astype(np.int64)) ** 2).sum())
+    z = np.zeros(960, np.uint8); f = np.full(960, 255, np.uint8)
+    assert o.dist(z, f) == 960 * 255 * 255 < 2 ** 31
+    of = mk(96, dtype=go.F32)
+    x = rng.standard_normal(96).astype(np.float32); y = rng.standard_normal(96).astype(np.float32)
+    assert of.dist(x, y) == of.dist(y, x)
+    exact = ((x.astype(np.float64) - y.astype(np.float64)) ** 2).sum()
+    assert abs(of.dist(x, y) - exact) <= 2 ** -23 * exact      # one rounding to float
+    assert of.dist(x, y) == float(np.float32(of.dist(x, y)))   # result is a float32 value
+
+
+def test_unsupported_vamana_ip():
+    with pytest.raises(go.OracleError):
+        mk(4, metric=go.IP)
+
+
+# ------------------------------------------------------------------ BeamSearch (Alg. 1)
+def test_search_complete_graph_equals_bruteforce():
+    rng = np.random.default_rng(2)
+    n, d = 40, 8
+    base = rng.integers(0, 256, (n, d)).astype(np.uint8)
+    base[7] = base[3]                      # an exact duplicate: ties must break by id
+    o = mk(d, R=n - 1, L=12, cap=n)
+    rows = {v: [w for w in range(n) if w != v] for v in range(n)}
+    load_graph(o, base, rows, entry=5)
+    qs = rng.integers(0, 256, (25, d)).astype(np.uint8)
+    qs[0] = base[3]
+    ids, dist = o.search(qs, 10, 12)
+    for i, q in enumerate(qs):
+        bi, bd = brute_knn(base, np.arange(n, dtype=np.uint32), q, 10)
+        assert (ids[i] == bi).all() and (dist[i] == bd).all()
+    assert o.stats()["dead_edges_seen"] == 0
+
+
+def test_search_large_beam_reaches_everything():
+    """With L >= N every reachable node enters the worklist, so the result is brute force over
+    the nodes reachable from the entry point (here: a ring plus chords, all reachable)."""
+    rng = np.random.default_rng(3)
+    n, d = 60, 6
+    base = rng.standard_normal((n, d)).astype(np.float32)
+    o = mk(d, dtype=go.F32, R=3, L=n, cap=n)
+    rows = {v: [(v + 1) % n, (v * 7 + 3) % n, (v * 11 + 5) % n] for v in range(n)}
+    rows = {v: list(dict.fromkeys(w for w in r if w != v)) for v, r in rows.items()}
+    load_graph(o, base, rows, entry=0)
+    q = rng.standard_normal((5, d)).astype(np.float32)
+    ids, dist = o.search(q, 10, n)
+    for i in range(5):
+        bi, _ = brute_knn(base, np.arange(n, dtype=np.uint32), q[i], 10)
+        assert (ids[i] == bi).all()
+        exact = ((base[bi].astype(np.float64) - q[i].astype(np.float64)) ** 2).sum(1)
+        assert np.allclose(dist[i], exact, rtol=2e-7, atol=0)
+
+
+def test_search_path_graph_walk():
+    """1-D path 0-1-2-3-4 at x = 10*id, query 41, L = 1 from node 0: visits 0,1,2,3,4, returns [4]."""
+    base = (10 * np.arange(5))[:, None].astype(np.uint8)
+    o = mk(1, R=2, L=1, cap=5)
+    rows = {0: [1], 1: [0, 2], 2: [1, 3], 3: [2, 4], 4: [3]}
+    load_graph(o, base, rows, entry=0)
+    (bi, bd), (vi, vd) = o.greedy(np.array([41], np.uint8), L=1, vmax=10)
+    assert vi.tolist() == [0, 1, 2, 3, 4]
+    assert vd.tolist() == [41 ** 2, 31 ** 2, 21 ** 2, 11 ** 2, 1]
+    assert bi.tolist() == [4] and bd.tolist() == [1]
+    # expansion cap: vmax = 3 stops after three expansions
+    (_, _), (vi, _) = o.greedy(np.array([41], np.uint8), L=1, vmax=3)
+    assert vi.tolist() == [0, 1, 2]
+
+
+def test_search_seen_set_independence():
+    """A full visited set only saves distance evaluations; results must not change."""
+    cfg = synth.scaled(synth.CONFIGS["tiny_u8_d32"], 0.2)
+    base = synth.uniform_u8(0, "base", 0, cfg["n"], 32)
+    o = go.Oracle(32, go.U8, go.L2, 16, 24, 1.2, cfg["n"])
+    for lo in range(0, cfg["n"], 500):
+        o.insert_batch(np.arange(lo, lo + 500, dtype=np.uint32), base[lo:lo + 500])
+    q = synth.uniform_u8(0, "query", 0, 200, 32)
+    a = o.search(q, 10, 24, use_seen_set=False)
+    b = o.search(q, 10, 24, use_seen_set=True)
+    assert (a[0] == b[0]).all() and (a[1] == b[1]).all()
+    (ca, va) = o.greedy(q[0], 24, 48, False)
+    (cb, vb) = o.greedy(q[0], 24, 48, True)
+    assert (ca[0] == cb[0]).all() and (va[0] == vb[0]).all()
+
+
+def test_search_empty_and_padding():
+    o = mk(2, R=2, L=4, cap=4)
+    ids, d = o.search(np.zeros((2, 2), np.uint8), 3, 4)
+    assert (ids == INV).all() and np.isinf(d).all()
+    o.insert_batch([2], np.array([[1, 1]], np.uint8))
+    ids, d = o.search(np.zeros((1, 2), np.uint8), 3, 4)
+    assert ids.tolist() == [[2, INV, INV]] and d[0, 0] == 2 and np.isinf(d[0, 1:]).all()
+
+
+# ------------------------------------------------------------------ RobustPrune (Alg. 4)
+def _read_prune_fixture():
+    spec = {}
+    for line in open(os.path.join(GOLD, "robust_prune_example.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        k, rest = line.split(" ", 1)
+        spec.setdefault(k, []).append(rest.strip())
+    vecs = np.array([[int(x) for x in p.split(",")] for p in spec["vectors"][0].split()], np.uint8)
+    cand = [int(x) for x in spec["candidates"][0].split()]
+    D = [float(x) for x in spec["D"][0].split()]
+    cases = {}
+    for a in spec["alpha"]:
+        al, res = a.split("->")
+        cases[float(al)] = [int(x) for x in res.split()]
+    return vecs, int(spec["p"][0]), cand, D, int(spec["R"][0]), cases
+
+
+def test_prune_hand_worked_example():
+    vecs, p, cand, D, R, cases = _read_prune_fixture()
+    for alpha, want in cases.items():
+        o = mk(2, R=R, L=8, alpha=alpha, cap=8)
+        load_graph(o, vecs, {}, entry=0)
+        # the fixture's D really are dist(p, .)
+        assert [o.dist(vecs[p], vecs[c]) for c in cand] == D
+        got = o.prune(p, cand, D, R)
+        assert got.tolist() == want, (alpha, got)
+        # candidate order must not matter, self and repeated ids are dropped
+        got2 = o.prune(p, cand[::-1] + [p, cand[0]], D[::-1] + [0.0, D[0]], R)
+        assert got2.tolist() == want
+
+
+def test_prune_large_alpha_is_partial_sort_and_bounds():
+    rng = np.random.default_rng(4)
+    n, d, R = 50, 5, 7
+    base = rng.integers(0, 256, (n, d)).astype(np.uint8)
+    o = mk(d, R=R, L=8, alpha=1e6, cap=n)
+    load_graph(o, base, {}, entry=0)
+    cand = np.arange(1, n, dtype=np.uint32)
+    D = [o.dist(base[0], base[c]) for c in cand]
+    got = o.prune(0, cand, D, R)
+    want, _ = brute_knn(base, cand, base[0], R)
+    assert (got == want).all()
+    o2 = mk(d, R=R, L=8, alpha=1.2, cap=n)
+    load_graph(o2, base, {}, entry=0)
+    got = o2.prune(0, cand, D, R)
+    assert 1 <= len(got) <= R and len(set(got.tolist())) == len(got) and set(got.tolist()) <= set(cand.tolist())
+    keys = [(o.dist(base[0], base[g]), g) for g in got]
+    assert keys == sorted(keys)
+    assert got[0] == want[0]                       # the nearest candidate always survives
+    # definition check of every selected node: no earlier selected p* satisfies alpha*d(p*,v) <= D[v]
+    for j, v in enumerate(got):
+        for s in got[:j]:
+            assert 1.2 * o.dist(base[s], base[v]) > o.dist(base[0], base[v])
+
+
+def test_prune_alpha_boundary_fixed_point_and_fp32():
+    # 1-D: p=0 at x=0, a at x=10 (D=100), b at x=20 (D=400): d(a,b)=100.  alpha*100 <= 400 iff alpha <= 4.
+    vecs = np.array([[0], [10], [20]], np.uint8)
+    for alpha, want in [(4.0, [1]), (4.001, [1, 2]), (1.0, [1])]:
+        o = mk(1, R=3, alpha=alpha, cap=4)
+        load_graph(o, vecs, {}, entry=0)
+        assert o.prune(0, [1, 2], [100.0, 400.0], 3).tolist() == want
+    for alpha, want in [(4.0, [1]), (4.001, [1, 2])]:
+        o = mk(1, dtype=go.F32, R=3, alpha=alpha, cap=4)
+        load_graph(o, vecs.astype(np.float32), {}, entry=0)
+        assert o.prune(0, [1, 2], [100.0, 400.0], 3).tolist() == want
+    # R = 1 stops right after the first pick
+    o = mk(1, R=1, alpha=1.2, cap=4)
+    load_graph(o, vecs, {}, entry=0)
+    assert o.prune(0, [2, 1], [400.0, 100.0], 1).tolist() == [1]
+
+
+# ------------------------------------------------------------------ reverse graph (Alg. 8)
+def test_transpose_hand_example():
+    rows, off, src = {}, None, None
+    for line in open(os.path.join(GOLD, "transpose_example.txt")):
+        if line.startswith("out"):
+            v, r = line[4:].split(":")
+            rows[int(v)] = [int(x) for x in r.split()]
+        elif line.startswith("off"):
+            off = [int(x) for x in line.split()[1:]]
+        elif line.startswith("src"):
+            src = [int(x) for x in line.split()[1:]]
+    o = mk(1, R=2, cap=4)
+    load_graph(o, np.zeros((4, 1), np.uint8), rows, entry=0)
+    goff, gsrc = o.reverse_graph()
+    assert goff.tolist() == off and gsrc.tolist() == src
+
+
+def edges_of(adj, deg, mask):
+    e = set()
+    for v in np.flatnonzero(mask):
+        for w in adj[v, :deg[v]]:
+            e.add((int(v), int(w)))
+    return e
+
+
+def test_transpose_properties_on_built_graph():
+    base = synth.uniform_u8(0, "base", 0, 1500, 32)
+    o = go.Oracle(32, go.U8, go.L2, 12, 24, 1.2, 1500)
+    for lo in range(0, 1500, 300):
+        o.insert_batch(np.arange(lo, lo + 300, dtype=np.uint32), base[lo:lo + 300])
+    adj, deg, live, _ = o.export_graph()
+    mask = go.live_mask(live, 1500)
+    off, src = o.reverse_graph()
+    assert off[-1] == deg[mask].sum() == len(src)
+    fwd = edges_of(adj, deg, mask)
+    rev = set()
+    for z in range(1500):
+        r = src[off[z]:off[z + 1]]
+        assert (np.diff(r.astype(np.int64)) > 0).all()      # rows ascending, no repeats
+        rev |= {(int(v), z) for v in r}
+    assert rev == fwd                                        # exact transpose
+
+
+# ------------------------------------------------------------------ batch insert (Alg. 5)
+def check_invariants(o, n_expected_live=None):
+    adj, deg, live, entry = o.export_graph()
+    mask = go.live_mask(live, o.capacity)
+    if n_expected_live is not None:
+        assert mask.sum() == n_expected_live == o.live_count
+    assert (deg <= o.R).all()
+    assert (deg[~mask] == 0).all()
+    for v in np.flatnonzero(mask):
+        r = adj[v, :deg[v]]
+        assert v not in r, "self loop"
+        assert len(set(r.tolist())) == len(r), "repeated neighbour"
+        assert mask[r].all(), "edge to a non-live node"
+    if mask.any():
+        assert mask[entry]
+    else:
+        assert entry == INV
+    return adj, deg, mask, entry
+
+
+def py_prune(base, p, cand, alpha, R):
+    """Textbook RobustPrune on exact integer distances (independent restatement used as a cross-check)."""
+    d = lambda a, b: int(((base[a].astype(np.int64) - base[b].astype(np.int64)) ** 2).sum())
+    C = sorted({c for c in cand if c != p}, key=lambda c: (d(p, c), c))
+    out = []
+    while C:
+        s = C.pop(0)
+        out.append(s)
+        if len(out) == R:
+            break
+        C = [c for c in C if not (alpha * d(s, c) <= d(p, c))]
+    return out
+
+
+def test_insert_batch_of_one_matches_sequential_textbook():
+    """Batch size 1 with L >= N: the search visits every reachable node, so the new node's row is
+    RobustPrune over all reachable nodes, and each reverse edge is an append or a prune of R+1."""
+    rng = np.random.default_rng(5)
+    n, d, R, alpha = 30, 3, 4, 2.0          # alpha = 2.0 is exact in fixed point
+    base = rng.integers(0, 64, (n, d)).astype(np.uint8)
+    o = mk(d, R=R, L=64, alpha=alpha, cap=n, vmax=1000)
+    rows = {}
+    o.insert_batch([0], base[:1])
+    rows[0] = []
+    for p in range(1, n):
+        o.insert_batch([p], base[p:p + 1])
+        # textbook: reachable set from the medoid (node 0 after a one-point bootstrap)
+        reach, stack = {0}, [0]
+        while stack:
+            for w in rows[stack.pop()]:
+                if w not in reach:
+                    reach.add(w); stack.append(w)
+        rows[p] = py_prune(base, p, reach, alpha, R)
+        for u in rows[p]:
+            if len(rows[u]) < R:
+                rows[u] = rows[u] + [p]
+            else:
+                rows[u] = py_prune(base, u, rows[u] + [p], alpha, R)
+        adj, deg, _, entry = o.export_graph()
+        assert entry == 0
+        for v in range(p + 1):
+            assert adj[v, :deg[v]].tolist() == rows[v], (p, v)
+
+
+def build_tiny(scale=0.3, R=16, L=32, perm_seed=None, **kw):
+    cfg = synth.scaled(synth.CONFIGS["tiny_u8_d32"], scale)
+    n = cfg["n"]
+    base = synth.uniform_u8(0, "base", 0, n, 32)
+    o = go.Oracle(32, go.U8, go.L2, R, L, 1.2, n, **kw)
+    rng = np.random.default_rng(perm_seed) if perm_seed is not None else None
+    b = cfg["first_batch"] // 2
+    for lo in range(0, n, b):
+        ids = np.arange(lo, min(n, lo + b), dtype=np.uint32)
+        if rng is not None:
+            ids = rng.permutation(ids).astype(np.uint32)
+        o.insert_batch(ids, base[ids])
+    return o, base, n
+
+
+def test_insert_invariants_and_batch_permutation_invariance():
+    o1, base, n = build_tiny()
+    a1 = check_invariants(o1, n)
+    o2, _, _ = build_tiny(perm_seed=7)
+    a2 = check_invariants(o2, n)
+    assert (a1[0] == a2[0]).all() and (a1[1] == a2[1]).all() and a1[3] == a2[3]
+    # thread count must not matter either
+    o3, _, _ = build_tiny(nthreads=1)
+    a3 = o3.export_graph()
+    assert (a1[0] == a3[0]).all() and (a1[1] == a3[1]).all()
+    assert o1.stats()["dead_edges_seen"] == 0
+
+
+def test_insert_errors_leave_index_unchanged():
+    o, base, n = build_tiny(scale=0.05)
+    before = o.export_graph()
+    for ids, code in [([3], -4), ([n + 5], -2)]:
+        with pytest.raises(go.OracleError) as e:
+            o.insert_batch(ids, base[:1])
+        assert e.value.code == code
+    o.delete_batch([3])
+    with pytest.raises(go.OracleError) as e:
+        o.insert_batch([3, 3], base[:2])
+    assert e.value.code == -3
+    with pytest.raises(go.OracleError) as e:
+        o.delete_batch([3])
+    assert e.value.code == -5
+    o.insert_batch([3], base[3:4])          # id reuse is legal
+    check_invariants(o, n)
+    assert before[3] == o.export_graph()[3]
+
+
+def test_scratch_capacity_keeps_P_nearest():
+    """A hub that receives more than P reverse-edge requests keeps the P smallest (dist, id)."""
+    # 1-D: hub at 0; existing nodes far away so every new point links to the hub.
+    d = 1
+    base = np.array([[0], [200], [210]] + [[10 + i] for i in range(12)], np.uint8)
+    o = mk(d, R=16, L=8, alpha=1000.0, cap=len(base), P=4)
+    o.insert_batch([0, 1, 2], base[:3])
+    o.insert_batch(np.arange(3, 15, dtype=np.uint32), base[3:15])
+    adj, deg, _, _ = o.export_graph()
+    hub = adj[0, :deg[0]].tolist()
+    assert hub[:2] == [1, 2] and hub[2:] == [3, 4, 5, 6]     # old order, then the 4 nearest requests
+
+
+# ------------------------------------------------------------------ batch delete (Alg. 6 + exact N_in)
+def test_delete_invariants_and_permutation_invariance():
+    outs = []
+    for perm in (None, 11):
+        o, base, n = build_tiny()
+        dele = synth.choose_ids(0, "del/0", np.arange(n, dtype=np.uint32), n // 10)
+        if perm is not None:
+            dele = np.random.default_rng(perm).permutation(dele).astype(np.uint32)
+        o.delete_batch(dele)
+        adj, deg, mask, entry = check_invariants(o, n - len(dele))
+        assert not mask[dele].any()
+        live_rows = adj[mask]
+        for v, dg in zip(np.flatnonzero(mask), deg[mask]):
+            assert not np.isin(adj[v, :dg], dele).any(), "edge to a deleted node survived"
+        q = synth.uniform_u8(0, "query", 0, 100, 32)
+        ids, _ = o.search(q, 10, 32)
+        assert not np.isin(ids, dele).any()
+        outs.append((adj.copy(), deg.copy(), entry))
+        assert o.stats()["dead_edges_seen"] == 0
+    assert (outs[0][0] == outs[1][0]).all() and (outs[0][1] == outs[1][1]).all() and outs[0][2] == outs[1][2]
+
+
+def test_delete_hand_case_line_graph():
+    """1-D points 0,10,20,30,40 (ids 0..4), R=2, chain rows.  Delete id 2 (x=20): in-neighbours {1,3},
+    out-neighbours {1,3}.  With c=1 and C_2 = nearest survivors of x=20: node 1 gains edge to 3 and
+    node 3 gains edge to 1 (both by in-repair and by out-repair, deduplicated)."""
+    base = (10 * np.arange(5))[:, None].astype(np.uint8)
+    o = mk(1, R=2, L=8, alpha=1.2, cap=5, c=1, k_repair=4)
+    rows = {0: [1], 1: [0, 2], 2: [1, 3], 3: [2, 4], 4: [3]}
+    load_graph(o, base, rows, entry=2)
+    o.delete_batch([2])
+    adj, deg, mask, entry = check_invariants(o, 4)
+    # C_2 = [(100,1),(100,3),(400,0),(400,4)]; z=1: closest of C\{1} to x=10 is id0 (100) -> 1 already has 0;
+    #   z=3: closest of C\{3} to x=30 is id4 (100) -> already present.
+    # out-repair w=1: closest y in C\{1} to x=10 is id0 -> request 0 -> 1 (already present);
+    #   w=3: closest y to x=30 is id4 -> request 4 -> 3 (already present).
+    assert adj[1, :deg[1]].tolist() == [0] and adj[3, :deg[3]].tolist() == [4]
+    assert adj[0, :deg[0]].tolist() == [1] and adj[4, :deg[4]].tolist() == [3]
+    assert entry == 1        # first repair candidate of the deleted medoid: (100, id1)
+    # c=2 adds the second-closest: z=1 gets {0,3}; z=3 gets {4,1} -> after dropping 2: [0,3] and [4,1]
+    o = mk(1, R=2, L=8, alpha=1.2, cap=5, c=2, k_repair=4)
+    load_graph(o, base, rows, entry=0)
+    o.delete_batch([2])
+    adj, deg, mask, entry = check_invariants(o, 4)
+    assert adj[1, :deg[1]].tolist() == [0, 3] and adj[3, :deg[3]].tolist() == [4, 1]
+    assert entry == 0
+
+
+def test_delete_everything_then_reinsert():
+    o, base, n = build_tiny(scale=0.05)
+    o.delete_batch(np.arange(n, dtype=np.uint32))
+    adj, deg, mask, entry = check_invariants(o, 0)
+    assert entry == INV
+    o.insert_batch(np.arange(n, dtype=np.uint32), base)
+    check_invariants(o, n)
+
+
+# ------------------------------------------------------------------ fixed-degree mode (Alg. 7 / 8)
+def test_fixed_degree_mode_invariants():
+    n, d, R = 1200, 16, 8
+    base = synth.aniso_unit_f32(0, "base", 0, n, d)
+    o = go.Oracle(d, go.F32, go.IP, R, 24, 1.2, n, mode=go.FIXED_DEGREE)
+    for lo in range(0, 1000, 200):
+        o.insert_batch(np.arange(lo, lo + 200, dtype=np.uint32), base[lo:lo + 200])
+    adj, deg, mask, entry = check_invariants(o, 1000)
+    assert (deg[mask] == R).all()                       # bootstrap fills rows, replacement keeps length
+    before = adj.copy()
+    o.insert_batch(np.arange(1000, 1200, dtype=np.uint32), base[1000:1200])
+    adj, deg, mask, entry = check_invariants(o, 1200)
+    new = set(range(1000, 1200))
+    # an old row changes only by replacing slots with new ids; at most once per slot
+    for v in range(1000):
+        diff = np.flatnonzero(before[v] != adj[v])
+        assert all(int(adj[v, s]) in new for s in diff)
+    # forward rows: the R nearest found, ascending key
+    for p in range(1000, 1010):
+        ds = [o.dist(base[p], base[w]) for w in adj[p, :deg[p]]]
+        assert ds == sorted(ds)
+    dele = synth.choose_ids(0, "del/0", np.arange(1200, dtype=np.uint32), 150)
+    o.delete_batch(dele)
+    adj, deg, mask, entry = check_invariants(o, 1050)
+    for v in np.flatnonzero(mask):
+        assert not np.isin(adj[v, :deg[v]], dele).any()
+
+
+def test_fixed_degree_delete_pick_one_hand_case():
+    """u=0 -> [1,2], p=1 -> [2,3,4] deleted.  N_in(1) = [0,5]; u=0 has rank 0 so the scan starts at
+    slot 0: 2 is already in N_out(0), 3 is free -> slot becomes 3.  u=5 -> [1] has rank 1, scan starts
+    at slot 1: 3 -> slot becomes 3."""
+    o = mk(1, dtype=go.F32, metric=go.IP, R=3, L=4, cap=6, mode=go.FIXED_DEGREE)
+    rows = {0: [1, 2], 1: [2, 3, 4], 2: [0], 3: [0], 4: [0], 5: [1]}
+    load_graph(o, np.zeros((6, 1), np.float32), rows, entry=0)
+    o.delete_batch([1])
+    adj, deg, mask, entry = check_invariants(o, 5)
+    assert adj[0, :deg[0]].tolist() == [3, 2]
+    assert adj[5, :deg[5]].tolist() == [3]
+
+
+# ------------------------------------------------------------------ end to end sanity
+def test_recall_sanity_band_tiny():
+    """Not a pin (the paper prints no recall for this set-up): the built index must be a usable one."""
+    o, base, n = build_tiny(scale=0.3, R=32, L=64)
+    dele = synth.choose_ids(0, "del/0", np.arange(n, dtype=np.uint32), n // 10)
+    o.delete_batch(dele)
+    live = np.setdiff1d(np.arange(n, dtype=np.uint32), dele)
+    q = synth.uniform_u8(0, "query", 0, 200, 32)
+    ids, _ = o.search(q, 10, 64)
+    hit = 0
+    for i in range(len(q)):
+        bi, _ = brute_knn(base, live, q[i], 10)
+        hit += len(set(bi.tolist()) & set(ids[i].tolist()))
+    assert hit / (10 * len(q)) > 0.9
