@@ -1,0 +1,157 @@
+/*
+ * grand.h -- C ABI of the B200 (sm_100a) library for batched dynamic maintenance and search of a
+ * Vamana-style proximity graph (GrAND).
+ *
+ * One handle = one index on one GPU = one mutator at a time.  The library owns the device-resident
+ * vector store (row stride padded to 16 B), the fixed-stride adjacency array uint32[capacity x R]
+ * with a degree counter per node, the live bitmap and a grow-only workspace pool; the caller owns
+ * every buffer it passes in, and the library keeps no caller pointer past a call.  Unless a
+ * function says "host", pointer arguments are DEVICE pointers, row-major and densely packed.
+ *
+ * Batch semantics are deterministic (one legal outcome of the lock-free scheme of Sec. 4): every
+ * search of a batch runs on the batch-start snapshot, reverse-edge candidates of one target merge
+ * in (distance, id) order, ties break by id.  Distances: L2 = squared Euclidean, IP = negated dot
+ * product; uint8/int8 vectors use exact int32 arithmetic, fp32 vectors accumulate in fp32.
+ *
+ * Errors: every function returns 0 (GRAND_OK) or a negative grand_status.  Update calls validate the
+ * whole batch on the device before mutating anything, so a failing call leaves the index unchanged.
+ * No exception crosses this boundary and there is no CPU fallback.
+ */
+#ifndef GRAND_H_
+#define GRAND_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct grand_index grand_index; /* opaque */
+typedef void* grand_stream;             /* a cudaStream_t; NULL = the default stream */
+
+typedef enum { GRAND_U8 = 0, GRAND_I8 = 1, GRAND_F32 = 2 } grand_dtype;
+typedef enum { GRAND_L2 = 0, GRAND_IP = 1 } grand_metric;
+typedef enum { GRAND_MODE_VAMANA = 0, GRAND_MODE_FIXED_DEGREE = 1 } grand_mode;
+
+typedef enum {
+  GRAND_OK = 0,
+  GRAND_ERR_INVALID_ARG = -1,  /* null pointer, k > L, parameter beyond a compile-time bound */
+  GRAND_ERR_CAPACITY = -2,     /* id >= capacity, or batch larger than max_batch */
+  GRAND_ERR_DUPLICATE_ID = -3, /* the same id twice in one batch */
+  GRAND_ERR_ALREADY_LIVE = -4, /* insert of a live id */
+  GRAND_ERR_NOT_LIVE = -5,     /* delete of an id that is not live */
+  GRAND_ERR_UNSUPPORTED = -6,  /* Vamana mode with the IP metric (alpha-pruning needs a metric) */
+  GRAND_ERR_CUDA = -7,         /* a CUDA call failed; text in grand_last_error */
+  GRAND_ERR_LIMIT = -8,        /* a bounded device loop hit its bound */
+  GRAND_ERR_NOMEM = -9         /* device allocation failed */
+} grand_status;
+
+#define GRAND_INVALID_ID 0xFFFFFFFFu
+#define GRAND_MAX_R 128u      /* degree bound limit */
+#define GRAND_MAX_L 512u      /* worklist size limit */
+#define GRAND_MAX_ROW_BYTES 4096u /* dim * sizeof(element), after padding to 16 B */
+
+/* Optional parameters; a zero field selects the default.  P, c and k follow the parameter list of
+ * Alg. 5 / Alg. 6 (scratch capacity, replacement edges per repair, repair candidates). */
+typedef struct {
+  uint64_t capacity;  /* peak number of ids N; ids live in [0, N-1]; default 1<<20; < 2^31 */
+  uint64_t max_batch; /* largest update batch; default 1<<17 */
+  uint32_t P;         /* reverse-edge candidates kept per target and batch; default 64; <= 256 */
+  uint32_t c;         /* replacement edges per repaired neighbour; default 2; <= 8 */
+  uint32_t k_repair;  /* repair candidates per deleted node; default min(50, L); <= 128 */
+  uint32_t vmax;      /* expansion cap of update searches; default 2*L; <= 1024 */
+  uint32_t mode;      /* grand_mode; default GRAND_MODE_VAMANA */
+  uint32_t hash_bits; /* log2 of the per-query visited cache; default 11; 10..13 */
+  /* device allocator hooks (default cudaMalloc / cudaFree); lets a host runtime pool the memory */
+  void* (*dev_alloc)(size_t bytes, void* user);
+  void (*dev_free)(void* ptr, void* user);
+  void* user;
+} grand_options;
+
+/* Counters since creation (or the last grand_reset_stats).  Times are accumulated only while
+ * profiling is on (grand_set_profiling), from CUDA events recorded on the caller's stream. */
+typedef struct {
+  uint64_t expansions;     /* worklist entries expanded by all beam searches */
+  uint64_t dist_evals;     /* query-to-node distances evaluated by beam searches */
+  uint64_t pair_dists;     /* node-to-node distances (prune, repair picks, rebuild) */
+  uint64_t dirty_nodes;    /* adjacency rows rebuilt */
+  uint64_t prunes;         /* RobustPrune invocations (forward + rebuild) */
+  uint64_t requests;       /* reverse-edge / repair requests grouped */
+  uint64_t kernel_launches;
+  uint64_t reserved;
+  double ms_search;        /* beam-search kernels (search, insert and delete searches) */
+  double ms_prune;         /* forward RobustPrune */
+  double ms_group;         /* request emission, grouping */
+  double ms_rebuild;       /* dirty-node rebuild */
+  double ms_transpose;     /* reverse-graph construction */
+  double ms_picks;         /* delete repair picks */
+  double ms_other;         /* validation, store write, publish / retire */
+  uint64_t n_search_launches;
+} grand_stats;
+
+/* Index life cycle (problem statement of Sec. 3-4: capacity fixed at initialisation, ids in
+ * [0, N-1], deleted ids reusable).  dim * sizeof(element) <= GRAND_MAX_ROW_BYTES, R <= GRAND_MAX_R,
+ * L <= GRAND_MAX_L.  The device current at creation owns the index. */
+int grand_create(uint32_t dim, uint32_t dtype, uint32_t metric, uint32_t R, uint32_t L, float alpha,
+                 grand_index** out);
+int grand_create_ex(uint32_t dim, uint32_t dtype, uint32_t metric, uint32_t R, uint32_t L, float alpha,
+                    const grand_options* opts, grand_index** out);
+int grand_destroy(grand_index* idx);
+
+/* BatchInsert (Alg. 5 in Vamana mode, Alg. 7 in fixed-degree mode).  ids_dev: n distinct non-live ids;
+ * vecs_dev: n x dim elements.  Work is enqueued on `stream`; the call returns after the batch is
+ * applied (it reads back one status block). */
+int grand_insert_batch(grand_index* idx, const uint32_t* ids_dev, const void* vecs_dev, uint64_t n,
+                       grand_stream stream);
+
+/* BatchDelete (Alg. 6 with in-neighbours from the on-demand CSR reverse graph of Alg. 8; Alg. 8 itself
+ * in fixed-degree mode).  ids_dev: n distinct live ids.  After the call no row holds a deleted id. */
+int grand_delete_batch(grand_index* idx, const uint32_t* ids_dev, uint64_t n, grand_stream stream);
+
+/* BeamSearch (Alg. 1) from the medoid with worklist size L (k <= L <= GRAND_MAX_L; expansion cap 2L).
+ * out_ids_dev: nq x k ids sorted by (distance, id), padded with GRAND_INVALID_ID; out_dists_dev: nq x k
+ * int32 (uint8/int8 vectors; padding INT32_MAX) or float (fp32 vectors; padding +inf).  Asynchronous
+ * on `stream`; concurrent searches on a quiescent index are allowed. */
+int grand_search(const grand_index* idx, const void* queries_dev, uint64_t nq, uint32_t k, uint32_t L,
+                 uint32_t* out_ids_dev, void* out_dists_dev, grand_stream stream);
+
+/* The same three calls with HOST buffers (pinned memory gives asynchronous copies): the host-to-device
+ * copy of the inputs and the device-to-host copy of the results happen inside the call, which returns
+ * after they complete. */
+int grand_insert_batch_host(grand_index* idx, const uint32_t* ids_host, const void* vecs_host, uint64_t n,
+                            grand_stream stream);
+int grand_delete_batch_host(grand_index* idx, const uint32_t* ids_host, uint64_t n, grand_stream stream);
+int grand_search_host(grand_index* idx, const void* queries_host, uint64_t nq, uint32_t k, uint32_t L,
+                      uint32_t* out_ids_host, void* out_dists_host, grand_stream stream);
+
+/* Introspection for parity checks and measurement.  Any output pointer may be NULL.
+ * adj_dev: capacity x R (unused slots hold GRAND_INVALID_ID); deg_dev: capacity; live_bitmap_dev:
+ * ceil(capacity/32) words, bit v%32 of word v/32; entry_out_host: HOST pointer to the medoid id. */
+int grand_export_graph(const grand_index* idx, uint32_t* adj_dev, uint32_t* deg_dev, uint32_t* live_bitmap_dev,
+                       uint32_t* entry_out_host, grand_stream stream);
+/* Replaces the whole state (tests only).  vecs_dev: capacity x dim packed elements. */
+int grand_import_graph(grand_index* idx, const uint32_t* adj_dev, const uint32_t* deg_dev,
+                       const uint32_t* live_bitmap_dev, uint32_t entry, const void* vecs_dev, grand_stream stream);
+/* Exact reverse graph in CSR (Alg. 8): off_dev has capacity+1 entries, row z of src_dev lists every live
+ * v with z in N_out(v), ascending.  src_dev needs room for capacity*R entries in the worst case;
+ * pass src_dev = NULL to obtain only offsets and *E_out_host (HOST pointer, total edges). */
+int grand_reverse_graph(grand_index* idx, uint32_t* off_dev, uint32_t* src_dev, uint64_t* E_out_host,
+                        grand_stream stream);
+
+int grand_get_entry(const grand_index* idx, uint32_t* entry_out_host);
+int grand_set_entry(grand_index* idx, uint32_t entry);
+int grand_live_count(const grand_index* idx, uint64_t* n_out_host);
+int grand_row_bytes(const grand_index* idx, uint32_t* row_bytes_out_host);
+
+int grand_get_stats(const grand_index* idx, grand_stats* out_host);
+int grand_reset_stats(grand_index* idx);
+int grand_set_profiling(grand_index* idx, int on);
+
+const char* grand_strerror(int status);
+const char* grand_last_error(const grand_index* idx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GRAND_H_ */

@@ -1,0 +1,679 @@
+// C-ABI entry points (include/grand.h) and the host orchestration of each batch call: argument
+// checks, workspace pool (allocated at creation, grow-only), the kernel sequence of one batch on
+// the caller's stream, and the single status read-back that ends an update call.
+#include <atomic>
+#include <cmath>
+#include <cstddef>
+#include <cstdio>
+#include <cstring>
+#include <string>
+#include <vector>
+
+#include "../../include/grand.h"
+#include "grand_kernels.h"
+
+namespace grand {
+
+static std::atomic<unsigned long long> g_launches{0};
+void count_launches(unsigned n) { g_launches += n; }
+unsigned long long launches_so_far() { return g_launches.load(); }
+
+Layout make_layout(uint32_t dim, uint32_t dtype, uint32_t metric) {
+  Layout l{};
+  l.dim = dim; l.dtype = dtype; l.metric = metric;
+  l.esize = dtype == GRAND_F32 ? 4 : 1;
+  l.row_bytes = (uint32_t)(((uint64_t)dim * l.esize + 15) / 16 * 16);
+  l.nchunk = l.row_bytes / 16;
+  static const int Gs[8] = {2, 8, 8, 8, 8, 32, 32, 32};
+  static const int Cs[8] = {1, 1, 2, 3, 4, 2, 4, 8};
+  static const uint32_t lim[8] = {2, 8, 16, 24, 32, 64, 128, 256};
+  l.code = -1;
+  for (int i = 0; i < 8; ++i)
+    if (l.nchunk <= lim[i]) { l.code = i; l.G = Gs[i]; l.CPL = Cs[i]; break; }
+  return l;
+}
+
+}  // namespace grand
+
+using namespace grand;
+
+enum Phase { PH_SEARCH = 0, PH_PRUNE, PH_GROUP, PH_REBUILD, PH_TRANSPOSE, PH_PICKS, PH_OTHER, PH_COUNT };
+
+struct Buf {
+  void* p = nullptr;
+  size_t bytes = 0;
+};
+
+struct grand_index {
+  Layout lay;
+  uint32_t R, L, P, c, k_repair, vmax, mode, hash_bits;
+  float alpha;
+  long long A_fix;
+  uint64_t cap, max_batch;
+  int device;
+  void* (*dev_alloc)(size_t, void*);
+  void (*dev_free)(void*, void*);
+  void* user;
+  // index state
+  uint8_t* store = nullptr;
+  uint32_t *adj = nullptr, *deg = nullptr, *live = nullptr;
+  DevState* d_state = nullptr;
+  DevState* h_state = nullptr;  // pinned mirror
+  uint32_t entry = GRAND_INVALID_ID;
+  uint64_t nlive = 0;
+  // workspace pool
+  uint32_t *mark = nullptr, *cnt = nullptr, *fill = nullptr, *start = nullptr, *flag = nullptr, *slot_of = nullptr;
+  unsigned long long* wk_keys = nullptr;  // max_batch x max(vmax, L): visited lists / worklists of update searches
+  uint32_t* wk_n = nullptr;
+  uint32_t wk_stride = 0;
+  unsigned long long* Ci = nullptr;
+  uint32_t *Ci_n = nullptr, *in_cnt = nullptr, *pair_off = nullptr, *scan_tmp = nullptr;
+  uint8_t* mean_row = nullptr;
+  Buf req_tgt, req_key, seg_keys, dirty;              // grow-only, sized by the number of requests
+  Buf t_indeg, t_off, t_fill, t_src;                  // reverse graph, allocated at the first delete
+  Buf st_ids, st_vecs, st_out_ids, st_out_d;          // staging of the *_host entry points
+  std::vector<void*> owned;
+  // stats
+  grand_stats stats{};
+  bool profiling = false;
+  std::vector<cudaEvent_t> ev_pool;
+  struct Span { int phase; cudaEvent_t a, b; };
+  std::vector<Span> spans;
+  size_t ev_used = 0;
+  std::string last_error;
+};
+
+namespace {
+
+int fail(const grand_index* idx, int code, const std::string& msg) {
+  if (idx) const_cast<grand_index*>(idx)->last_error = msg;
+  return code;
+}
+int cuda_fail(const grand_index* idx, cudaError_t e, const char* what) {
+  return fail(idx, GRAND_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
+}
+#define CK(call)                                                        \
+  do {                                                                  \
+    cudaError_t e__ = (call);                                           \
+    if (e__ != cudaSuccess) return cuda_fail(idx, e__, #call);          \
+  } while (0)
+
+void* default_alloc(size_t bytes, void*) {
+  void* p = nullptr;
+  if (cudaMalloc(&p, bytes) != cudaSuccess) return nullptr;
+  return p;
+}
+void default_free(void* p, void*) { cudaFree(p); }
+
+template <typename T>
+int alloc_dev(grand_index* idx, T** out, size_t count, bool zero) {
+  const size_t bytes = (count ? count : 1) * sizeof(T);
+  void* p = idx->dev_alloc(bytes, idx->user);
+  if (!p) return fail(idx, GRAND_ERR_NOMEM, "device allocation of " + std::to_string(bytes) + " bytes failed");
+  idx->owned.push_back(p);
+  if (zero) CK(cudaMemset(p, 0, bytes));
+  *out = reinterpret_cast<T*>(p);
+  return GRAND_OK;
+}
+int ensure(grand_index* idx, Buf& b, size_t bytes, cudaStream_t s) {
+  if (b.bytes >= bytes) return GRAND_OK;
+  if (b.p) {
+    CK(cudaStreamSynchronize(s));
+    idx->dev_free(b.p, idx->user);
+    b.p = nullptr;
+    b.bytes = 0;
+  }
+  size_t want = bytes + bytes / 4;
+  void* p = idx->dev_alloc(want, idx->user);
+  if (!p) return fail(idx, GRAND_ERR_NOMEM, "workspace growth to " + std::to_string(want) + " bytes failed");
+  b.p = p;
+  b.bytes = want;
+  return GRAND_OK;
+}
+
+GraphView view(const grand_index* idx) {
+  GraphView g;
+  g.store = idx->store; g.adj = idx->adj; g.deg = idx->deg; g.live = idx->live; g.R = idx->R; g.cap = idx->cap;
+  return g;
+}
+
+struct PhaseTimer {
+  grand_index* idx;
+  cudaStream_t s;
+  int phase;
+  cudaEvent_t a = nullptr, b = nullptr;
+  PhaseTimer(grand_index* i, cudaStream_t st, int ph) : idx(i), s(st), phase(ph) {
+    if (!idx->profiling) return;
+    while (idx->ev_pool.size() < idx->ev_used + 2) {
+      cudaEvent_t e;
+      cudaEventCreate(&e);
+      idx->ev_pool.push_back(e);
+    }
+    a = idx->ev_pool[idx->ev_used++];
+    b = idx->ev_pool[idx->ev_used++];
+    cudaEventRecord(a, s);
+  }
+  ~PhaseTimer() {
+    if (!a) return;
+    cudaEventRecord(b, s);
+    idx->spans.push_back({phase, a, b});
+  }
+};
+// after the stream is synchronised: fold recorded spans into the stats
+void collect_spans(grand_index* idx) {
+  for (auto& sp : idx->spans) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, sp.a, sp.b) != cudaSuccess) continue;
+    double* slot[PH_COUNT] = {&idx->stats.ms_search, &idx->stats.ms_prune, &idx->stats.ms_group, &idx->stats.ms_rebuild,
+                              &idx->stats.ms_transpose, &idx->stats.ms_picks, &idx->stats.ms_other};
+    *slot[sp.phase] += ms;
+  }
+  idx->spans.clear();
+  idx->ev_used = 0;
+}
+
+int read_state(grand_index* idx, cudaStream_t s) {
+  CK(cudaMemcpyAsync(idx->h_state, idx->d_state, sizeof(DevState), cudaMemcpyDeviceToHost, s));
+  CK(cudaStreamSynchronize(s));
+  return GRAND_OK;
+}
+int write_state_head(grand_index* idx, cudaStream_t s) {
+  // status, entry, ndirty, cursor, nlive, total_in: reset per call, counters untouched
+  idx->h_state->status = 0;
+  idx->h_state->entry = idx->entry;
+  idx->h_state->ndirty = 0;
+  idx->h_state->cursor = 0;
+  idx->h_state->nlive = idx->nlive;
+  idx->h_state->total_in = 0;
+  CK(cudaMemcpyAsync(idx->d_state, idx->h_state, offsetof(DevState, medoid_key), cudaMemcpyHostToDevice, s));
+  return GRAND_OK;
+}
+
+SearchArgs search_args(const grand_index* idx) {
+  SearchArgs a{};
+  a.lay = idx->lay;
+  a.g = view(idx);
+  a.entry = idx->entry;
+  a.hash_bits = idx->hash_bits;
+  a.state = idx->d_state;
+  return a;
+}
+
+int ensure_requests(grand_index* idx, uint64_t nreq, cudaStream_t s) {
+  int rc;
+  if ((rc = ensure(idx, idx->req_tgt, nreq * 4, s))) return rc;
+  if ((rc = ensure(idx, idx->req_key, nreq * 8, s))) return rc;
+  if ((rc = ensure(idx, idx->seg_keys, nreq * 8, s))) return rc;
+  if ((rc = ensure(idx, idx->dirty, nreq * 4, s))) return rc;
+  return GRAND_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* grand_strerror(int st) {
+  switch (st) {
+    case GRAND_OK: return "ok";
+    case GRAND_ERR_INVALID_ARG: return "invalid argument";
+    case GRAND_ERR_CAPACITY: return "id or batch size beyond capacity";
+    case GRAND_ERR_DUPLICATE_ID: return "duplicate id in batch";
+    case GRAND_ERR_ALREADY_LIVE: return "id is already live";
+    case GRAND_ERR_NOT_LIVE: return "id is not live";
+    case GRAND_ERR_UNSUPPORTED: return "unsupported configuration";
+    case GRAND_ERR_CUDA: return "CUDA error";
+    case GRAND_ERR_LIMIT: return "device loop limit reached";
+    case GRAND_ERR_NOMEM: return "device memory allocation failed";
+    default: return "unknown status";
+  }
+}
+const char* grand_last_error(const grand_index* idx) { return idx ? idx->last_error.c_str() : ""; }
+
+int grand_create(uint32_t dim, uint32_t dtype, uint32_t metric, uint32_t R, uint32_t L, float alpha, grand_index** out) {
+  return grand_create_ex(dim, dtype, metric, R, L, alpha, nullptr, out);
+}
+
+int grand_create_ex(uint32_t dim, uint32_t dtype, uint32_t metric, uint32_t R, uint32_t L, float alpha,
+                    const grand_options* o, grand_index** out) {
+  if (!out) return GRAND_ERR_INVALID_ARG;
+  *out = nullptr;
+  grand_options z{};
+  if (!o) o = &z;
+  if (dim == 0 || dtype > GRAND_F32 || metric > GRAND_IP || R == 0 || R > GRAND_MAX_R || L == 0 || L > GRAND_MAX_L ||
+      o->mode > GRAND_MODE_FIXED_DEGREE || !(alpha >= 1.0f))
+    return GRAND_ERR_INVALID_ARG;
+  if (o->mode == GRAND_MODE_VAMANA && metric == GRAND_IP) return GRAND_ERR_UNSUPPORTED;
+  Layout lay = make_layout(dim, dtype, metric);
+  if (lay.code < 0 || lay.row_bytes > GRAND_MAX_ROW_BYTES) return GRAND_ERR_INVALID_ARG;
+  grand_index* idx = new grand_index();
+  idx->lay = lay;
+  idx->R = R; idx->L = L; idx->alpha = alpha;
+  idx->A_fix = (long long)llround((double)alpha * 65536.0);
+  idx->cap = o->capacity ? o->capacity : (1ull << 20);
+  idx->max_batch = o->max_batch ? o->max_batch : (1ull << 17);
+  idx->P = o->P ? o->P : 64;
+  idx->c = o->c ? o->c : 2;
+  idx->k_repair = o->k_repair ? o->k_repair : (L < 50 ? L : 50);
+  idx->vmax = o->vmax ? o->vmax : 2 * L;
+  idx->mode = o->mode;
+  idx->hash_bits = o->hash_bits ? o->hash_bits : 11;
+  idx->dev_alloc = o->dev_alloc ? o->dev_alloc : default_alloc;
+  idx->dev_free = o->dev_free ? o->dev_free : default_free;
+  idx->user = o->user;
+  if (idx->cap >= (1ull << 31) || idx->cap * R >= (1ull << 32) || idx->P > 256 || idx->c > 8 || idx->k_repair > 128 ||
+      idx->k_repair > L || idx->vmax > 1024 || idx->vmax == 0 || idx->hash_bits < 10 || idx->hash_bits > 13 ||
+      idx->max_batch * R >= (1ull << 32)) {
+    delete idx;
+    return GRAND_ERR_INVALID_ARG;
+  }
+  cudaGetDevice(&idx->device);
+  const uint64_t cap = idx->cap, mb = idx->max_batch;
+  const size_t words = (cap + 31) / 32;
+  int rc = GRAND_OK;
+  auto A = [&](int r) { if (rc == GRAND_OK) rc = r; };
+  A(alloc_dev(idx, &idx->store, (size_t)cap * lay.row_bytes, true));
+  A(alloc_dev(idx, &idx->adj, (size_t)cap * R, false));
+  A(alloc_dev(idx, &idx->deg, cap, true));
+  A(alloc_dev(idx, &idx->live, words, true));
+  A(alloc_dev(idx, &idx->d_state, 1, true));
+  A(alloc_dev(idx, &idx->mark, words, true));
+  A(alloc_dev(idx, &idx->cnt, cap, true));
+  A(alloc_dev(idx, &idx->fill, cap, true));
+  A(alloc_dev(idx, &idx->start, cap, true));
+  A(alloc_dev(idx, &idx->flag, cap, true));
+  if (idx->mode == GRAND_MODE_FIXED_DEGREE) A(alloc_dev(idx, &idx->slot_of, cap, true));
+  idx->wk_stride = idx->vmax > L ? idx->vmax : L;
+  A(alloc_dev(idx, &idx->wk_keys, (size_t)mb * idx->wk_stride, false));
+  A(alloc_dev(idx, &idx->wk_n, mb, true));
+  A(alloc_dev(idx, &idx->Ci, (size_t)mb * idx->k_repair, false));
+  A(alloc_dev(idx, &idx->Ci_n, mb, true));
+  A(alloc_dev(idx, &idx->in_cnt, mb + 1, true));
+  A(alloc_dev(idx, &idx->pair_off, mb + 1, true));
+  A(alloc_dev(idx, &idx->scan_tmp, (cap + 1) / 2048 + mb / 2048 + 8, true));
+  A(alloc_dev(idx, &idx->mean_row, lay.row_bytes, true));
+  if (rc == GRAND_OK && cudaMemset(idx->adj, 0xFF, (size_t)cap * R * 4) != cudaSuccess) rc = GRAND_ERR_CUDA;
+  if (rc == GRAND_OK && cudaMallocHost(&idx->h_state, sizeof(DevState)) != cudaSuccess) rc = GRAND_ERR_CUDA;
+  if (rc == GRAND_OK) {
+    memset(idx->h_state, 0, sizeof(DevState));
+    idx->h_state->entry = GRAND_INVALID_ID;
+    if (cudaMemcpy(idx->d_state, idx->h_state, sizeof(DevState), cudaMemcpyHostToDevice) != cudaSuccess) rc = GRAND_ERR_CUDA;
+  }
+  if (rc == GRAND_OK) rc = ensure_requests(idx, mb * R, 0);
+  if (rc != GRAND_OK) {
+    grand_destroy(idx);
+    return rc;
+  }
+  *out = idx;
+  return GRAND_OK;
+}
+
+int grand_destroy(grand_index* idx) {
+  if (!idx) return GRAND_OK;
+  cudaDeviceSynchronize();
+  for (void* p : idx->owned) idx->dev_free(p, idx->user);
+  for (Buf* b : {&idx->req_tgt, &idx->req_key, &idx->seg_keys, &idx->dirty, &idx->t_indeg, &idx->t_off, &idx->t_fill, &idx->t_src,
+                 &idx->st_ids, &idx->st_vecs, &idx->st_out_ids, &idx->st_out_d})
+    if (b->p) idx->dev_free(b->p, idx->user);
+  if (idx->h_state) cudaFreeHost(idx->h_state);
+  for (auto e : idx->ev_pool) cudaEventDestroy(e);
+  delete idx;
+  return GRAND_OK;
+}
+
+int grand_insert_batch(grand_index* idx, const uint32_t* ids, const void* vecs, uint64_t n, grand_stream stream) {
+  if (!idx || (n && (!ids || !vecs))) return fail(idx, GRAND_ERR_INVALID_ARG, "null argument");
+  if (n == 0) return GRAND_OK;
+  if (n > idx->max_batch) return fail(idx, GRAND_ERR_CAPACITY, "batch larger than max_batch");
+  cudaStream_t s = (cudaStream_t)stream;
+  const bool fixed = idx->mode == GRAND_MODE_FIXED_DEGREE;
+  const uint32_t R = idx->R;
+  int rc;
+  if ((rc = write_state_head(idx, s))) return rc;
+  {
+    PhaseTimer pt(idx, s, PH_OTHER);
+    CK(launch_validate(ids, n, idx->cap, idx->live, idx->mark, 0, idx->d_state, s));
+  }
+  if ((rc = read_state(idx, s))) return rc;
+  if (idx->h_state->status != 0) {
+    CK(launch_clear_marks(ids, n, idx->cap, idx->mark, s));
+    CK(cudaStreamSynchronize(s));
+    collect_spans(idx);
+    return fail(idx, idx->h_state->status, grand_strerror(idx->h_state->status));
+  }
+  if ((rc = ensure_requests(idx, n * R, s))) return rc;
+  GraphView g = view(idx);
+  {
+    PhaseTimer pt(idx, s, PH_OTHER);
+    CK(launch_store_write(idx->lay, idx->store, idx->deg, idx->slot_of, ids, vecs, n, s));
+  }
+  const bool bootstrap = idx->nlive == 0;
+  {
+    // forward candidates: snapshot search (Alg. 5: visited list; Alg. 7: worklist) or bootstrap scan
+    PhaseTimer pt(idx, s, PH_SEARCH);
+    SearchArgs a = search_args(idx);
+    a.qids = ids;
+    a.nq = n;
+    a.L = idx->L;
+    a.vmax = idx->vmax;
+    if (bootstrap) {
+      a.boot_ids = ids;
+      a.boot_n = (uint32_t)n;
+      a.out_vis = idx->wk_keys; a.out_vis_n = idx->wk_n; a.vis_stride = idx->wk_stride;
+    } else if (fixed) {
+      a.out_beam = idx->wk_keys; a.out_beam_n = idx->wk_n; a.beam_stride = idx->wk_stride;
+    } else {
+      a.out_vis = idx->wk_keys; a.out_vis_n = idx->wk_n; a.vis_stride = idx->wk_stride;
+    }
+    CK(launch_beam_search(a, s));
+    idx->stats.n_search_launches++;
+  }
+  {
+    PhaseTimer pt(idx, s, PH_PRUNE);
+    PruneArgs a{};
+    a.lay = idx->lay; a.g = g; a.A_fix = idx->A_fix; a.alpha = idx->alpha;
+    a.ids = ids; a.n = n;
+    a.cand = idx->wk_keys; a.cand_n = idx->wk_n; a.cand_stride = idx->wk_stride;
+    a.fixed_mode = fixed;
+    a.req_tgt = (uint32_t*)idx->req_tgt.p; a.req_key = (unsigned long long*)idx->req_key.p;
+    a.state = idx->d_state;
+    CK(launch_forward_prune(a, s));
+  }
+  {
+    PhaseTimer pt(idx, s, PH_GROUP);
+    GroupArgs a{};
+    a.req_tgt = (uint32_t*)idx->req_tgt.p; a.req_key = (unsigned long long*)idx->req_key.p; a.nreq = n * R;
+    a.cnt = idx->cnt; a.fill = idx->fill; a.start = idx->start; a.flag = idx->flag;
+    a.dirty = (uint32_t*)idx->dirty.p; a.seg_keys = (unsigned long long*)idx->seg_keys.p; a.state = idx->d_state;
+    CK(launch_group_requests(a, s));
+  }
+  {
+    PhaseTimer pt(idx, s, PH_REBUILD);
+    const uint64_t mbk = n * R < 148u * 16u ? n * R : 148u * 16u;
+    if (fixed) {
+      FixedReverseArgs a{};
+      a.g = g; a.slot_of = idx->slot_of; a.fwd_rows = (uint32_t*)idx->req_tgt.p;
+      a.cnt = idx->cnt; a.fill = idx->fill; a.start = idx->start; a.flag = idx->flag;
+      a.dirty = (uint32_t*)idx->dirty.p; a.seg_keys = (unsigned long long*)idx->seg_keys.p;
+      a.max_blocks = (uint32_t)mbk; a.state = idx->d_state;
+      CK(launch_fixed_reverse(a, s));
+    } else {
+      RebuildArgs a{};
+      a.lay = idx->lay; a.g = g; a.A_fix = idx->A_fix; a.alpha = idx->alpha; a.P = idx->P; a.delmap = nullptr;
+      a.cnt = idx->cnt; a.fill = idx->fill; a.start = idx->start; a.flag = idx->flag;
+      a.dirty = (uint32_t*)idx->dirty.p; a.seg_keys = (unsigned long long*)idx->seg_keys.p;
+      a.max_blocks = (uint32_t)mbk; a.state = idx->d_state;
+      CK(launch_rebuild(a, s));
+    }
+  }
+  {
+    PhaseTimer pt(idx, s, PH_OTHER);
+    CK(launch_publish(ids, n, idx->live, idx->mark, idx->d_state, s));
+    if (idx->entry == GRAND_INVALID_ID) CK(launch_pick_medoid(idx->lay, g, ids, n, idx->mean_row, idx->d_state, s));
+  }
+  if ((rc = read_state(idx, s))) return rc;
+  collect_spans(idx);
+  idx->entry = idx->h_state->entry;
+  idx->nlive = idx->h_state->nlive;
+  if (idx->h_state->status != 0) return fail(idx, idx->h_state->status, grand_strerror(idx->h_state->status));
+  return GRAND_OK;
+}
+
+static int build_reverse(grand_index* idx, bool sort_rows, cudaStream_t s) {
+  int rc;
+  const uint64_t cap = idx->cap;
+  if ((rc = ensure(idx, idx->t_indeg, (cap + 1) * 4, s))) return rc;
+  if ((rc = ensure(idx, idx->t_off, (cap + 1) * 4, s))) return rc;
+  if ((rc = ensure(idx, idx->t_fill, cap * 4, s))) return rc;
+  if ((rc = ensure(idx, idx->t_src, cap * idx->R * 4, s))) return rc;
+  TransposeArgs t{};
+  t.g = view(idx);
+  t.indeg = (uint32_t*)idx->t_indeg.p; t.off = (uint32_t*)idx->t_off.p; t.fillc = (uint32_t*)idx->t_fill.p;
+  t.src = (uint32_t*)idx->t_src.p; t.scan_tmp = idx->scan_tmp; t.sort_rows = sort_rows;
+  CK(launch_transpose(t, s));
+  return GRAND_OK;
+}
+
+int grand_delete_batch(grand_index* idx, const uint32_t* ids, uint64_t n, grand_stream stream) {
+  if (!idx || (n && !ids)) return fail(idx, GRAND_ERR_INVALID_ARG, "null argument");
+  if (n == 0) return GRAND_OK;
+  if (n > idx->max_batch) return fail(idx, GRAND_ERR_CAPACITY, "batch larger than max_batch");
+  cudaStream_t s = (cudaStream_t)stream;
+  const bool fixed = idx->mode == GRAND_MODE_FIXED_DEGREE;
+  const uint32_t R = idx->R;
+  int rc;
+  if ((rc = write_state_head(idx, s))) return rc;
+  {
+    PhaseTimer pt(idx, s, PH_OTHER);
+    CK(launch_validate(ids, n, idx->cap, idx->live, idx->mark, 1, idx->d_state, s));
+  }
+  GraphView g = view(idx);
+  DeleteArgs d{};
+  d.lay = idx->lay; d.g = g; d.ids = ids; d.n = n; d.delmap = idx->mark;
+  d.beam = idx->wk_keys; d.beam_n = idx->wk_n; d.beam_stride = idx->wk_stride;
+  d.Ci = idx->Ci; d.Ci_n = idx->Ci_n; d.k_repair = idx->k_repair; d.c = idx->c;
+  d.in_cnt = idx->in_cnt; d.pair_off = idx->pair_off; d.scan_tmp = idx->scan_tmp;
+  d.flag = idx->flag; d.state = idx->d_state;
+  {
+    // reverse graph of the snapshot: exact in-neighbours, rebuilt per batch and not kept
+    PhaseTimer pt(idx, s, PH_TRANSPOSE);
+    if ((rc = build_reverse(idx, false, s))) return rc;
+    d.off = (uint32_t*)idx->t_off.p; d.src = (uint32_t*)idx->t_src.p;
+    CK(launch_delete_prepare(d, s));
+  }
+  if ((rc = read_state(idx, s))) return rc;
+  if (idx->h_state->status != 0) {
+    CK(launch_clear_marks(ids, n, idx->cap, idx->mark, s));
+    CK(cudaStreamSynchronize(s));
+    collect_spans(idx);
+    return fail(idx, idx->h_state->status, grand_strerror(idx->h_state->status));
+  }
+  const uint64_t total_in = idx->h_state->total_in;
+  const uint64_t nreq = fixed ? total_in + 1 : (total_in + n * R) * idx->c;
+  if (nreq >= (1ull << 32)) return fail(idx, GRAND_ERR_CAPACITY, "delete batch touches too many edges");
+  if ((rc = ensure_requests(idx, nreq, s))) return rc;
+  d.req_tgt = (uint32_t*)idx->req_tgt.p; d.req_key = (unsigned long long*)idx->req_key.p; d.dirty = (uint32_t*)idx->dirty.p;
+  if (fixed) {
+    PhaseTimer pt(idx, s, PH_REBUILD);
+    FixedDeleteArgs f{};
+    f.g = g; f.ids = ids; f.n = n; f.delmap = idx->mark; f.off = d.off; f.src = d.src; f.pair_off = idx->pair_off;
+    f.flag = idx->flag; f.dirty = (uint32_t*)idx->dirty.p; f.state = idx->d_state;
+    CK(launch_fixed_delete(f, total_in, s));
+  } else {
+    {
+      PhaseTimer pt(idx, s, PH_SEARCH);
+      SearchArgs a = search_args(idx);
+      a.qids = ids; a.nq = n; a.L = idx->L; a.vmax = idx->vmax;
+      a.out_beam = idx->wk_keys; a.out_beam_n = idx->wk_n; a.beam_stride = idx->wk_stride;
+      CK(launch_beam_search(a, s));
+      idx->stats.n_search_launches++;
+    }
+    {
+      PhaseTimer pt(idx, s, PH_PICKS);
+      CK(launch_delete_ci(d, s));
+      CK(launch_delete_picks(d, total_in, s));
+    }
+    {
+      PhaseTimer pt(idx, s, PH_GROUP);
+      GroupArgs a{};
+      a.req_tgt = d.req_tgt; a.req_key = d.req_key; a.nreq = nreq;
+      a.cnt = idx->cnt; a.fill = idx->fill; a.start = idx->start; a.flag = idx->flag;
+      a.dirty = d.dirty; a.seg_keys = (unsigned long long*)idx->seg_keys.p; a.state = idx->d_state;
+      CK(launch_group_requests(a, s));
+    }
+    {
+      PhaseTimer pt(idx, s, PH_REBUILD);
+      RebuildArgs a{};
+      a.lay = idx->lay; a.g = g; a.A_fix = idx->A_fix; a.alpha = idx->alpha; a.P = idx->P; a.delmap = idx->mark;
+      a.cnt = idx->cnt; a.fill = idx->fill; a.start = idx->start; a.flag = idx->flag;
+      a.dirty = d.dirty; a.seg_keys = (unsigned long long*)idx->seg_keys.p;
+      a.max_blocks = (uint32_t)(nreq < 148u * 16u ? nreq : 148u * 16u); a.state = idx->d_state;
+      CK(launch_rebuild(a, s));
+    }
+  }
+  {
+    PhaseTimer pt(idx, s, PH_OTHER);
+    CK(launch_retire(g, ids, n, idx->mark, idx->Ci, idx->Ci_n, idx->k_repair, fixed, idx->d_state, s));
+  }
+  if ((rc = read_state(idx, s))) return rc;
+  collect_spans(idx);
+  idx->entry = idx->h_state->entry;
+  idx->nlive = idx->h_state->nlive;
+  if (idx->h_state->status != 0) return fail(idx, idx->h_state->status, grand_strerror(idx->h_state->status));
+  return GRAND_OK;
+}
+
+int grand_search(const grand_index* cidx, const void* queries, uint64_t nq, uint32_t k, uint32_t L, uint32_t* out_ids,
+                 void* out_dists, grand_stream stream) {
+  grand_index* idx = const_cast<grand_index*>(cidx);
+  if (!idx || (nq && (!queries || !out_ids))) return fail(idx, GRAND_ERR_INVALID_ARG, "null argument");
+  if (k == 0 || k > L || L > GRAND_MAX_L) return fail(idx, GRAND_ERR_INVALID_ARG, "need 1 <= k <= L <= GRAND_MAX_L");
+  if (nq == 0) return GRAND_OK;
+  cudaStream_t s = (cudaStream_t)stream;
+  {
+    PhaseTimer pt(idx, s, PH_SEARCH);
+    SearchArgs a = search_args(idx);
+    a.queries = queries; a.nq = nq; a.L = L; a.vmax = 2 * L; a.k = k;
+    a.out_ids = out_ids; a.out_dists = out_dists;
+    CK(launch_beam_search(a, s));
+    idx->stats.n_search_launches++;
+  }
+  if (idx->profiling) {
+    CK(cudaStreamSynchronize(s));
+    collect_spans(idx);
+  }
+  return GRAND_OK;
+}
+
+// ---- host-buffer variants: copies inside the call
+int grand_insert_batch_host(grand_index* idx, const uint32_t* ids, const void* vecs, uint64_t n, grand_stream stream) {
+  if (!idx || (n && (!ids || !vecs))) return fail(idx, GRAND_ERR_INVALID_ARG, "null argument");
+  if (n == 0) return GRAND_OK;
+  cudaStream_t s = (cudaStream_t)stream;
+  int rc;
+  const size_t vb = (size_t)n * idx->lay.dim * idx->lay.esize;
+  if ((rc = ensure(idx, idx->st_ids, n * 4, s))) return rc;
+  if ((rc = ensure(idx, idx->st_vecs, vb, s))) return rc;
+  CK(cudaMemcpyAsync(idx->st_ids.p, ids, n * 4, cudaMemcpyHostToDevice, s));
+  CK(cudaMemcpyAsync(idx->st_vecs.p, vecs, vb, cudaMemcpyHostToDevice, s));
+  return grand_insert_batch(idx, (const uint32_t*)idx->st_ids.p, idx->st_vecs.p, n, stream);
+}
+int grand_delete_batch_host(grand_index* idx, const uint32_t* ids, uint64_t n, grand_stream stream) {
+  if (!idx || (n && !ids)) return fail(idx, GRAND_ERR_INVALID_ARG, "null argument");
+  if (n == 0) return GRAND_OK;
+  cudaStream_t s = (cudaStream_t)stream;
+  int rc;
+  if ((rc = ensure(idx, idx->st_ids, n * 4, s))) return rc;
+  CK(cudaMemcpyAsync(idx->st_ids.p, ids, n * 4, cudaMemcpyHostToDevice, s));
+  return grand_delete_batch(idx, (const uint32_t*)idx->st_ids.p, n, stream);
+}
+int grand_search_host(grand_index* idx, const void* queries, uint64_t nq, uint32_t k, uint32_t L, uint32_t* out_ids,
+                      void* out_dists, grand_stream stream) {
+  if (!idx || (nq && (!queries || !out_ids))) return fail(idx, GRAND_ERR_INVALID_ARG, "null argument");
+  if (nq == 0) return GRAND_OK;
+  cudaStream_t s = (cudaStream_t)stream;
+  int rc;
+  const size_t qb = (size_t)nq * idx->lay.dim * idx->lay.esize;
+  if ((rc = ensure(idx, idx->st_vecs, qb, s))) return rc;
+  if ((rc = ensure(idx, idx->st_out_ids, nq * k * 4, s))) return rc;
+  if ((rc = ensure(idx, idx->st_out_d, nq * k * 4, s))) return rc;
+  CK(cudaMemcpyAsync(idx->st_vecs.p, queries, qb, cudaMemcpyHostToDevice, s));
+  if ((rc = grand_search(idx, idx->st_vecs.p, nq, k, L, (uint32_t*)idx->st_out_ids.p, idx->st_out_d.p, stream))) return rc;
+  CK(cudaMemcpyAsync(out_ids, idx->st_out_ids.p, nq * k * 4, cudaMemcpyDeviceToHost, s));
+  if (out_dists) CK(cudaMemcpyAsync(out_dists, idx->st_out_d.p, nq * k * 4, cudaMemcpyDeviceToHost, s));
+  CK(cudaStreamSynchronize(s));
+  return GRAND_OK;
+}
+
+// ---- introspection
+int grand_export_graph(const grand_index* idx, uint32_t* adj, uint32_t* deg, uint32_t* live, uint32_t* entry_out, grand_stream stream) {
+  if (!idx) return GRAND_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (adj) CK(cudaMemcpyAsync(adj, idx->adj, (size_t)idx->cap * idx->R * 4, cudaMemcpyDeviceToDevice, s));
+  if (deg) CK(cudaMemcpyAsync(deg, idx->deg, idx->cap * 4, cudaMemcpyDeviceToDevice, s));
+  if (live) CK(cudaMemcpyAsync(live, idx->live, (idx->cap + 31) / 32 * 4, cudaMemcpyDeviceToDevice, s));
+  if (entry_out) *entry_out = idx->entry;
+  return GRAND_OK;
+}
+int grand_import_graph(grand_index* idx, const uint32_t* adj, const uint32_t* deg, const uint32_t* live, uint32_t entry,
+                       const void* vecs, grand_stream stream) {
+  if (!idx || !adj || !deg || !live || !vecs) return fail(idx, GRAND_ERR_INVALID_ARG, "null argument");
+  cudaStream_t s = (cudaStream_t)stream;
+  CK(cudaMemcpyAsync(idx->adj, adj, (size_t)idx->cap * idx->R * 4, cudaMemcpyDeviceToDevice, s));
+  CK(cudaMemcpyAsync(idx->deg, deg, idx->cap * 4, cudaMemcpyDeviceToDevice, s));
+  CK(cudaMemcpyAsync(idx->live, live, (idx->cap + 31) / 32 * 4, cudaMemcpyDeviceToDevice, s));
+  CK(launch_pad_rows(idx->lay, idx->store, vecs, idx->cap, s));
+  idx->entry = entry;
+  idx->nlive = 0;
+  int rc;
+  if ((rc = write_state_head(idx, s))) return rc;
+  CK(launch_count_live(idx->live, idx->cap, idx->d_state, s));
+  if ((rc = read_state(idx, s))) return rc;
+  idx->nlive = idx->h_state->nlive;
+  return GRAND_OK;
+}
+int grand_reverse_graph(grand_index* idx, uint32_t* off, uint32_t* src, uint64_t* E_out, grand_stream stream) {
+  if (!idx) return GRAND_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  int rc;
+  if ((rc = build_reverse(idx, true, s))) return rc;
+  uint32_t E = 0;
+  CK(cudaMemcpyAsync(&E, (uint32_t*)idx->t_off.p + idx->cap, 4, cudaMemcpyDeviceToHost, s));
+  CK(cudaStreamSynchronize(s));
+  if (off) CK(cudaMemcpyAsync(off, idx->t_off.p, (idx->cap + 1) * 4, cudaMemcpyDeviceToDevice, s));
+  if (src && E) CK(cudaMemcpyAsync(src, idx->t_src.p, (size_t)E * 4, cudaMemcpyDeviceToDevice, s));
+  if (E_out) *E_out = E;
+  CK(cudaStreamSynchronize(s));
+  return GRAND_OK;
+}
+
+int grand_get_entry(const grand_index* idx, uint32_t* e) {
+  if (!idx || !e) return GRAND_ERR_INVALID_ARG;
+  *e = idx->entry;
+  return GRAND_OK;
+}
+int grand_set_entry(grand_index* idx, uint32_t e) {
+  if (!idx || (e != GRAND_INVALID_ID && e >= idx->cap)) return GRAND_ERR_INVALID_ARG;
+  idx->entry = e;
+  return GRAND_OK;
+}
+int grand_live_count(const grand_index* idx, uint64_t* n) {
+  if (!idx || !n) return GRAND_ERR_INVALID_ARG;
+  *n = idx->nlive;
+  return GRAND_OK;
+}
+int grand_row_bytes(const grand_index* idx, uint32_t* rb) {
+  if (!idx || !rb) return GRAND_ERR_INVALID_ARG;
+  *rb = idx->lay.row_bytes;
+  return GRAND_OK;
+}
+
+int grand_get_stats(const grand_index* cidx, grand_stats* out) {
+  grand_index* idx = const_cast<grand_index*>(cidx);
+  if (!idx || !out) return GRAND_ERR_INVALID_ARG;
+  DevState st;
+  CK(cudaMemcpy(&st, idx->d_state, sizeof(DevState), cudaMemcpyDeviceToHost));
+  idx->stats.expansions = st.counters[CTR_EXP];
+  idx->stats.dist_evals = st.counters[CTR_DIST];
+  idx->stats.pair_dists = st.counters[CTR_PAIR];
+  idx->stats.dirty_nodes = st.counters[CTR_DIRTY];
+  idx->stats.prunes = st.counters[CTR_PRUNE];
+  idx->stats.requests = st.counters[CTR_REQ];
+  idx->stats.kernel_launches = launches_so_far();
+  *out = idx->stats;
+  return GRAND_OK;
+}
+int grand_reset_stats(grand_index* idx) {
+  if (!idx) return GRAND_ERR_INVALID_ARG;
+  CK(cudaMemset(idx->d_state->counters, 0, sizeof(idx->d_state->counters)));
+  const uint64_t keep = idx->stats.kernel_launches;
+  idx->stats = grand_stats{};
+  idx->stats.kernel_launches = keep;
+  return GRAND_OK;
+}
+int grand_set_profiling(grand_index* idx, int on) {
+  if (!idx) return GRAND_ERR_INVALID_ARG;
+  idx->profiling = on != 0;
+  return GRAND_OK;
+}
+
+}  // extern "C"

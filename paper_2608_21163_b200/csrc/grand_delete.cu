@@ -1,0 +1,333 @@
+// Delete-repair kernels (Alg. 6 with exact in-neighbours, Alg. 8 in fixed-degree mode) and the
+// initial-medoid choice.  The work is flattened over (deleted node, in-neighbour) and (deleted
+// node, out-slot) pairs so that hubs with a long in-neighbour row do not serialise a block.
+#include "grand_common.cuh"
+#include "grand_kernels.h"
+
+namespace grand {
+
+constexpr int kPickWarps = 4;
+constexpr uint32_t kMaxKRepair = 128;
+constexpr uint32_t kMaxC = 8;
+
+__device__ __forceinline__ void touch_dirty2(uint32_t* flag, uint32_t* dirty, DevState* st, uint32_t u) {
+  if (atomicExch(&flag[u], 1u) == 0u) dirty[atomicAdd(&st->ndirty, 1u)] = u;
+}
+
+// in_cnt[i] = in-degree of p_i in the reverse graph (0 for an id that fails validation), then the
+// prefix over the batch and the total number of (deleted node, in-neighbour) pairs.
+__global__ void delete_incnt_kernel(const DeleteArgs a) {
+  for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i <= a.n; i += (uint64_t)gridDim.x * blockDim.x) {
+    uint32_t c = 0;
+    if (i < a.n) {
+      const uint32_t p = a.ids[i];
+      if (p < a.g.cap) c = a.off[p + 1] - a.off[p];
+    }
+    a.in_cnt[i] = c;
+  }
+}
+__global__ void delete_total_kernel(const uint32_t* pair_off, uint64_t n, DevState* st) { st->total_in = pair_off[n]; }
+
+cudaError_t launch_delete_prepare(const DeleteArgs& a, cudaStream_t s) {
+  const unsigned blocks = (unsigned)((a.n + 256) / 256 > 148u * 16u ? 148u * 16u : (a.n + 256) / 256);
+  delete_incnt_kernel<<<blocks, 256, 0, s>>>(a);
+  cudaError_t e = launch_exclusive_scan(a.in_cnt, a.pair_off, a.n + 1, a.scan_tmp, s);
+  if (e != cudaSuccess) return e;
+  delete_total_kernel<<<1, 1, 0, s>>>(a.pair_off, a.n, a.state);
+  count_launches(2);
+  return cudaGetLastError();
+}
+
+// C_i = first k_repair worklist entries of the per-deleted search that are not in the batch.
+__global__ void delete_ci_kernel(const DeleteArgs a) {
+  constexpr unsigned FULL = 0xFFFFFFFFu;
+  const int lane = threadIdx.x & 31;
+  const uint64_t wglobal = (blockIdx.x * (uint64_t)blockDim.x + threadIdx.x) >> 5;
+  const uint64_t wtotal = ((uint64_t)gridDim.x * blockDim.x) >> 5;
+  for (uint64_t i = wglobal; i < a.n; i += wtotal) {
+    const uint32_t nb = min(a.beam_n[i], a.beam_stride);
+    uint32_t nc = 0;
+    for (uint32_t jb = 0; jb < nb && nc < a.k_repair; jb += 32) {
+      const uint32_t j = jb + lane;
+      unsigned long long k = 0;
+      bool ok = false;
+      if (j < nb) {
+        k = a.beam[i * a.beam_stride + j];
+        ok = !bit_test(a.delmap, key_id(k));
+      }
+      const unsigned bal = __ballot_sync(FULL, ok);
+      const uint32_t pos = nc + __popc(bal & ((1u << lane) - 1u));
+      if (ok && pos < a.k_repair) a.Ci[i * a.k_repair + pos] = k;
+      nc += __popc(bal);
+    }
+    if (lane == 0) a.Ci_n[i] = min(nc, a.k_repair);
+  }
+}
+cudaError_t launch_delete_ci(const DeleteArgs& a, cudaStream_t s) {
+  const unsigned blocks = (unsigned)((a.n + 3) / 4 > 148u * 16u ? 148u * 16u : (a.n + 3) / 4);
+  delete_ci_kernel<<<blocks ? blocks : 1, 128, 0, s>>>(a);
+  count_launches(1);
+  return cudaGetLastError();
+}
+
+// One warp per pair.  In-pair (p_i, z): z gets the c members of C_i \ {z} closest to z (requests
+// z <- y).  Out-pair (p_i, w): the c members y of C_i \ {w} closest to w each get w (requests y <- w).
+template <typename T, int METRIC, int G, int CPL>
+__global__ void __launch_bounds__(kPickWarps * 32) delete_picks_kernel(const DeleteArgs a, const uint64_t total_in) {
+  using Dist = typename Elem<T>::Dist;
+  constexpr unsigned FULL = 0xFFFFFFFFu;
+  constexpr int NT = 32 / G;
+  __shared__ unsigned long long keys_s[kPickWarps][kMaxKRepair];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int t = lane % G, team = lane / G;
+  unsigned long long* keys = keys_s[warp];
+  const uint32_t R = a.g.R, c = a.c;
+  const uint32_t row_bytes = a.lay.row_bytes, nchunk = a.lay.nchunk;
+  const uint64_t total = total_in + a.n * R;
+  const uint64_t wglobal = (uint64_t)blockIdx.x * kPickWarps + warp, wtotal = (uint64_t)gridDim.x * kPickWarps;
+  unsigned long long npair = 0;
+  for (uint64_t pair = wglobal; pair < total; pair += wtotal) {
+    const bool is_in = pair < total_in;
+    uint64_t i;
+    uint32_t x = kInvalid;
+    if (is_in) {
+      uint64_t lo = 0, hi = a.n;  // largest i with pair_off[i] <= pair
+      while (hi - lo > 1) {
+        const uint64_t mid = (lo + hi) >> 1;
+        if (a.pair_off[mid] <= pair) lo = mid; else hi = mid;
+      }
+      i = lo;
+      x = a.src[a.off[a.ids[i]] + (uint32_t)(pair - a.pair_off[i])];
+    } else {
+      const uint64_t o = pair - total_in;
+      i = o / R;
+      const uint32_t s = (uint32_t)(o - i * R);
+      const uint32_t p = a.ids[i];
+      if (s < a.g.deg[p]) x = a.g.adj[(size_t)p * R + s];
+    }
+    const bool act = x != kInvalid && !bit_test(a.delmap, x);
+    const uint64_t rbase = pair * c;
+    if (!act) {
+      if (lane < c) a.req_tgt[rbase + lane] = kInvalid;
+      continue;
+    }
+    if (is_in && lane == 0) touch_dirty2(a.flag, a.dirty, a.state, x);  // dirty even without a candidate
+    uint4 xr[CPL];
+    load_row<G, CPL>(a.g.store + (size_t)x * row_bytes, nchunk, t, xr);
+    const uint32_t nc = a.Ci_n[i];
+    for (uint32_t jb = 0; jb < nc; jb += NT) {
+      const uint32_t j = jb + team;
+      uint32_t y = kInvalid;
+      if (j < nc) y = key_id(a.Ci[i * a.k_repair + j]);
+      const bool go = y != kInvalid && y != x;
+      uint4 v[CPL];
+      if (go) {
+        load_row<G, CPL>(a.g.store + (size_t)y * row_bytes, nchunk, t, v);
+      } else {
+#pragma unroll
+        for (int cc = 0; cc < CPL; ++cc) v[cc] = make_uint4(0, 0, 0, 0);
+      }
+      const Dist d = team_dist_regs<T, kMetricL2, G, CPL>(xr, v);
+      if (t == 0 && j < nc) {
+        keys[j] = go ? make_key(d, y) : kKeyMax;
+        npair += go;
+      }
+    }
+    __syncwarp();
+    for (uint32_t r = 0; r < c; ++r) {  // r-th smallest (dist, id)
+      unsigned long long best = kKeyMax;
+      for (uint32_t j = lane; j < nc; j += 32) best = min(best, keys[j]);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) best = min(best, __shfl_xor_sync(FULL, best, o));
+      if (best != kKeyMax) {
+        for (uint32_t j = lane; j < nc; j += 32)
+          if (keys[j] == best) keys[j] = kKeyMax;
+      }
+      if (lane == 0) {
+        if (best == kKeyMax) {
+          a.req_tgt[rbase + r] = kInvalid;
+        } else if (is_in) {
+          a.req_tgt[rbase + r] = x;
+          a.req_key[rbase + r] = best;
+        } else {
+          a.req_tgt[rbase + r] = key_id(best);
+          a.req_key[rbase + r] = (best & 0xFFFFFFFF00000000ull) | x;
+        }
+      }
+      __syncwarp();
+    }
+  }
+  if (npair) atomicAdd(&a.state->counters[CTR_PAIR], npair);
+}
+template <typename T, int METRIC, int G, int CPL>
+static cudaError_t launch_delete_picks_t(const DeleteArgs& a, uint64_t total_in, cudaStream_t s) {
+  const uint64_t total = total_in + a.n * a.g.R;
+  if (total == 0) return cudaSuccess;
+  uint64_t blocks = (total + kPickWarps - 1) / kPickWarps;
+  if (blocks > 148u * 16u) blocks = 148u * 16u;
+  delete_picks_kernel<T, METRIC, G, CPL><<<(unsigned)blocks, kPickWarps * 32, 0, s>>>(a, total_in);
+  count_launches(1);
+  return cudaGetLastError();
+}
+cudaError_t launch_delete_picks(const DeleteArgs& a, uint64_t total_in, cudaStream_t s) {
+  GRAND_DISPATCH_L2(a.lay, launch_delete_picks_t, a, total_in, s);
+  return cudaErrorInvalidValue;
+}
+
+// ---- fixed-degree delete (Alg. 8): mark every surviving in-neighbour of a deleted node dirty, then
+// one warp per dirty node rewrites its deleted slots in slot order with PickOne.
+__global__ void fixed_delete_mark_kernel(const FixedDeleteArgs a, const uint64_t total_in) {
+  for (uint64_t pair = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; pair < total_in; pair += (uint64_t)gridDim.x * blockDim.x) {
+    uint64_t lo = 0, hi = a.n;
+    while (hi - lo > 1) {
+      const uint64_t mid = (lo + hi) >> 1;
+      if (a.pair_off[mid] <= pair) lo = mid; else hi = mid;
+    }
+    const uint32_t u = a.src[a.off[a.ids[lo]] + (uint32_t)(pair - a.pair_off[lo])];
+    if (!bit_test(a.delmap, u)) touch_dirty2(a.flag, a.dirty, a.state, u);
+  }
+}
+__global__ void __launch_bounds__(128) fixed_delete_rewire_kernel(const FixedDeleteArgs a) {
+  constexpr unsigned FULL = 0xFFFFFFFFu;
+  constexpr uint32_t kMaxR = 128;
+  __shared__ uint32_t rows[4][kMaxR];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint32_t* row = rows[warp];
+  const uint32_t R = a.g.R;
+  const uint32_t nd = a.state->ndirty;
+  const uint64_t wglobal = (uint64_t)blockIdx.x * 4 + warp, wtotal = (uint64_t)gridDim.x * 4;
+  uint32_t ndone = 0;
+  for (uint64_t k = wglobal; k < nd; k += wtotal) {
+    const uint32_t u = a.dirty[k];
+    const uint32_t du = min(a.g.deg[u], R);
+    for (uint32_t s = lane; s < du; s += 32) row[s] = a.g.adj[(size_t)u * R + s];
+    __syncwarp();
+    for (uint32_t s = 0; s < du; ++s) {
+      const uint32_t p = row[s];
+      if (p == kInvalid || !bit_test(a.delmap, p)) continue;  // warp-uniform
+      // round-robin offset: rank of u among the in-neighbours of p
+      const uint32_t b = a.off[p], e = a.off[p + 1];
+      uint32_t rank = 0;
+      for (uint32_t jb = b; jb < e; jb += 32) {
+        const uint32_t j = jb + lane;
+        rank += __popc(__ballot_sync(FULL, j < e && a.src[j] < u));
+      }
+      const uint32_t np = min(a.g.deg[p], R);
+      uint32_t chosen = kInvalid;
+      for (uint32_t tt = 0; tt < np && chosen == kInvalid; ++tt) {
+        const uint32_t cand = a.g.adj[(size_t)p * R + (rank + tt) % np];
+        if (bit_test(a.delmap, cand) || cand == u) continue;
+        bool inrow = false;
+        for (uint32_t sb = 0; sb < du; sb += 32) inrow |= __any_sync(FULL, sb + lane < du && row[sb + lane] == cand);
+        if (!inrow) chosen = cand;
+      }
+      __syncwarp();
+      if (lane == 0) row[s] = chosen;
+      __syncwarp();
+    }
+    // stable compaction of the surviving slots
+    uint32_t w = 0;
+    for (uint32_t sb = 0; sb < R; sb += 32) {
+      const uint32_t s = sb + lane;
+      const uint32_t v = s < du ? row[s] : kInvalid;
+      const bool ok = v != kInvalid;
+      const unsigned bal = __ballot_sync(FULL, ok);
+      if (ok) a.g.adj[(size_t)u * R + w + __popc(bal & ((1u << lane) - 1u))] = v;
+      w += __popc(bal);
+    }
+    for (uint32_t s = w + lane; s < R; s += 32) a.g.adj[(size_t)u * R + s] = kInvalid;
+    if (lane == 0) {
+      a.g.deg[u] = w;
+      a.flag[u] = 0;
+      ++ndone;
+    }
+    __syncwarp();
+  }
+  if (lane == 0 && ndone) atomicAdd(&a.state->counters[CTR_DIRTY], (unsigned long long)ndone);
+}
+cudaError_t launch_fixed_delete(const FixedDeleteArgs& a, uint64_t total_in, cudaStream_t s) {
+  if (total_in) {
+    uint64_t blocks = (total_in + 255) / 256;
+    if (blocks > 148u * 32u) blocks = 148u * 32u;
+    fixed_delete_mark_kernel<<<(unsigned)blocks, 256, 0, s>>>(a, total_in);
+    count_launches(1);
+  }
+  fixed_delete_rewire_kernel<<<148 * 8, 128, 0, s>>>(a);
+  count_launches(1);
+  return cudaGetLastError();
+}
+
+// ---- initial medoid: the batch point closest to the per-dimension mean (ties by id)
+template <typename T>
+__global__ void medoid_mean_kernel(const uint8_t* store, const uint32_t* ids, uint64_t n, uint32_t dim, uint32_t row_bytes,
+                                   uint8_t* mean_row) {
+  const uint32_t per_row = row_bytes / sizeof(T);
+  for (uint32_t j = blockIdx.x * blockDim.x + threadIdx.x; j < per_row; j += gridDim.x * blockDim.x) {
+    T m = T(0);
+    if (j < dim) {
+      if constexpr (sizeof(T) == 4) {
+        double s = 0.0;
+        for (uint64_t i = 0; i < n; ++i) s += (double)reinterpret_cast<const float*>(store + (size_t)ids[i] * row_bytes)[j];
+        m = (float)(s / (double)n);
+      } else {
+        long long s = 0;
+        for (uint64_t i = 0; i < n; ++i) s += (long long)reinterpret_cast<const T*>(store + (size_t)ids[i] * row_bytes)[j];
+        const long long num = 2 * s + (long long)n, den = 2 * (long long)n;  // round-half-up via floor division
+        long long q = num / den;
+        if (num % den != 0 && num < 0) --q;
+        m = (T)q;
+      }
+    }
+    reinterpret_cast<T*>(mean_row)[j] = m;
+  }
+}
+template <typename T, int METRIC, int G, int CPL>
+__global__ void medoid_argmin_kernel(const uint8_t* store, const uint32_t* ids, uint64_t n, uint32_t row_bytes, uint32_t nchunk,
+                                     const uint8_t* mean_row, DevState* st) {
+  using Dist = typename Elem<T>::Dist;
+  constexpr int NT = 32 / G;
+  const int lane = threadIdx.x & 31;
+  const int t = lane % G, team = lane / G;
+  uint4 mr[CPL];
+  load_row<G, CPL>(mean_row, nchunk, t, mr);
+  const uint64_t wglobal = (blockIdx.x * (uint64_t)blockDim.x + threadIdx.x) >> 5;
+  const uint64_t wtotal = ((uint64_t)gridDim.x * blockDim.x) >> 5;
+  for (uint64_t b0 = wglobal * NT; b0 < n; b0 += wtotal * NT) {
+    const uint64_t i = b0 + team;
+    uint4 v[CPL];
+    uint32_t id = kInvalid;
+    if (i < n) {
+      id = ids[i];
+      load_row<G, CPL>(store + (size_t)id * row_bytes, nchunk, t, v);
+    } else {
+#pragma unroll
+      for (int c = 0; c < CPL; ++c) v[c] = make_uint4(0, 0, 0, 0);
+    }
+    const Dist d = team_dist_regs<T, METRIC, G, CPL>(v, mr);
+    if (t == 0 && id != kInvalid) atomicMin(&st->medoid_key, make_key(d, id));
+  }
+}
+__global__ void medoid_begin_kernel(DevState* st) { st->medoid_key = kKeyMax; }
+__global__ void medoid_end_kernel(DevState* st) {
+  if (st->medoid_key != kKeyMax) st->entry = key_id(st->medoid_key);
+}
+template <typename T, int METRIC, int G, int CPL>
+static cudaError_t launch_pick_medoid_t(const Layout& lay, const GraphView& g, const uint32_t* ids, uint64_t n, uint8_t* mean_row,
+                                        DevState* st, cudaStream_t s) {
+  medoid_begin_kernel<<<1, 1, 0, s>>>(st);
+  medoid_mean_kernel<T><<<(lay.row_bytes / sizeof(T) + 127) / 128, 128, 0, s>>>(g.store, ids, n, lay.dim, lay.row_bytes, mean_row);
+  uint64_t blocks = (n + 3) / 4;
+  if (blocks > 148u * 8u) blocks = 148u * 8u;
+  if (blocks < 1) blocks = 1;
+  medoid_argmin_kernel<T, METRIC, G, CPL><<<(unsigned)blocks, 128, 0, s>>>(g.store, ids, n, lay.row_bytes, lay.nchunk, mean_row, st);
+  medoid_end_kernel<<<1, 1, 0, s>>>(st);
+  count_launches(4);
+  return cudaGetLastError();
+}
+cudaError_t launch_pick_medoid(const Layout& lay, const GraphView& g, const uint32_t* ids, uint64_t n, uint8_t* mean_row,
+                               DevState* st, cudaStream_t s) {
+  GRAND_DISPATCH_ALL(lay, launch_pick_medoid_t, lay, g, ids, n, mean_row, st, s);
+  return cudaErrorInvalidValue;
+}
+
+}  // namespace grand

@@ -1,0 +1,372 @@
+// Integer plumbing kernels: grouping of reverse-edge / repair requests by target (the stand-in for
+// the per-node scratch buffers of Alg. 5/6), the on-demand reverse graph (Alg. 8: histogram ->
+// exclusive scan -> scatter, CSR), batch validation, store writes and live-set bookkeeping.
+#include "grand_common.cuh"
+#include "grand_kernels.h"
+
+namespace grand {
+
+constexpr int kThreads = 256;
+static inline unsigned grid_for(uint64_t n, int threads = kThreads, unsigned maxb = 148u * 32u) {
+  uint64_t b = (n + threads - 1) / threads;
+  if (b < 1) b = 1;
+  return (unsigned)(b > maxb ? maxb : b);
+}
+
+__device__ __forceinline__ void touch_dirty(uint32_t* flag, uint32_t* dirty, DevState* st, uint32_t u) {
+  if (atomicExch(&flag[u], 1u) == 0u) dirty[atomicAdd(&st->ndirty, 1u)] = u;
+}
+
+// ---- request grouping: count per target (first touch appends to the dirty list), allocate one
+// segment per dirty target from a global cursor, scatter keys into the segments.
+__global__ void group_count_kernel(const GroupArgs a) {
+  unsigned long long nv = 0;
+  for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < a.nreq; i += (uint64_t)gridDim.x * blockDim.x) {
+    const uint32_t tg = a.req_tgt[i];
+    if (tg == kInvalid) continue;
+    atomicAdd(&a.cnt[tg], 1u);
+    touch_dirty(a.flag, a.dirty, a.state, tg);
+    ++nv;
+  }
+  if (nv) atomicAdd(&a.state->counters[CTR_REQ], nv);
+}
+__global__ void group_alloc_kernel(const GroupArgs a) {
+  const uint32_t nd = a.state->ndirty;
+  for (uint32_t k = blockIdx.x * blockDim.x + threadIdx.x; k < nd; k += gridDim.x * blockDim.x) {
+    const uint32_t u = a.dirty[k];
+    a.start[u] = atomicAdd(&a.state->cursor, a.cnt[u]);
+  }
+}
+__global__ void group_scatter_kernel(const GroupArgs a) {
+  for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < a.nreq; i += (uint64_t)gridDim.x * blockDim.x) {
+    const uint32_t tg = a.req_tgt[i];
+    if (tg == kInvalid) continue;
+    a.seg_keys[a.start[tg] + atomicAdd(&a.fill[tg], 1u)] = a.req_key[i];
+  }
+}
+cudaError_t launch_group_requests(const GroupArgs& a, cudaStream_t s) {
+  if (a.nreq) group_count_kernel<<<grid_for(a.nreq), kThreads, 0, s>>>(a);
+  group_alloc_kernel<<<grid_for(a.nreq ? a.nreq : 1), kThreads, 0, s>>>(a);
+  if (a.nreq) group_scatter_kernel<<<grid_for(a.nreq), kThreads, 0, s>>>(a);
+  count_launches(a.nreq ? 3 : 1);
+  return cudaGetLastError();
+}
+
+// ---- exclusive scan of uint32 (three phases; 2048 elements per block)
+constexpr int kScanThreads = 256, kScanPer = 8, kScanBlock = kScanThreads * kScanPer;
+
+__device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* sh, uint32_t* total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint32_t inc = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+    if (lane >= o) inc += y;
+  }
+  if (lane == 31) sh[warp] = inc;
+  __syncthreads();
+  if (warp == 0) {
+    uint32_t w = lane < (int)(blockDim.x >> 5) ? sh[lane] : 0u;
+    uint32_t winc = w;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, winc, o);
+      if (lane >= o) winc += y;
+    }
+    sh[32 + lane] = winc - w;
+    if (lane == 31) sh[64] = winc;
+  }
+  __syncthreads();
+  const uint32_t r = sh[32 + warp] + inc - v;
+  *total = sh[64];
+  __syncthreads();
+  return r;
+}
+
+__global__ void __launch_bounds__(kScanThreads) scan_sums_kernel(const uint32_t* in, uint64_t n, uint32_t* sums) {
+  __shared__ uint32_t sh[65];
+  const uint64_t base = (uint64_t)blockIdx.x * kScanBlock + (uint64_t)threadIdx.x * kScanPer;
+  uint32_t s = 0;
+#pragma unroll
+  for (int j = 0; j < kScanPer; ++j) s += base + j < n ? in[base + j] : 0u;
+  uint32_t total;
+  block_exclusive_scan(s, sh, &total);
+  if (threadIdx.x == 0) sums[blockIdx.x] = total;
+}
+__global__ void __launch_bounds__(kScanThreads) scan_top_kernel(uint32_t* sums, uint32_t nblocks) {
+  __shared__ uint32_t sh[65];
+  uint32_t carry = 0;
+  for (uint32_t b0 = 0; b0 < nblocks; b0 += kScanThreads) {
+    const uint32_t i = b0 + threadIdx.x;
+    const uint32_t v = i < nblocks ? sums[i] : 0u;
+    uint32_t total;
+    const uint32_t ex = block_exclusive_scan(v, sh, &total);
+    if (i < nblocks) sums[i] = carry + ex;
+    carry += total;
+  }
+}
+__global__ void __launch_bounds__(kScanThreads) scan_final_kernel(const uint32_t* in, uint32_t* out, uint64_t n, const uint32_t* sums) {
+  __shared__ uint32_t sh[65];
+  const uint64_t base = (uint64_t)blockIdx.x * kScanBlock + (uint64_t)threadIdx.x * kScanPer;
+  uint32_t v[kScanPer];
+  uint32_t s = 0;
+#pragma unroll
+  for (int j = 0; j < kScanPer; ++j) {
+    v[j] = base + j < n ? in[base + j] : 0u;
+    s += v[j];
+  }
+  uint32_t total;
+  uint32_t ex = block_exclusive_scan(s, sh, &total) + sums[blockIdx.x];
+#pragma unroll
+  for (int j = 0; j < kScanPer; ++j) {
+    if (base + j < n) out[base + j] = ex;
+    ex += v[j];
+  }
+}
+cudaError_t launch_exclusive_scan(const uint32_t* in, uint32_t* out, uint64_t n, uint32_t* tmp, cudaStream_t s) {
+  if (n == 0) return cudaSuccess;
+  const uint32_t nblocks = (uint32_t)((n + kScanBlock - 1) / kScanBlock);
+  scan_sums_kernel<<<nblocks, kScanThreads, 0, s>>>(in, n, tmp);
+  scan_top_kernel<<<1, kScanThreads, 0, s>>>(tmp, nblocks);
+  scan_final_kernel<<<nblocks, kScanThreads, 0, s>>>(in, out, n, tmp);
+  count_launches(3);
+  return cudaGetLastError();
+}
+
+// ---- reverse graph
+__global__ void transpose_hist_kernel(const GraphView g, uint32_t* indeg) {
+  const uint64_t total = g.cap * g.R;
+  for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < total; i += (uint64_t)gridDim.x * blockDim.x) {
+    const uint64_t v = i / g.R;
+    const uint32_t s = (uint32_t)(i - v * g.R);
+    if (s < g.deg[v]) atomicAdd(&indeg[g.adj[i]], 1u);
+  }
+}
+__global__ void transpose_scatter_kernel(const GraphView g, const uint32_t* off, uint32_t* fillc, uint32_t* src) {
+  const uint64_t total = g.cap * g.R;
+  for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < total; i += (uint64_t)gridDim.x * blockDim.x) {
+    const uint64_t v = i / g.R;
+    const uint32_t s = (uint32_t)(i - v * g.R);
+    if (s < g.deg[v]) {
+      const uint32_t z = g.adj[i];
+      src[off[z] + atomicAdd(&fillc[z], 1u)] = (uint32_t)v;
+    }
+  }
+}
+// ascending rows: shared-memory sort for short rows, in place in global memory for long ones
+__global__ void __launch_bounds__(128) transpose_sort_rows_kernel(uint64_t cap, const uint32_t* off, uint32_t* src) {
+  constexpr uint32_t kRowCap = 4096;
+  __shared__ uint32_t sh[kRowCap];
+  auto sync = [] { __syncthreads(); };
+  for (uint64_t z = blockIdx.x; z < cap; z += gridDim.x) {
+    const uint32_t b = off[z], n = off[z + 1] - b;
+    if (n < 2) continue;
+    if (n <= kRowCap) {
+      for (uint32_t j = threadIdx.x; j < n; j += blockDim.x) sh[j] = src[b + j];
+      __syncthreads();
+      bitonic_sort_any(sh, n, threadIdx.x, blockDim.x, sync);
+      for (uint32_t j = threadIdx.x; j < n; j += blockDim.x) src[b + j] = sh[j];
+      __syncthreads();
+    } else {
+      bitonic_sort_any(src + b, n, threadIdx.x, blockDim.x, sync);
+    }
+  }
+}
+cudaError_t launch_transpose(const TransposeArgs& a, cudaStream_t s) {
+  const uint64_t cap = a.g.cap;
+  cudaMemsetAsync(a.indeg, 0, (cap + 1) * 4, s);
+  transpose_hist_kernel<<<grid_for(cap * a.g.R), kThreads, 0, s>>>(a.g, a.indeg);
+  count_launches(1);
+  cudaError_t e = launch_exclusive_scan(a.indeg, a.off, cap + 1, a.scan_tmp, s);
+  if (e != cudaSuccess) return e;
+  if (a.src) {
+    cudaMemsetAsync(a.fillc, 0, cap * 4, s);
+    transpose_scatter_kernel<<<grid_for(cap * a.g.R), kThreads, 0, s>>>(a.g, a.off, a.fillc, a.src);
+    count_launches(a.sort_rows ? 2 : 1);
+    if (a.sort_rows) transpose_sort_rows_kernel<<<(unsigned)(cap < 148u * 16u ? cap : 148u * 16u), 128, 0, s>>>(cap, a.off, a.src);
+  }
+  return cudaGetLastError();
+}
+
+// ---- validation: ids < capacity, liveness as required, no repeated id (bitmap atomics)
+__device__ __forceinline__ void set_status(DevState* st, int code) { atomicMin(&st->status, code); }
+
+__global__ void validate_range_kernel(const uint32_t* ids, uint64_t n, uint64_t cap, DevState* st) {
+  for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < n; i += (uint64_t)gridDim.x * blockDim.x)
+    if (ids[i] >= cap) set_status(st, -2);
+}
+__global__ void validate_mark_kernel(const uint32_t* ids, uint64_t n, uint64_t cap, const uint32_t* live, uint32_t* mark,
+                                     int want_live, DevState* st) {
+  for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < n; i += (uint64_t)gridDim.x * blockDim.x) {
+    const uint32_t v = ids[i];
+    if (v >= cap) continue;
+    const uint32_t bit = 1u << (v & 31);
+    if (atomicOr(&mark[v >> 5], bit) & bit) set_status(st, -3);
+  }
+}
+__global__ void validate_live_kernel(const uint32_t* ids, uint64_t n, uint64_t cap, const uint32_t* live, int want_live, DevState* st) {
+  for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < n; i += (uint64_t)gridDim.x * blockDim.x) {
+    const uint32_t v = ids[i];
+    if (v >= cap) continue;
+    const bool is_live = bit_test(live, v);
+    // error precedence (capacity, duplicate, liveness) mirrors a sequential check of the whole batch
+    if (want_live && !is_live) atomicCAS(&st->status, 0, -5);
+    if (!want_live && is_live) atomicCAS(&st->status, 0, -4);
+  }
+}
+cudaError_t launch_validate(const uint32_t* ids, uint64_t n, uint64_t cap, const uint32_t* live, uint32_t* mark, int want_live,
+                            DevState* st, cudaStream_t s) {
+  validate_range_kernel<<<grid_for(n), kThreads, 0, s>>>(ids, n, cap, st);
+  validate_mark_kernel<<<grid_for(n), kThreads, 0, s>>>(ids, n, cap, live, mark, want_live, st);
+  validate_live_kernel<<<grid_for(n), kThreads, 0, s>>>(ids, n, cap, live, want_live, st);
+  count_launches(3);
+  return cudaGetLastError();
+}
+__global__ void clear_marks_kernel(const uint32_t* ids, uint64_t n, uint64_t cap, uint32_t* mark) {
+  for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < n; i += (uint64_t)gridDim.x * blockDim.x) {
+    const uint32_t v = ids[i];
+    if (v < cap) atomicAnd(&mark[v >> 5], ~(1u << (v & 31)));
+  }
+}
+cudaError_t launch_clear_marks(const uint32_t* ids, uint64_t n, uint64_t cap, uint32_t* mark, cudaStream_t s) {
+  clear_marks_kernel<<<grid_for(n), kThreads, 0, s>>>(ids, n, cap, mark);
+  count_launches(1);
+  return cudaGetLastError();
+}
+
+// ---- store write: re-stride packed vectors into 16-byte padded rows, zero the padding, deg <- 0
+template <typename T>
+__global__ void store_write_kernel(uint8_t* store, uint32_t* deg, uint32_t* slot_of, const uint32_t* ids, const T* vecs,
+                                   uint64_t n, uint32_t dim, uint32_t row_bytes) {
+  const uint32_t per_row = row_bytes / sizeof(T);
+  const uint64_t total = n * per_row;
+  for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < total; i += (uint64_t)gridDim.x * blockDim.x) {
+    const uint64_t r = i / per_row;
+    const uint32_t j = (uint32_t)(i - r * per_row);
+    const uint64_t dst_row = ids ? ids[r] : r;
+    reinterpret_cast<T*>(store + dst_row * row_bytes)[j] = j < dim ? vecs[r * dim + j] : T(0);
+    if (j == 0 && ids) {
+      if (deg) deg[dst_row] = 0;
+      if (slot_of) slot_of[dst_row] = (uint32_t)r;
+    }
+  }
+}
+cudaError_t launch_store_write(const Layout& lay, uint8_t* store, uint32_t* deg, uint32_t* slot_of, const uint32_t* ids,
+                               const void* vecs, uint64_t n, cudaStream_t s) {
+  if (n == 0) return cudaSuccess;
+  const uint64_t total = n * (lay.row_bytes / lay.esize);
+  if (lay.esize == 4)
+    store_write_kernel<float><<<grid_for(total), kThreads, 0, s>>>(store, deg, slot_of, ids, (const float*)vecs, n, lay.dim, lay.row_bytes);
+  else
+    store_write_kernel<uint8_t><<<grid_for(total), kThreads, 0, s>>>(store, deg, slot_of, ids, (const uint8_t*)vecs, n, lay.dim, lay.row_bytes);
+  count_launches(1);
+  return cudaGetLastError();
+}
+cudaError_t launch_pad_rows(const Layout& lay, uint8_t* store, const void* vecs, uint64_t n, cudaStream_t s) {
+  return launch_store_write(lay, store, nullptr, nullptr, nullptr, vecs, n, s);
+}
+
+// ---- publish (insert epilogue): live bits on, batch marks off
+__global__ void publish_kernel(const uint32_t* ids, uint64_t n, uint32_t* live, uint32_t* mark, DevState* st) {
+  for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < n; i += (uint64_t)gridDim.x * blockDim.x) {
+    const uint32_t v = ids[i];
+    atomicOr(&live[v >> 5], 1u << (v & 31));
+    atomicAnd(&mark[v >> 5], ~(1u << (v & 31)));
+  }
+  if (blockIdx.x == 0 && threadIdx.x == 0) st->nlive += n;
+}
+cudaError_t launch_publish(const uint32_t* ids, uint64_t n, uint32_t* live, uint32_t* mark, DevState* st, cudaStream_t s) {
+  publish_kernel<<<grid_for(n), kThreads, 0, s>>>(ids, n, live, mark, st);
+  count_launches(1);
+  return cudaGetLastError();
+}
+
+// ---- retire (delete epilogue): choose a new medoid if the old one is deleted, clear rows and bits
+__global__ void __launch_bounds__(256) new_entry_kernel(const GraphView g, const uint32_t* ids, uint64_t n, const uint32_t* delmap,
+                                                        const unsigned long long* Ci, const uint32_t* Ci_n, uint32_t k_repair,
+                                                        uint32_t fixed_mode, DevState* st) {
+  const uint32_t m = st->entry;
+  if (m == kInvalid || !bit_test(delmap, m)) return;
+  __shared__ uint32_t found;
+  if (threadIdx.x == 0) found = kInvalid;
+  __syncthreads();
+  if (fixed_mode) {  // first surviving out-neighbour of the old medoid (rows are nearest-first)
+    if (threadIdx.x == 0) {
+      const uint32_t d = min(g.deg[m], g.R);
+      for (uint32_t s = 0; s < d; ++s) {
+        const uint32_t v = g.adj[(size_t)m * g.R + s];
+        if (!bit_test(delmap, v)) {
+          found = v;
+          break;
+        }
+      }
+    }
+  } else {  // first repair candidate of the deleted medoid
+    for (uint64_t i = threadIdx.x; i < n; i += blockDim.x)
+      if (ids[i] == m && Ci_n[i] > 0) found = key_id(Ci[i * k_repair]);
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) st->entry = found;  // kInvalid -> smallest live id, resolved after the bits are cleared
+}
+__global__ void retire_kernel(const GraphView g, const uint32_t* ids, uint64_t n, uint32_t* delmap, DevState* st) {
+  const uint64_t total = n * g.R;
+  for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < total; i += (uint64_t)gridDim.x * blockDim.x) {
+    const uint64_t r = i / g.R;
+    const uint32_t s = (uint32_t)(i - r * g.R);
+    const uint32_t p = ids[r];
+    g.adj[(size_t)p * g.R + s] = kInvalid;
+    if (s == 0) {
+      g.deg[p] = 0;
+      atomicAnd(&g.live[p >> 5], ~(1u << (p & 31)));
+      atomicAnd(&delmap[p >> 5], ~(1u << (p & 31)));
+    }
+  }
+  if (blockIdx.x == 0 && threadIdx.x == 0) st->nlive -= n;
+}
+__global__ void fallback_entry_kernel(const uint32_t* live, uint64_t nwords, DevState* st, uint32_t* scratch_min) {
+  // runs only when the medoid was deleted without a replacement candidate
+  for (uint64_t w = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; w < nwords; w += (uint64_t)gridDim.x * blockDim.x) {
+    const uint32_t x = live[w];
+    if (x) atomicMin(scratch_min, (uint32_t)(w * 32 + __ffs(x) - 1));
+  }
+}
+__global__ void fallback_entry_begin(DevState* st, uint32_t* scratch_min) {
+  scratch_min[0] = kInvalid;
+  scratch_min[1] = st->entry == kInvalid ? 1u : 0u;
+}
+__global__ void fallback_entry_end(DevState* st, const uint32_t* scratch_min) {
+  if (scratch_min[1]) st->entry = scratch_min[0];
+}
+cudaError_t launch_retire(const GraphView& g, const uint32_t* ids, uint64_t n, uint32_t* delmap, const unsigned long long* Ci,
+                          const uint32_t* Ci_n, uint32_t k_repair, uint32_t fixed_mode, DevState* st, cudaStream_t s) {
+  new_entry_kernel<<<1, 256, 0, s>>>(g, ids, n, delmap, Ci, Ci_n, k_repair, fixed_mode, st);
+  retire_kernel<<<grid_for(n * g.R), kThreads, 0, s>>>(g, ids, n, delmap, st);
+  // smallest live id as the last resort (cheap: one pass over the bitmap); scratch = medoid_key words
+  uint32_t* scratch = reinterpret_cast<uint32_t*>(&st->medoid_key);
+  fallback_entry_begin<<<1, 1, 0, s>>>(st, scratch);
+  fallback_entry_kernel<<<grid_for((g.cap + 31) / 32), kThreads, 0, s>>>(g.live, (g.cap + 31) / 32, st, scratch);
+  fallback_entry_end<<<1, 1, 0, s>>>(st, scratch);
+  count_launches(5);
+  return cudaGetLastError();
+}
+
+__global__ void count_live_kernel(const uint32_t* live, uint64_t nwords, DevState* st) {
+  unsigned long long c = 0;
+  for (uint64_t w = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; w < nwords; w += (uint64_t)gridDim.x * blockDim.x) c += __popc(live[w]);
+  if (c) atomicAdd(&st->nlive, c);
+}
+cudaError_t launch_count_live(const uint32_t* live, uint64_t cap, DevState* st, cudaStream_t s) {
+  count_live_kernel<<<grid_for((cap + 31) / 32), kThreads, 0, s>>>(live, (cap + 31) / 32, st);
+  count_launches(1);
+  return cudaGetLastError();
+}
+
+__global__ void fill_u32_kernel(uint32_t* p, uint32_t v, uint64_t n) {
+  for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < n; i += (uint64_t)gridDim.x * blockDim.x) p[i] = v;
+}
+cudaError_t launch_fill_u32(uint32_t* p, uint32_t v, uint64_t n, cudaStream_t s) {
+  if (n) { fill_u32_kernel<<<grid_for(n), kThreads, 0, s>>>(p, v, n); count_launches(1); }
+  return cudaGetLastError();
+}
+
+}  // namespace grand

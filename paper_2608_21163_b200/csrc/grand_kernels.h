@@ -1,0 +1,226 @@
+// Host-side launch interface between the C-ABI orchestration (grand_api.cu) and the kernel
+// translation units.  Plain structs of device pointers and sizes; every launcher enqueues on the
+// given stream and returns the cudaError_t of the launch.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace grand {
+
+// Number of kernels launched by this library in this process (every launcher adds its own).
+void count_launches(unsigned n);
+unsigned long long launches_so_far();
+
+// Row layout shared by every distance kernel: a padded row has nchunk 16-byte chunks; a team of G
+// lanes covers it with CPL chunks per lane.  layout_code selects the (G, CPL) instantiation.
+struct Layout {
+  uint32_t dim, dtype, metric;
+  uint32_t esize, row_bytes, nchunk;
+  int code;  // index into the (G, CPL) table, -1 = unsupported
+  int G, CPL;
+};
+Layout make_layout(uint32_t dim, uint32_t dtype, uint32_t metric);
+
+// Device-resident scalar state, read back by the host at the end of each update call.
+struct DevState {
+  int status;            // first error seen by a kernel (0 = ok); atomicMin of negative codes
+  uint32_t entry;        // medoid
+  uint32_t ndirty;       // length of the dirty list
+  uint32_t cursor;       // segment allocator for grouped requests
+  unsigned long long nlive;
+  unsigned long long total_in;   // sum of in-degrees of the delete batch
+  unsigned long long medoid_key; // argmin scratch
+  unsigned long long counters[8];  // expansions, dist_evals, pair_dists, dirty, prunes, requests
+};
+enum { CTR_EXP = 0, CTR_DIST = 1, CTR_PAIR = 2, CTR_DIRTY = 3, CTR_PRUNE = 4, CTR_REQ = 5 };
+
+struct GraphView {
+  const uint8_t* store;
+  uint32_t* adj;
+  uint32_t* deg;
+  uint32_t* live;  // bitmap
+  uint32_t R;
+  uint64_t cap;
+};
+
+struct SearchArgs {
+  Layout lay;
+  GraphView g;
+  uint32_t entry;
+  const void* queries;   // packed nq x dim elements (used when qids == nullptr)
+  const uint32_t* qids;  // queries are the store rows of these ids
+  uint64_t nq;
+  uint32_t L, vmax, k;
+  uint32_t* out_ids;     // nq x k (nullable)
+  void* out_dists;       // nq x k int32/float (nullable)
+  unsigned long long* out_beam;  // nq x beam_stride clean keys, ascending (nullable)
+  uint32_t* out_beam_n;
+  uint32_t beam_stride;
+  unsigned long long* out_vis;   // nq x vis_stride clean keys in expansion order (nullable)
+  uint32_t* out_vis_n;
+  uint32_t vis_stride;
+  const uint32_t* boot_ids;  // bootstrap: scan these ids (all batch-mates) instead of walking the graph
+  uint32_t boot_n;
+  uint32_t hash_bits;
+  DevState* state;
+};
+cudaError_t launch_beam_search(const SearchArgs& a, cudaStream_t s);
+size_t beam_search_smem_per_warp(uint32_t L, uint32_t R, uint32_t hash_bits);
+
+struct PruneArgs {
+  Layout lay;
+  GraphView g;
+  long long A_fix;
+  float alpha;
+  const uint32_t* ids;  // batch ids, n
+  uint64_t n;
+  const unsigned long long* cand;  // n x cand_stride keys (visited lists)
+  const uint32_t* cand_n;
+  uint32_t cand_stride;
+  uint32_t fixed_mode;  // 1: no prune, row = first R candidates in key order (Alg. 7)
+  // outputs: adjacency row + request tuples (target = selected neighbour, key = (dist, new id))
+  uint32_t* req_tgt;             // n x R
+  unsigned long long* req_key;   // n x R
+  DevState* state;
+};
+cudaError_t launch_forward_prune(const PruneArgs& a, cudaStream_t s);
+
+struct GroupArgs {
+  const uint32_t* req_tgt;
+  const unsigned long long* req_key;
+  uint64_t nreq;
+  uint32_t* cnt;    // per node, zero between calls
+  uint32_t* fill;   // per node, zero between calls
+  uint32_t* start;  // per node
+  uint32_t* flag;   // per node dirty flag, zero between calls
+  uint32_t* dirty;  // dirty list
+  unsigned long long* seg_keys;  // grouped keys
+  DevState* state;
+};
+cudaError_t launch_group_requests(const GroupArgs& a, cudaStream_t s);
+
+struct RebuildArgs {
+  Layout lay;
+  GraphView g;
+  long long A_fix;
+  float alpha;
+  uint32_t P;
+  const uint32_t* delmap;  // bitmap of the delete batch, or nullptr on insert
+  uint32_t* cnt; uint32_t* fill; uint32_t* start; uint32_t* flag;
+  const uint32_t* dirty;
+  unsigned long long* seg_keys;
+  uint32_t max_blocks;
+  DevState* state;
+};
+cudaError_t launch_rebuild(const RebuildArgs& a, cudaStream_t s);
+
+// fixed-degree reverse edges (Alg. 7): one owner per target, detour find-and-replace
+struct FixedReverseArgs {
+  GraphView g;
+  const uint32_t* slot_of;   // id -> batch position
+  const uint32_t* fwd_rows;  // batch position x R: forward rows as written (INVALID padded)
+  uint32_t* cnt; uint32_t* fill; uint32_t* start; uint32_t* flag;
+  const uint32_t* dirty;
+  unsigned long long* seg_keys;
+  uint32_t max_blocks;
+  DevState* state;
+};
+cudaError_t launch_fixed_reverse(const FixedReverseArgs& a, cudaStream_t s);
+
+// ---- reverse graph (Alg. 8): histogram -> exclusive scan -> scatter (-> sort rows)
+struct TransposeArgs {
+  GraphView g;
+  uint32_t* indeg;  // cap+1 scratch (zeroed inside)
+  uint32_t* off;    // cap+1
+  uint32_t* fillc;  // cap scratch (zeroed inside)
+  uint32_t* src;    // >= total edges (nullable: offsets only)
+  uint32_t* scan_tmp;  // >= ceil((cap+1)/4096)+1
+  bool sort_rows;
+};
+cudaError_t launch_transpose(const TransposeArgs& a, cudaStream_t s);
+cudaError_t launch_exclusive_scan(const uint32_t* in, uint32_t* out, uint64_t n, uint32_t* tmp, cudaStream_t s);
+
+// ---- delete repair (Alg. 6)
+struct DeleteArgs {
+  Layout lay;
+  GraphView g;
+  const uint32_t* ids; uint64_t n;   // delete batch
+  const uint32_t* delmap;
+  const unsigned long long* beam; const uint32_t* beam_n; uint32_t beam_stride;  // per-deleted search result
+  unsigned long long* Ci; uint32_t* Ci_n; uint32_t k_repair;                    // repair candidates
+  uint32_t c;
+  const uint32_t* off; const uint32_t* src;   // reverse graph
+  uint32_t* in_cnt; uint32_t* pair_off;       // n+1
+  uint32_t* scan_tmp;
+  uint32_t* req_tgt; unsigned long long* req_key;   // (total_in + n*R) * c
+  uint32_t* flag; uint32_t* dirty;
+  DevState* state;
+};
+cudaError_t launch_delete_prepare(const DeleteArgs& a, cudaStream_t s);   // in-degree prefix, total_in
+cudaError_t launch_delete_ci(const DeleteArgs& a, cudaStream_t s);        // repair candidates C_i
+cudaError_t launch_delete_picks(const DeleteArgs& a, uint64_t total_in, cudaStream_t s);
+
+struct FixedDeleteArgs {
+  GraphView g;
+  const uint32_t* ids; uint64_t n;
+  const uint32_t* delmap;
+  const uint32_t* off; const uint32_t* src;
+  const uint32_t* pair_off;  // n+1 prefix of in-degrees
+  uint32_t* flag; uint32_t* dirty;
+  DevState* state;
+};
+cudaError_t launch_fixed_delete(const FixedDeleteArgs& a, uint64_t total_in, cudaStream_t s);
+
+// ---- small kernels
+cudaError_t launch_validate(const uint32_t* ids, uint64_t n, uint64_t cap, const uint32_t* live, uint32_t* mark,
+                            int want_live, DevState* st, cudaStream_t s);
+cudaError_t launch_clear_marks(const uint32_t* ids, uint64_t n, uint64_t cap, uint32_t* mark, cudaStream_t s);
+cudaError_t launch_store_write(const Layout& lay, uint8_t* store, uint32_t* deg, uint32_t* slot_of, const uint32_t* ids,
+                               const void* vecs, uint64_t n, cudaStream_t s);
+cudaError_t launch_publish(const uint32_t* ids, uint64_t n, uint32_t* live, uint32_t* mark, DevState* st, cudaStream_t s);
+cudaError_t launch_retire(const GraphView& g, const uint32_t* ids, uint64_t n, uint32_t* delmap,
+                          const unsigned long long* Ci, const uint32_t* Ci_n, uint32_t k_repair, uint32_t fixed_mode,
+                          DevState* st, cudaStream_t s);
+cudaError_t launch_pick_medoid(const Layout& lay, const GraphView& g, const uint32_t* ids, uint64_t n, uint8_t* mean_row,
+                               DevState* st, cudaStream_t s);
+cudaError_t launch_count_live(const uint32_t* live, uint64_t cap, DevState* st, cudaStream_t s);
+cudaError_t launch_pad_rows(const Layout& lay, uint8_t* store, const void* vecs, uint64_t n, cudaStream_t s);
+cudaError_t launch_fill_u32(uint32_t* p, uint32_t v, uint64_t n, cudaStream_t s);
+
+}  // namespace grand
+
+// ---- (G, CPL) dispatch table.  nchunk <= 2 -> (2,1); <= 8 -> (8,1); <= 16 -> (8,2); <= 24 -> (8,3);
+// <= 32 -> (8,4); <= 64 -> (32,2); <= 128 -> (32,4); <= 256 -> (32,8).
+#define GRAND_LAYOUT_SWITCH(code, FN, T, M, ...)            \
+  switch (code) {                                           \
+    case 0: return FN<T, M, 2, 1>(__VA_ARGS__);             \
+    case 1: return FN<T, M, 8, 1>(__VA_ARGS__);             \
+    case 2: return FN<T, M, 8, 2>(__VA_ARGS__);             \
+    case 3: return FN<T, M, 8, 3>(__VA_ARGS__);             \
+    case 4: return FN<T, M, 8, 4>(__VA_ARGS__);             \
+    case 5: return FN<T, M, 32, 2>(__VA_ARGS__);            \
+    case 6: return FN<T, M, 32, 4>(__VA_ARGS__);            \
+    case 7: return FN<T, M, 32, 8>(__VA_ARGS__);            \
+    default: return cudaErrorInvalidValue;                  \
+  }
+// all dtypes x both metrics
+#define GRAND_DISPATCH_ALL(lay, FN, ...)                                                        \
+  do {                                                                                          \
+    if ((lay).dtype == 0) {                                                                     \
+      if ((lay).metric == 0) { GRAND_LAYOUT_SWITCH((lay).code, FN, uint8_t, 0, __VA_ARGS__) }   \
+      else { GRAND_LAYOUT_SWITCH((lay).code, FN, uint8_t, 1, __VA_ARGS__) }                     \
+    } else if ((lay).dtype == 1) {                                                              \
+      if ((lay).metric == 0) { GRAND_LAYOUT_SWITCH((lay).code, FN, int8_t, 0, __VA_ARGS__) }    \
+      else { GRAND_LAYOUT_SWITCH((lay).code, FN, int8_t, 1, __VA_ARGS__) }                      \
+    } else {                                                                                    \
+      if ((lay).metric == 0) { GRAND_LAYOUT_SWITCH((lay).code, FN, float, 0, __VA_ARGS__) }     \
+      else { GRAND_LAYOUT_SWITCH((lay).code, FN, float, 1, __VA_ARGS__) }                       \
+    }                                                                                           \
+  } while (0)
+// L2 only (Vamana-mode kernels: alpha-pruning is defined for the L2 metric)
+#define GRAND_DISPATCH_L2(lay, FN, ...)                                                         \
+  do {                                                                                          \
+    if ((lay).dtype == 0) { GRAND_LAYOUT_SWITCH((lay).code, FN, uint8_t, 0, __VA_ARGS__) }      \
+    else if ((lay).dtype == 1) { GRAND_LAYOUT_SWITCH((lay).code, FN, int8_t, 0, __VA_ARGS__) }  \
+    else { GRAND_LAYOUT_SWITCH((lay).code, FN, float, 0, __VA_ARGS__) }                         \
+  } while (0)

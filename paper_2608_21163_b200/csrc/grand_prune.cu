@@ -1,0 +1,387 @@
+// RobustPrune kernels: forward edges of new nodes (Alg. 5, first parallel loop), the rebuild of
+// dirty nodes after reverse-edge / repair requests were grouped (Alg. 5 dirty loop, Alg. 6 rebuild
+// loop), and the fixed-degree detour find-and-replace (Alg. 7).  One thread block owns one node, so
+// no two blocks ever write the same adjacency row.
+#include "grand_common.cuh"
+#include "grand_kernels.h"
+
+namespace grand {
+
+constexpr int kPruneThreads = 128;
+constexpr uint32_t kMaxCand = 1024;  // >= vmax limit
+constexpr uint32_t kSegCap = 1024;   // request segment sorted in shared memory up to this length
+constexpr uint32_t kMaxP = 256;
+constexpr uint32_t kMaxR = 128;
+
+// GrANDRobustPrune (Alg. 4) over candidate keys sorted ascending in shared memory.  The whole
+// block takes part.  Selected candidate indices go to out_idx; returns how many were selected.
+template <typename T, int G, int CPL>
+__device__ uint32_t block_prune(const uint8_t* __restrict__ store, uint32_t row_bytes, uint32_t nchunk, const AlphaParam ap,
+                                const unsigned long long* cand, uint32_t n, uint32_t R, uint32_t* validw,
+                                uint32_t* out_idx, volatile uint32_t* sh_sel, unsigned long long& npair) {
+  using Dist = typename Elem<T>::Dist;
+  constexpr unsigned FULL = 0xFFFFFFFFu;
+  const uint32_t tid = threadIdx.x, nthreads = blockDim.x;
+  const int lane = tid & 31, warp = tid >> 5;
+  const int t = lane % G;
+  const uint32_t team_global = tid / G, nteams = nthreads / G;
+  const uint32_t nwords = (n + 31) >> 5;
+  for (uint32_t w = tid; w < nwords; w += nthreads)
+    validw[w] = (w * 32 + 32 <= n) ? 0xFFFFFFFFu : ((1u << (n - w * 32)) - 1u);
+  __syncthreads();
+  uint32_t cnt = 0;
+  for (;;) {
+    if (warp == 0) {  // p* = first valid candidate
+      uint32_t s = kInvalid;
+      for (uint32_t wb = 0; wb < nwords; wb += 32) {
+        const uint32_t w = wb + lane;
+        const uint32_t word = w < nwords ? validw[w] : 0u;
+        const unsigned bal = __ballot_sync(FULL, word != 0u);
+        if (bal) {
+          const int srcl = __ffs(bal) - 1;
+          const uint32_t ww = __shfl_sync(FULL, word, srcl);
+          s = (wb + srcl) * 32 + __ffs(ww) - 1;
+          break;
+        }
+      }
+      if (lane == 0) {
+        *sh_sel = s;
+        if (s != kInvalid) {
+          out_idx[cnt] = s;
+          validw[s >> 5] &= ~(1u << (s & 31));
+        }
+      }
+    }
+    __syncthreads();
+    const uint32_t s = *sh_sel;
+    if (s == kInvalid) break;
+    ++cnt;
+    if (cnt == R) break;
+    // invalidate every remaining p' with alpha * dist(p*, p') <= D_p[p']
+    uint4 pstar[CPL];
+    load_row<G, CPL>(store + (size_t)key_id(cand[s]) * row_bytes, nchunk, t, pstar);
+    for (uint32_t jb = s + 1; jb < n; jb += nteams) {
+      const uint32_t j = jb + team_global;
+      const bool act = j < n && ((validw[j >> 5] >> (j & 31)) & 1u);
+      uint4 v[CPL];
+      if (act) {
+        load_row<G, CPL>(store + (size_t)key_id(cand[j]) * row_bytes, nchunk, t, v);
+      } else {
+#pragma unroll
+        for (int c = 0; c < CPL; ++c) v[c] = make_uint4(0, 0, 0, 0);
+      }
+      const Dist d = team_dist_regs<T, kMetricL2, G, CPL>(pstar, v);
+      if (act && t == 0) {
+        ++npair;
+        if (alpha_test(ap, d, key_dist<Dist>(cand[j]))) atomicAnd(&validw[j >> 5], ~(1u << (j & 31)));
+      }
+    }
+    __syncthreads();
+  }
+  __syncthreads();
+  return cnt;
+}
+
+template <typename T, int METRIC, int G, int CPL>
+__global__ void __launch_bounds__(kPruneThreads) forward_prune_kernel(const PruneArgs a) {
+  __shared__ unsigned long long cand[kMaxCand];
+  __shared__ uint32_t validw[kMaxCand / 32];
+  __shared__ uint32_t out_idx[kMaxR];
+  __shared__ uint32_t sh_sel;
+  const uint32_t tid = threadIdx.x, nthreads = blockDim.x;
+  const uint32_t R = a.g.R;
+  const AlphaParam ap{a.A_fix, a.alpha};
+  unsigned long long npair = 0;
+  uint32_t nprune = 0;
+  auto sync = [] { __syncthreads(); };
+  for (uint64_t i = blockIdx.x; i < a.n; i += gridDim.x) {
+    const uint32_t p = a.ids[i];
+    const uint32_t nc = min(min(a.cand_n[i], a.cand_stride), kMaxCand);
+    for (uint32_t j = tid; j < nc; j += nthreads) {
+      const unsigned long long k = a.cand[i * a.cand_stride + j];
+      cand[j] = key_id(k) == p ? kKeyMax : k;
+    }
+    __syncthreads();
+    bitonic_sort_any(cand, nc, tid, nthreads, sync);
+    uint32_t n = nc;
+    while (n > 0 && cand[n - 1] == kKeyMax) --n;
+    uint32_t cnt;
+    if (a.fixed_mode) {
+      cnt = min(n, R);
+      for (uint32_t j = tid; j < cnt; j += nthreads) out_idx[j] = j;
+      __syncthreads();
+    } else {
+      cnt = block_prune<T, G, CPL>(a.g.store, a.lay.row_bytes, a.lay.nchunk, ap, cand, n, R, validw, out_idx, &sh_sel, npair);
+      ++nprune;
+    }
+    for (uint32_t s = tid; s < R; s += nthreads) {
+      uint32_t id = kInvalid;
+      unsigned long long rk = 0;
+      if (s < cnt) {
+        const unsigned long long k = cand[out_idx[s]];
+        id = key_id(k);
+        rk = (k & 0xFFFFFFFF00000000ull) | p;  // dist(p, id) is symmetric: the request carries it
+      }
+      a.g.adj[(size_t)p * R + s] = id;
+      a.req_tgt[i * R + s] = id;
+      a.req_key[i * R + s] = rk;
+    }
+    if (tid == 0) a.g.deg[p] = cnt;
+    __syncthreads();
+  }
+  if (npair) atomicAdd(&a.state->counters[CTR_PAIR], npair);
+  if (tid == 0 && nprune) atomicAdd(&a.state->counters[CTR_PRUNE], (unsigned long long)nprune);
+}
+
+template <typename T, int METRIC, int G, int CPL>
+static cudaError_t launch_forward_prune_t(const PruneArgs& a, cudaStream_t s) {
+  if (a.n == 0) return cudaSuccess;
+  const unsigned blocks = (unsigned)(a.n < 148u * 16u ? a.n : 148u * 16u);
+  forward_prune_kernel<T, METRIC, G, CPL><<<blocks, kPruneThreads, 0, s>>>(a);
+  count_launches(1);
+  return cudaGetLastError();
+}
+cudaError_t launch_forward_prune(const PruneArgs& a, cudaStream_t s) {
+  GRAND_DISPATCH_ALL(a.lay, launch_forward_prune_t, a, s);
+  return cudaErrorInvalidValue;
+}
+
+// Sort one target's request segment by (dist, id) and return the pointer to the sorted keys
+// (shared memory copy for short segments, in place in global memory for long ones).
+__device__ __forceinline__ unsigned long long* sort_segment(unsigned long long* seg_global, uint32_t n,
+                                                            unsigned long long* seg_smem) {
+  const uint32_t tid = threadIdx.x, nthreads = blockDim.x;
+  auto sync = [] { __syncthreads(); };
+  unsigned long long* seg = seg_global;
+  if (n <= kSegCap) {
+    for (uint32_t j = tid; j < n; j += nthreads) seg_smem[j] = seg_global[j];
+    seg = seg_smem;
+  }
+  __syncthreads();
+  bitonic_sort_any(seg, n, tid, nthreads, sync);
+  return seg;
+}
+
+// Rebuild of dirty nodes: C = (N_out(u) \ B) ++ (scratch_u \ N_out(u) \ {u}); store C if it fits R,
+// else compute D_u for the old neighbours (requests already carry dist(u, id)) and prune.
+template <typename T, int METRIC, int G, int CPL>
+__global__ void __launch_bounds__(kPruneThreads) rebuild_kernel(const RebuildArgs a) {
+  using Dist = typename Elem<T>::Dist;
+  constexpr unsigned FULL = 0xFFFFFFFFu;
+  __shared__ unsigned long long seg_smem[kSegCap];
+  __shared__ unsigned long long scratch[kMaxP];
+  __shared__ unsigned long long cand[kMaxR + kMaxP];
+  __shared__ uint32_t keep[kMaxR];
+  __shared__ uint32_t validw[(kMaxR + kMaxP) / 32];
+  __shared__ uint32_t out_idx[kMaxR];
+  __shared__ uint32_t sh_sel, sh_ns, sh_nk, sh_nf;
+  const uint32_t tid = threadIdx.x, nthreads = blockDim.x;
+  const int lane = tid & 31, warp = tid >> 5;
+  const int t = lane % G;
+  const uint32_t team_global = tid / G, nteams = nthreads / G;
+  const uint32_t R = a.g.R;
+  const AlphaParam ap{a.A_fix, a.alpha};
+  const uint32_t row_bytes = a.lay.row_bytes, nchunk = a.lay.nchunk;
+  unsigned long long npair = 0;
+  uint32_t nprune = 0, ndone = 0;
+  auto sync = [] { __syncthreads(); };
+  const uint32_t ndirty = a.state->ndirty;
+  for (uint32_t k = blockIdx.x; k < ndirty; k += gridDim.x) {
+    const uint32_t u = a.dirty[k];
+    const uint32_t cntu = a.cnt[u];
+    unsigned long long* seg = sort_segment(a.seg_keys + a.start[u], cntu, seg_smem);
+    // scratch_u: first P distinct requests in key order (equal pairs are adjacent after the sort)
+    if (tid == 0) {
+      uint32_t ns = 0;
+      unsigned long long prev = kKeyMax;
+      for (uint32_t j = 0; j < cntu && ns < a.P; ++j) {
+        const unsigned long long kk = seg[j];
+        if (kk != prev) scratch[ns++] = kk;
+        prev = kk;
+      }
+      sh_ns = ns;
+    }
+    // keep = N_out(u) \ B, stable
+    if (warp == 1 || nthreads == 32) {
+      const uint32_t du = min(a.g.deg[u], R);
+      const uint32_t* row = a.g.adj + (size_t)u * R;
+      uint32_t nk = 0;
+      for (uint32_t sb = 0; sb < du; sb += 32) {
+        const uint32_t s = sb + lane;
+        uint32_t v = kInvalid;
+        bool ok = false;
+        if (s < du) {
+          v = row[s];
+          ok = !(a.delmap && bit_test(a.delmap, v));
+        }
+        const unsigned bal = __ballot_sync(FULL, ok);
+        if (ok) keep[nk + __popc(bal & ((1u << lane) - 1u))] = v;
+        nk += __popc(bal);
+      }
+      if (lane == 0) sh_nk = nk;
+    }
+    __syncthreads();
+    const uint32_t ns = sh_ns, nk = sh_nk;
+    // fresh = scratch \ keep \ {u}, stable, appended after the keep slots of cand
+    if (warp == 0) {
+      uint32_t nf = 0;
+      for (uint32_t jb = 0; jb < ns; jb += 32) {
+        const uint32_t j = jb + lane;
+        bool ok = false;
+        unsigned long long kk = 0;
+        if (j < ns) {
+          kk = scratch[j];
+          const uint32_t id = key_id(kk);
+          ok = id != u;
+          for (uint32_t x = 0; ok && x < nk; ++x) ok = keep[x] != id;
+        }
+        const unsigned bal = __ballot_sync(FULL, ok);
+        if (ok) cand[nk + nf + __popc(bal & ((1u << lane) - 1u))] = kk;
+        nf += __popc(bal);
+      }
+      if (lane == 0) sh_nf = nf;
+    }
+    __syncthreads();
+    const uint32_t nf = sh_nf, nC = nk + nf;
+    uint32_t* row_out = a.g.adj + (size_t)u * R;
+    if (nC <= R) {
+      for (uint32_t s = tid; s < R; s += nthreads)
+        row_out[s] = s < nk ? keep[s] : (s < nC ? key_id(cand[s]) : kInvalid);
+      if (tid == 0) a.g.deg[u] = nC;
+    } else {
+      // D_u for the kept neighbours
+      uint4 ur[CPL];
+      load_row<G, CPL>(a.g.store + (size_t)u * row_bytes, nchunk, t, ur);
+      for (uint32_t jb = 0; jb < nk; jb += nteams) {
+        const uint32_t j = jb + team_global;
+        const bool act = j < nk;
+        uint4 v[CPL];
+        if (act) {
+          load_row<G, CPL>(a.g.store + (size_t)keep[j] * row_bytes, nchunk, t, v);
+        } else {
+#pragma unroll
+          for (int c = 0; c < CPL; ++c) v[c] = make_uint4(0, 0, 0, 0);
+        }
+        const Dist d = team_dist_regs<T, kMetricL2, G, CPL>(ur, v);
+        if (act && t == 0) {
+          cand[j] = make_key(d, keep[j]);
+          ++npair;
+        }
+      }
+      __syncthreads();
+      bitonic_sort_any(cand, nC, tid, nthreads, sync);
+      const uint32_t cnt = block_prune<T, G, CPL>(a.g.store, row_bytes, nchunk, ap, cand, nC, R, validw, out_idx, &sh_sel, npair);
+      ++nprune;
+      for (uint32_t s = tid; s < R; s += nthreads) row_out[s] = s < cnt ? key_id(cand[out_idx[s]]) : kInvalid;
+      if (tid == 0) a.g.deg[u] = cnt;
+    }
+    if (tid == 0) {
+      a.cnt[u] = 0;
+      a.fill[u] = 0;
+      a.flag[u] = 0;
+      ++ndone;
+    }
+    __syncthreads();
+  }
+  if (npair) atomicAdd(&a.state->counters[CTR_PAIR], npair);
+  if (tid == 0) {
+    if (nprune) atomicAdd(&a.state->counters[CTR_PRUNE], (unsigned long long)nprune);
+    if (ndone) atomicAdd(&a.state->counters[CTR_DIRTY], (unsigned long long)ndone);
+  }
+}
+
+template <typename T, int METRIC, int G, int CPL>
+static cudaError_t launch_rebuild_t(const RebuildArgs& a, cudaStream_t s) {
+  rebuild_kernel<T, METRIC, G, CPL><<<a.max_blocks, kPruneThreads, 0, s>>>(a);
+  count_launches(1);
+  return cudaGetLastError();
+}
+cudaError_t launch_rebuild(const RebuildArgs& a, cudaStream_t s) {
+  GRAND_DISPATCH_L2(a.lay, launch_rebuild_t, a, s);
+  return cudaErrorInvalidValue;
+}
+
+// Fixed-degree backward edges (Alg. 7): the owner of target q takes its requests in (dist, id)
+// order; a request from new node p appends while deg(q) < R, else replaces the highest-index slot
+// of N_out(q) that also occurs in N_out(p) and was not replaced earlier in this batch.
+__global__ void __launch_bounds__(kPruneThreads) fixed_reverse_kernel(const FixedReverseArgs a) {
+  constexpr unsigned FULL = 0xFFFFFFFFu;
+  __shared__ unsigned long long seg_smem[kSegCap];
+  __shared__ uint32_t row[kMaxR];
+  __shared__ uint32_t replaced[kMaxR];
+  const uint32_t tid = threadIdx.x;
+  const int lane = tid & 31, warp = tid >> 5;
+  const uint32_t R = a.g.R;
+  uint32_t ndone = 0;
+  const uint32_t ndirty = a.state->ndirty;
+  for (uint32_t k = blockIdx.x; k < ndirty; k += gridDim.x) {
+    const uint32_t q = a.dirty[k];
+    const uint32_t cntq = a.cnt[q];
+    unsigned long long* seg = sort_segment(a.seg_keys + a.start[q], cntq, seg_smem);
+    for (uint32_t s = tid; s < R; s += blockDim.x) {
+      row[s] = a.g.adj[(size_t)q * R + s];
+      replaced[s] = 0;
+    }
+    __syncthreads();
+    if (warp == 0) {
+      uint32_t dq = min(a.g.deg[q], R);
+      unsigned long long prev = kKeyMax;
+      for (uint32_t j = 0; j < cntq; ++j) {
+        const unsigned long long kk = seg[j];
+        if (kk == prev) continue;
+        prev = kk;
+        const uint32_t p = key_id(kk);
+        // already linked?
+        bool present = false;
+        for (uint32_t sb = 0; sb < dq; sb += 32) {
+          const uint32_t s = sb + lane;
+          present |= __any_sync(FULL, s < dq && row[s] == p);
+        }
+        if (present) continue;
+        if (dq < R) {
+          if (lane == 0) row[dq] = p;
+          ++dq;
+          __syncwarp();
+          continue;
+        }
+        const uint32_t* prow = a.fwd_rows + (size_t)a.slot_of[p] * R;
+        int pick = -1;
+        for (uint32_t sb = 0; sb < dq; sb += 32) {
+          const uint32_t s = sb + lane;
+          bool hit = false;
+          if (s < dq && !replaced[s]) {
+            const uint32_t x = row[s];
+            for (uint32_t y = 0; y < R; ++y) hit |= prow[y] == x;   // INVALID padding never equals a live id
+          }
+          const unsigned bal = __ballot_sync(FULL, hit);
+          if (bal) pick = (int)sb + 31 - __clz(bal);
+        }
+        if (pick >= 0) {
+          if (lane == 0) {
+            row[pick] = p;
+            replaced[pick] = 1;
+          }
+          __syncwarp();
+        }
+      }
+      for (uint32_t s = lane; s < R; s += 32) a.g.adj[(size_t)q * R + s] = s < dq ? row[s] : kInvalid;
+      if (lane == 0) {
+        a.g.deg[q] = dq;
+        a.cnt[q] = 0;
+        a.fill[q] = 0;
+        a.flag[q] = 0;
+        ++ndone;
+      }
+    }
+    __syncthreads();
+  }
+  if (tid == 0 && ndone) atomicAdd(&a.state->counters[CTR_DIRTY], (unsigned long long)ndone);
+}
+
+cudaError_t launch_fixed_reverse(const FixedReverseArgs& a, cudaStream_t s) {
+  fixed_reverse_kernel<<<a.max_blocks, kPruneThreads, 0, s>>>(a);
+  count_launches(1);
+  return cudaGetLastError();
+}
+
+}  // namespace grand

@@ -1,0 +1,302 @@
+// Batched greedy beam search (BeamSearch, Alg. 1): one warp per query.
+//
+// Per warp, in shared memory: the sorted worklist C (L keys; the expanded flag rides in bit 31 of
+// the id word), a direct-mapped visited cache that may forget but never lies (full ids), and the
+// candidate staging arrays of one expansion.  One expansion = read the adjacency row of the best
+// unexpanded entry, drop ids the cache has seen, gather the surviving neighbours' vectors with
+// 128-bit loads (a team of G lanes per vector, several vectors in flight per lane), reduce the
+// distances with shuffles, and merge the survivors into the worklist in parallel.
+//
+// The worklist always equals the L smallest (dist, id) keys seen so far, so the result does not
+// depend on what the cache forgets: a re-evaluated node either matches an entry exactly (dropped
+// as a duplicate by key equality) or fails the comparison with the worst entry.
+#include "grand_common.cuh"
+#include "grand_kernels.h"
+
+namespace grand {
+
+constexpr int kSearchWarps = 4;
+
+static inline uint32_t even_up(uint32_t x) { return (x + 1u) & ~1u; }
+
+size_t beam_search_smem_per_warp(uint32_t L, uint32_t R, uint32_t hash_bits) {
+  const size_t Lp = even_up(L), Rp = even_up(R);
+  return Lp * 8 + Rp * 8 + Rp * 8 + Rp * 4 + Rp * 4 + ((size_t)4 << hash_bits);
+}
+
+template <typename T, int METRIC, int G, int CPL>
+__global__ void __launch_bounds__(kSearchWarps * 32) beam_search_kernel(const SearchArgs a, const uint32_t per_warp_bytes) {
+  using Dist = typename Elem<T>::Dist;
+  constexpr int NT = 32 / G;                                   // teams per warp
+  constexpr int U = CPL == 1 ? 4 : (CPL == 2 ? 2 : 1);         // vectors in flight per team
+  constexpr unsigned FULL = 0xFFFFFFFFu;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int t = lane % G, team = lane / G;
+  const uint32_t L = a.L, R = a.g.R, H = 1u << a.hash_bits;
+  const uint32_t Lp = (L + 1u) & ~1u, Rp = (R + 1u) & ~1u;
+  unsigned char* base = smem_raw + (size_t)warp * per_warp_bytes;
+  unsigned long long* beam = reinterpret_cast<unsigned long long*>(base);
+  unsigned long long* ckey = beam + Lp;     // candidate keys of this expansion (unsorted)
+  unsigned long long* cskey = ckey + Rp;    // surviving candidate keys, ascending
+  uint32_t* cid = reinterpret_cast<uint32_t*>(cskey + Rp);  // candidate ids, later their worklist ranks
+  uint32_t* csb = cid + Rp;                 // worklist rank of each sorted survivor
+  uint32_t* hash = csb + Rp;                // visited cache (also query staging)
+
+  const uint32_t nchunk = a.lay.nchunk, row_bytes = a.lay.row_bytes;
+  const uint8_t* __restrict__ store = a.g.store;
+  unsigned long long n_exp = 0, n_dist = 0;
+
+  const uint64_t wglobal = (uint64_t)blockIdx.x * kSearchWarps + warp;
+  const uint64_t wtotal = (uint64_t)gridDim.x * kSearchWarps;
+  for (uint64_t qi = wglobal; qi < a.nq; qi += wtotal) {
+    // ---- query into registers: lane t of each team holds chunks t, t+G, ...
+    uint4 q[CPL];
+    uint32_t self = kInvalid;
+    if (a.qids) {
+      self = a.qids[qi];
+      load_row<G, CPL>(store + (size_t)self * row_bytes, nchunk, t, q);
+    } else {
+      T* stage = reinterpret_cast<T*>(hash);
+      const T* src = reinterpret_cast<const T*>(a.queries) + qi * a.lay.dim;
+      const uint32_t npad = row_bytes / sizeof(T);
+      for (uint32_t j = lane; j < npad; j += 32) stage[j] = j < a.lay.dim ? src[j] : T(0);
+      __syncwarp();
+#pragma unroll
+      for (int c = 0; c < CPL; ++c) {
+        const uint32_t ch = t + c * G;
+        q[c] = ch < nchunk ? reinterpret_cast<const uint4*>(stage)[ch] : make_uint4(0, 0, 0, 0);
+      }
+      __syncwarp();
+    }
+    for (uint32_t j = lane; j < H; j += 32) hash[j] = kInvalid;
+    __syncwarp();
+
+    uint32_t beam_n = 0, nvis = 0, cursor = 0;
+
+    // Evaluate cid[0..n) against the query and merge the survivors into the worklist.
+    auto process = [&](uint32_t n) {
+      // 1. distances: NT teams, U vectors in flight per team
+      for (uint32_t b0 = 0; b0 < n; b0 += NT * U) {
+        uint4 v[U][CPL];
+        uint32_t idv[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          const uint32_t idx = b0 + u * NT + team;
+          idv[u] = idx < n ? cid[idx] : kInvalid;
+          if (idv[u] != kInvalid) {
+            load_row<G, CPL>(store + (size_t)idv[u] * row_bytes, nchunk, t, v[u]);
+          } else {
+#pragma unroll
+            for (int c = 0; c < CPL; ++c) v[u][c] = make_uint4(0, 0, 0, 0);
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          const Dist d = team_dist_regs<T, METRIC, G, CPL>(q, v[u]);
+          if (t == 0 && idv[u] != kInvalid) ckey[b0 + u * NT + team] = make_key(d, idv[u]);
+        }
+      }
+      n_dist += n;
+      __syncwarp();
+      // 2. keep keys below the worst entry that are not already in the worklist
+      const unsigned long long worst = beam_n == L ? key_clean(beam[L - 1]) : kKeyMax;
+      uint32_t m = 0;
+      for (uint32_t jb = 0; jb < n; jb += 32) {
+        const uint32_t j = jb + lane;
+        bool pass = false;
+        if (j < n) {
+          const unsigned long long key = ckey[j];
+          pass = key < worst;
+          if (pass) {
+            const uint32_t b = lower_bound_clean(beam, beam_n, key);
+            if (b < beam_n && key_clean(beam[b]) == key) pass = false;
+            cid[j] = b;
+          }
+          if (!pass) ckey[j] = kKeyMax;
+        }
+        m += __popc(__ballot_sync(FULL, pass));
+      }
+      __syncwarp();
+      if (m == 0) return;
+      // rank survivors among themselves (counting sort by comparison; n <= R is small)
+      for (uint32_t j = lane; j < n; j += 32) {
+        const unsigned long long key = ckey[j];
+        if (key != kKeyMax) {
+          uint32_t r = 0;
+          for (uint32_t i = 0; i < n; ++i) r += ckey[i] < key;
+          cskey[r] = key;
+          csb[r] = cid[j];
+        }
+      }
+      __syncwarp();
+      // 3. shift worklist entries to their final places, highest chunk first (a move never goes
+      //    down, so an entry that is still unread is never overwritten)
+      const uint32_t minb = csb[0];
+      if (beam_n > minb) {
+        const int top = (int)((beam_n - 1) >> 5), low = (int)(minb >> 5);
+        for (int ch = top; ch >= low; --ch) {
+          const uint32_t i = (uint32_t)ch * 32 + lane;
+          unsigned long long e = 0;
+          uint32_t np = kInvalid;
+          if (i < beam_n && i >= minb) {
+            e = beam[i];
+            np = i + lower_bound_clean(cskey, m, key_clean(e));
+          }
+          __syncwarp();
+          if (np < L) beam[np] = e;
+          __syncwarp();
+        }
+      }
+      // 4. drop the survivors in
+      for (uint32_t r = lane; r < m; r += 32) {
+        const uint32_t np = r + csb[r];
+        if (np < L) beam[np] = cskey[r];
+      }
+      __syncwarp();
+      beam_n = min(L, beam_n + m);
+      cursor = min(cursor, minb);
+    };
+
+    if (a.boot_ids) {
+      // bootstrap batch: no graph yet, scan every batch-mate (brute force through the same merge)
+      for (uint32_t c0 = 0; c0 < a.boot_n; c0 += R) {
+        uint32_t n = 0;
+        for (uint32_t sb = 0; sb < R; sb += 32) {
+          const uint32_t s = sb + lane;
+          uint32_t v = kInvalid;
+          if (s < R && c0 + s < a.boot_n) v = a.boot_ids[c0 + s];
+          const bool ok = v != kInvalid && v != self;
+          const unsigned bal = __ballot_sync(FULL, ok);
+          if (ok) cid[n + __popc(bal & ((1u << lane) - 1u))] = v;
+          n += __popc(bal);
+        }
+        __syncwarp();
+        if (n) process(n);
+      }
+    } else if (a.entry != kInvalid) {
+      if (lane == 0) {
+        cid[0] = a.entry;
+        hash[(a.entry * 2654435761u) >> (32 - a.hash_bits)] = a.entry;
+      }
+      __syncwarp();
+      process(1);
+      while (nvis < a.vmax) {
+        // closest unexpanded entry; everything before `cursor` is expanded
+        uint32_t pos = kInvalid;
+        for (uint32_t cb = cursor & ~31u; cb < beam_n; cb += 32) {
+          const uint32_t i = cb + lane;
+          const bool un = i < beam_n && i >= cursor && !(beam[i] & kExpandedBit);
+          const unsigned bal = __ballot_sync(FULL, un);
+          if (bal) {
+            pos = cb + __ffs(bal) - 1;
+            break;
+          }
+        }
+        if (pos == kInvalid) break;
+        const unsigned long long ek = beam[pos];
+        __syncwarp();
+        if (lane == 0) {
+          beam[pos] = ek | kExpandedBit;
+          if (a.out_vis) a.out_vis[qi * a.vis_stride + nvis] = ek;
+        }
+        cursor = pos + 1;
+        ++nvis;
+        const uint32_t u = key_id(ek);
+        const uint32_t du = min(a.g.deg[u], R);
+        const uint32_t* __restrict__ row = a.g.adj + (size_t)u * R;
+        uint32_t n = 0;
+        for (uint32_t sb = 0; sb < du; sb += 32) {
+          const uint32_t s = sb + lane;
+          bool fresh = false;
+          uint32_t v = kInvalid;
+          if (s < du) {
+            v = __ldg(row + s);
+            const uint32_t h = (v * 2654435761u) >> (32 - a.hash_bits);
+            if (hash[h] != v) {
+              hash[h] = v;
+              fresh = true;
+            }
+          }
+          const unsigned bal = __ballot_sync(FULL, fresh);
+          if (fresh) cid[n + __popc(bal & ((1u << lane) - 1u))] = v;
+          n += __popc(bal);
+        }
+        __syncwarp();
+        if (n) process(n);
+      }
+      n_exp += nvis;
+    }
+
+    // ---- outputs
+    if (a.out_ids) {
+      for (uint32_t j = lane; j < a.k; j += 32) {
+        const bool have = j < beam_n;
+        const unsigned long long key = have ? beam[j] : 0ull;
+        a.out_ids[qi * a.k + j] = have ? key_id(key) : kInvalid;
+        if (a.out_dists) {
+          if constexpr (sizeof(T) == 4) {
+            reinterpret_cast<float*>(a.out_dists)[qi * a.k + j] = have ? key_dist<float>(key) : __int_as_float(0x7f800000);
+          } else {
+            reinterpret_cast<int*>(a.out_dists)[qi * a.k + j] = have ? key_dist<int>(key) : 0x7fffffff;
+          }
+        }
+      }
+    }
+    if (a.out_beam) {
+      for (uint32_t j = lane; j < beam_n; j += 32) a.out_beam[qi * a.beam_stride + j] = key_clean(beam[j]);
+      if (lane == 0) a.out_beam_n[qi] = beam_n;
+    }
+    if (a.out_vis) {
+      if (a.boot_ids) {  // bootstrap: the candidate list handed to the prune is the sorted worklist
+        const uint32_t nv = min(beam_n, a.vis_stride);
+        for (uint32_t j = lane; j < nv; j += 32) a.out_vis[qi * a.vis_stride + j] = key_clean(beam[j]);
+        if (lane == 0) a.out_vis_n[qi] = nv;
+      } else if (lane == 0) {
+        a.out_vis_n[qi] = nvis;
+      }
+    }
+    __syncwarp();
+  }
+  if (lane == 0 && a.state) {
+    if (n_exp) atomicAdd(&a.state->counters[CTR_EXP], n_exp);
+    if (n_dist) atomicAdd(&a.state->counters[CTR_DIST], n_dist);
+  }
+}
+
+template <typename T, int METRIC, int G, int CPL>
+static cudaError_t launch_beam_search_t(const SearchArgs& a, cudaStream_t s) {
+  const size_t per_warp = beam_search_smem_per_warp(a.L, a.g.R, a.hash_bits);
+  const size_t smem = per_warp * kSearchWarps;
+  auto kern = beam_search_kernel<T, METRIC, G, CPL>;
+  static size_t smem_set = 0;
+  static int sm_count = 0;
+  if (smem > smem_set) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    smem_set = smem;
+  }
+  if (!sm_count) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
+  }
+  int occ = 1;
+  cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, kSearchWarps * 32, smem);
+  if (occ < 1) occ = 1;
+  uint64_t blocks = (a.nq + kSearchWarps - 1) / kSearchWarps;
+  const uint64_t cap = (uint64_t)sm_count * occ;
+  if (blocks > cap) blocks = cap;
+  if (blocks == 0) return cudaSuccess;
+  kern<<<(unsigned)blocks, kSearchWarps * 32, smem, s>>>(a, (uint32_t)per_warp);
+  count_launches(1);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_beam_search(const SearchArgs& a, cudaStream_t s) {
+  GRAND_DISPATCH_ALL(a.lay, launch_beam_search_t, a, s);
+  return cudaErrorInvalidValue;
+}
+
+}  // namespace grand

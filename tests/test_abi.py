@@ -1,0 +1,46 @@
+"""The C-ABI library builds for sm_100a, loads without a GPU, and exports every symbol that
+include/grand.h declares (no compute is attempted here)."""
+import ctypes
+import os
+import re
+
+from paper_2608_21163_b200 import binding, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "grand.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(grand_[a-z_]+)\s*\(", text)))
+
+
+def test_library_builds_and_exports_every_declared_symbol():
+    path = build.build()
+    assert os.path.exists(path)
+    lib = ctypes.CDLL(path)
+    syms = declared_symbols()
+    assert len(syms) >= 20
+    for s in syms:
+        assert hasattr(lib, s), f"{s} declared in grand.h but not exported"
+    assert set(binding.EXPORTS) == set(syms)
+
+
+def test_strerror_and_argument_checks_need_no_gpu():
+    lib = binding.load()
+    assert lib.grand_strerror(0) == b"ok"
+    assert b"duplicate" in lib.grand_strerror(-3)
+    h = ctypes.c_void_p()
+    # Vamana mode + inner product is rejected before any CUDA call
+    rc = lib.grand_create(ctypes.c_uint32(8), ctypes.c_uint32(0), ctypes.c_uint32(1), ctypes.c_uint32(8),
+                          ctypes.c_uint32(16), ctypes.c_float(1.2), ctypes.byref(h))
+    assert rc == -6
+    rc = lib.grand_create(ctypes.c_uint32(8), ctypes.c_uint32(0), ctypes.c_uint32(0), ctypes.c_uint32(1000),
+                          ctypes.c_uint32(16), ctypes.c_float(1.2), ctypes.byref(h))
+    assert rc == -1
+
+
+def test_options_struct_layout_matches_header():
+    # 2 x u64, 6 x u32, 3 pointers
+    assert ctypes.sizeof(binding.GrandOptions) == 16 + 24 + 24
+    assert ctypes.sizeof(binding.GrandStats) == 8 * 8 + 7 * 8 + 8

@@ -1,0 +1,329 @@
+"""GPU parity: the CUDA library against the CPU oracle on the same seeded inputs, through the
+C-ABI.  Integer vectors must match bit for bit (adjacency rows, degrees, live bitmap, medoid,
+search ids and distances); fp32 vectors are held to 1e-5 relative distance error and a recall@10
+within 0.005 of the oracle's."""
+import numpy as np
+import pytest
+
+from oracle import grand_oracle as go
+from paper_2608_21163_b200 import synth
+from tests.helpers import (INV, assert_same_graph, brute_force_topk, gpu_graph, make_pair, recall_at_k, run_stream)
+
+pytestmark = pytest.mark.gpu
+
+
+def torch_():
+    import torch
+    return torch
+
+
+def gpu_search(g, q, k, L):
+    torch = torch_()
+    ids, d = g.search(torch.from_numpy(q), k, L)
+    torch.cuda.synchronize()
+    return ids.cpu().numpy(), d.cpu().numpy()
+
+
+def import_from_oracle(o, g, base_full):
+    torch = torch_()
+    adj, deg, live, entry = o.export_graph()
+    R = adj.shape[1]
+    adj = adj.copy()
+    adj[np.arange(R)[None, :] >= deg[:, None]] = INV
+    g.import_graph(torch.from_numpy(adj), torch.from_numpy(deg), torch.from_numpy(live), entry, torch.from_numpy(base_full))
+
+
+def small_cfg(name, scale, **over):
+    c = synth.scaled(synth.CONFIGS[name], scale)
+    c.update(over)
+    return c
+
+
+# ------------------------------------------------------------------ search on an imported graph
+@pytest.mark.parametrize("dim,dtype", [(32, go.U8), (33, go.U8), (128, go.U8), (20, go.I8), (200, go.U8)])
+def test_search_bit_exact_on_oracle_graph(dim, dtype):
+    n, R, L = 3000, 24, 48
+    rng = np.random.default_rng(dim)
+    if dtype == go.U8:
+        base = synth.uniform_u8(1, "base", 0, n, dim)
+        q = synth.uniform_u8(1, "query", 0, 300, dim)
+    else:
+        base = rng.integers(-128, 128, (n, dim)).astype(np.int8)
+        q = rng.integers(-128, 128, (300, dim)).astype(np.int8)
+        base[0] = -128; base[1] = 127           # extreme differences: |a-b| = 255 per coordinate
+        q[0] = 127; q[1] = -128
+    cfg = dict(dim=dim, dtype=dtype, metric=go.L2, R=R, L=L, alpha=1.2, mode=go.VAMANA, max_build_batch=500, ins=1, dele=1)
+    o, g = make_pair(cfg, n)
+    for lo in range(0, n, 500):
+        o.insert_batch(np.arange(lo, lo + 500, dtype=np.uint32), base[lo:lo + 500])
+    import_from_oracle(o, g, base)
+    assert g.live_count == n
+    for k, Ls in [(10, 48), (1, 1), (10, 10), (48, 48), (5, 200), (10, 512)]:
+        oi, od = o.search(q, k, Ls)
+        gi, gd = gpu_search(g, q, k, Ls)
+        assert (oi == gi).all(), (k, Ls, np.flatnonzero((oi != gi).any(1))[:5])
+        assert (od == gd.astype(np.float64)).all()
+
+
+def test_search_fp32_tolerance_and_ip():
+    n, dim, R, L = 4000, 96, 24, 64
+    base = synth.gaussian_unit_f32(2, "base", 0, n, dim)
+    q = synth.gaussian_unit_f32(2, "query", 0, 200, dim)
+    for metric, mode in [(go.L2, go.VAMANA), (go.IP, go.FIXED_DEGREE)]:
+        cfg = dict(dim=dim, dtype=go.F32, metric=metric, R=R, L=L, alpha=1.2, mode=mode, max_build_batch=500, ins=1, dele=1)
+        o, g = make_pair(cfg, n)
+        for lo in range(0, n, 500):
+            o.insert_batch(np.arange(lo, lo + 500, dtype=np.uint32), base[lo:lo + 500])
+        import_from_oracle(o, g, base)
+        oi, od = o.search(q, 10, L)
+        gi, gd = gpu_search(g, q, 10, L)
+        # returned distances against a float64 recomputation
+        for i in range(len(q)):
+            b = base[gi[i]].astype(np.float64)
+            exact = ((b - q[i].astype(np.float64)) ** 2).sum(1) if metric == go.L2 else -(b @ q[i].astype(np.float64))
+            scale = np.abs(exact) if metric == go.L2 else np.linalg.norm(b, axis=1) * np.linalg.norm(q[i])
+            assert (np.abs(gd[i] - exact) <= 1e-5 * scale).all()
+            assert (np.diff(gd[i]) >= 0).all()
+        # near-ties may reorder; the result sets must agree almost everywhere
+        same = np.mean([len(set(a.tolist()) & set(b.tolist())) / 10 for a, b in zip(oi, gi)])
+        assert same > 0.99
+
+
+def test_search_padding_and_empty_index():
+    torch = torch_()
+    cfg = dict(dim=8, dtype=go.U8, metric=go.L2, R=4, L=8, alpha=1.2, mode=go.VAMANA, max_build_batch=8, ins=1, dele=1)
+    o, g = make_pair(cfg, 16)
+    q = np.zeros((3, 8), np.uint8)
+    gi, gd = gpu_search(g, q, 4, 8)
+    assert (gi == INV).all() and (gd == np.iinfo(np.int32).max).all()
+    v = np.arange(24, dtype=np.uint8).reshape(3, 8)
+    ids = np.array([5, 2, 9], np.uint32)
+    o.insert_batch(ids, v)
+    g.insert_batch(torch.from_numpy(ids), torch.from_numpy(v))
+    assert_same_graph(o, g, "3-point bootstrap")
+    oi, od = o.search(q, 4, 8)
+    gi, gd = gpu_search(g, q, 4, 8)
+    assert (oi == gi).all() and gi[0, 3] == INV and gd[0, 3] == np.iinfo(np.int32).max
+    assert (od[:, :3] == gd[:, :3]).all()
+
+
+# ------------------------------------------------------------------ whole streams, bit exact
+def check_search(o, g, wl, cfg, k=10):
+    q = wl.queries()
+    oi, od = o.search(q, k, cfg["L"])
+    gi, gd = gpu_search(g, q, k, cfg["L"])
+    assert (oi == gi).all() and (od == gd.astype(np.float64)).all()
+
+
+def test_tiny_config_stream_bit_exact():
+    """The tiny config at full size: 8 x 1,000 build, +2,000, -1,000, 1,000 queries."""
+    cfg = synth.CONFIGS["tiny_u8_d32"]
+    o, g, wl, st = run_stream(cfg, seed=0)
+    check_search(o, g, wl, cfg)
+    assert o.stats()["dead_edges_seen"] == 0
+    # exact reverse graph
+    ooff, osrc = o.reverse_graph()
+    goff, gsrc = g.reverse_graph()
+    assert (ooff == goff.cpu().numpy().astype(np.uint64)).all() and (osrc == gsrc.cpu().numpy()).all()
+    # recall sanity
+    base = wl.vectors(0, cfg["n"])
+    live = np.flatnonzero(st.live).astype(np.uint32)
+    q = wl.queries()[:200]
+    gi, _ = gpu_search(g, q, 10, cfg["L"])
+    assert recall_at_k(gi, brute_force_topk(base, live, q, 10, go.L2)) > 0.9
+
+
+def test_sift_shaped_shrink_bit_exact():
+    """SIFT-shaped bytes (d=128, R=64, L=128) shrunk to 20k points: several insert/delete rounds."""
+    cfg = small_cfg("sift_u8_d128", 0.02, rounds=3)
+    o, g, wl, st = run_stream(cfg, seed=0)
+    check_search(o, g, wl, cfg)
+    q = wl.queries()
+    for L in (10, 32, 200):
+        oi, od = o.search(q, 10, L)
+        gi, gd = gpu_search(g, q, 10, L)
+        assert (oi == gi).all() and (od == gd.astype(np.float64)).all()
+
+
+def test_ragged_dim_int8_and_small_params_bit_exact():
+    """Odd dimension (tail chunk), int8 data, R/L not multiples of 32, tiny P and c=3."""
+    rng = np.random.default_rng(9)
+    torch = torch_()
+    n, dim = 2500, 45
+    base = rng.integers(-128, 128, (n, dim)).astype(np.int8)
+    cfg = dict(dim=dim, dtype=go.I8, metric=go.L2, R=13, L=21, alpha=1.1, mode=go.VAMANA, max_build_batch=400, ins=1, dele=300)
+    o, g = make_pair(cfg, n, P=3, c=3, k_repair=7, vmax=30)
+    for lo in range(0, n, 357):
+        ids = np.arange(lo, min(n, lo + 357), dtype=np.uint32)
+        o.insert_batch(ids, base[ids]); g.insert_batch(torch.from_numpy(ids), torch.from_numpy(base[ids]))
+        assert_same_graph(o, g, f"insert at {lo}")
+    dele = synth.choose_ids(3, "del", np.arange(n, dtype=np.uint32), 300)
+    o.delete_batch(dele); g.delete_batch(torch.from_numpy(dele))
+    assert_same_graph(o, g, "delete")
+    # id reuse
+    o.insert_batch(dele[:100], base[dele[:100]]); g.insert_batch(torch.from_numpy(dele[:100]), torch.from_numpy(base[dele[:100]]))
+    assert_same_graph(o, g, "reinsert")
+
+
+def test_hub_segment_longer_than_shared_memory_cap():
+    """Every point of a large batch links to the same few hubs: request segments far above the
+    in-kernel shared-memory cap take the in-place global-memory sort."""
+    torch = torch_()
+    dim = 4
+    hubs = np.array([[0, 0, 0, 0], [255, 255, 255, 255], [0, 255, 0, 255]], np.uint8)
+    pts = synth.uniform_u8(4, "hubpts", 0, 3000, dim) // 8 + 100          # clustered away from the hubs
+    cfg = dict(dim=dim, dtype=go.U8, metric=go.L2, R=8, L=16, alpha=1000.0, mode=go.VAMANA, max_build_batch=3000, ins=1, dele=1)
+    o, g = make_pair(cfg, 4000)
+    ids = np.arange(3, dtype=np.uint32)
+    o.insert_batch(ids, hubs); g.insert_batch(torch.from_numpy(ids), torch.from_numpy(hubs))
+    ids = np.arange(3, 3003, dtype=np.uint32)
+    o.insert_batch(ids, pts); g.insert_batch(torch.from_numpy(ids), torch.from_numpy(pts))
+    assert_same_graph(o, g, "hub insert")
+
+
+def test_delete_everything_and_reinsert():
+    torch = torch_()
+    cfg = small_cfg("tiny_u8_d32", 0.05)
+    n = cfg["n"]
+    base = synth.uniform_u8(0, "base", 0, n, 32)
+    o, g = make_pair(dict(cfg, max_build_batch=n, ins=n, dele=n), n)
+    ids = np.arange(n, dtype=np.uint32)
+    for lo in range(0, n, 100):
+        o.insert_batch(ids[lo:lo + 100], base[lo:lo + 100]); g.insert_batch(torch.from_numpy(ids[lo:lo + 100]), torch.from_numpy(base[lo:lo + 100]))
+    o.delete_batch(ids); g.delete_batch(torch.from_numpy(ids))
+    assert_same_graph(o, g, "all deleted")
+    assert g.entry == INV and g.live_count == 0
+    o.insert_batch(ids[::-1].copy(), base[::-1].copy()); g.insert_batch(torch.from_numpy(ids[::-1].copy()), torch.from_numpy(base[::-1].copy()))
+    assert_same_graph(o, g, "rebuilt in one bootstrap batch")
+
+
+def test_medoid_deletion_paths():
+    torch = torch_()
+    cfg = small_cfg("tiny_u8_d32", 0.1)
+    o, g, wl, st = run_stream(dict(cfg, rounds=0), seed=1)
+    m = np.array([o.entry], np.uint32)
+    o.delete_batch(m); g.delete_batch(torch.from_numpy(m))
+    assert_same_graph(o, g, "medoid deleted")
+    assert g.entry != m[0]
+
+
+# ------------------------------------------------------------------ fixed-degree mode
+def test_fixed_degree_mode_bit_exact_on_bytes():
+    """Alg. 7 / Alg. 8 logic is integer-only; with uint8 vectors and IP the whole state must match."""
+    cfg = dict(gen="uniform_u8", dim=24, dtype=go.U8, metric=go.IP, mode=go.FIXED_DEGREE, R=16, L=40, alpha=1.2,
+               n=6000, build=4000, first_batch=500, max_build_batch=1000, rounds=3, ins=500, dele=400, nq=200, reuse_ids=False)
+    o, g, wl, st = run_stream(cfg, seed=5)
+    check_search(o, g, wl, cfg)
+    cfg2 = dict(cfg, metric=go.L2, rounds=2)
+    o, g, wl, st = run_stream(cfg2, seed=6)
+    check_search(o, g, wl, cfg2)
+
+
+# ------------------------------------------------------------------ fp32 streams: tolerance + recall
+@pytest.mark.parametrize("name,scale", [("deep_f32_d96", 0.002), ("gist_f32_d960", 0.004), ("embed_f32_d768_ip", 0.001)])
+def test_fp32_streams_recall_matches_oracle(name, scale):
+    cfg = small_cfg(name, scale, rounds=2, nq=200)
+    cfg["first_batch"] = min(cfg["first_batch"], 500)
+    cfg["max_build_batch"] = max(cfg["max_build_batch"], 500)
+    o, g, wl, st = run_stream(cfg, seed=0, check_each=False, oracle=True, gpu=False)
+    _, g, _, st2 = run_stream(cfg, seed=0, check_each=False, oracle=False, gpu=True)
+    assert (st.live == st2.live).all()
+    # structural invariants of the GPU graph
+    adj, deg, live, entry = gpu_graph(g)
+    mask = go.live_mask(live, len(deg))
+    assert (mask == st.live).all() and (deg <= cfg["R"]).all() and (deg[~mask] == 0).all() and mask[entry]
+    for v in np.flatnonzero(mask)[:2000]:
+        r = adj[v, :deg[v]]
+        assert mask[r].all() and v not in r and len(set(r.tolist())) == len(r)
+    n_rows = st.next_row
+    base = np.zeros((wl.capacity(), cfg["dim"]), np.float32)
+    # regenerate what is live now (ids map to rows 1:1 unless ids are reused)
+    if not cfg["reuse_ids"]:
+        base[:n_rows] = wl.vectors(0, n_rows)
+        live_ids = np.flatnonzero(st.live).astype(np.uint32)
+        q = wl.queries()
+        truth = brute_force_topk(base, live_ids, q, 10, cfg["metric"])
+        oi, _ = o.search(q, 10, cfg["L"])
+        gi, gd = gpu_search(g, q, 10, cfg["L"])
+        r_o, r_g = recall_at_k(oi, truth), recall_at_k(gi, truth)
+        assert abs(r_o - r_g) <= 0.005, (r_o, r_g)
+        assert r_g > 0.8
+        for i in range(0, len(q), 7):
+            b = base[gi[i]].astype(np.float64)
+            qq = q[i].astype(np.float64)
+            exact = ((b - qq) ** 2).sum(1) if cfg["metric"] == go.L2 else -(b @ qq)
+            scale_ = np.abs(exact) if cfg["metric"] == go.L2 else np.linalg.norm(b, axis=1) * np.linalg.norm(qq)
+            assert (np.abs(gd[i] - exact) <= 1e-5 * scale_).all()
+    else:
+        q = wl.queries()
+        oi, _ = o.search(q, 10, cfg["L"])
+        gi, _ = gpu_search(g, q, 10, cfg["L"])
+        overlap = np.mean([len(set(a.tolist()) & set(b.tolist())) / 10 for a, b in zip(oi, gi)])
+        assert overlap > 0.97, overlap
+
+
+# ------------------------------------------------------------------ errors, host API, determinism
+def test_errors_leave_index_unchanged():
+    torch = torch_()
+    from paper_2608_21163_b200.binding import GrandError
+    cfg = small_cfg("tiny_u8_d32", 0.05)
+    o, g, wl, st = run_stream(dict(cfg, rounds=0), seed=2)
+    n = cfg["n"]
+    before = gpu_graph(g)
+    v = wl.vectors(0, 4)
+    cases = [(np.array([n + 7, 1], np.uint32), -2), (np.array([0, 1], np.uint32), -4)]
+    for ids, code in cases:
+        with pytest.raises(GrandError) as e:
+            g.insert_batch(torch.from_numpy(ids), torch.from_numpy(v[:len(ids)]))
+        assert e.value.code == code
+    d = np.array([3], np.uint32)
+    o.delete_batch(d); g.delete_batch(torch.from_numpy(d))
+    with pytest.raises(GrandError) as e:
+        g.insert_batch(torch.from_numpy(np.array([3, 3], np.uint32)), torch.from_numpy(v[:2]))
+    assert e.value.code == -3
+    with pytest.raises(GrandError) as e:
+        g.delete_batch(torch.from_numpy(d))
+    assert e.value.code == -5
+    with pytest.raises(GrandError) as e:
+        g.delete_batch(torch.from_numpy(np.array([5, 5], np.uint32)))
+    assert e.value.code == -3
+    assert_same_graph(o, g, "after failed calls")
+    with pytest.raises(GrandError):
+        g.search(torch.from_numpy(v), 20, 10)
+    # the index still works
+    o.insert_batch(d, v[:1]); g.insert_batch(torch.from_numpy(d), torch.from_numpy(v[:1]))
+    assert_same_graph(o, g, "after recovery")
+
+
+def test_host_entry_points_match_device_entry_points():
+    torch = torch_()
+    cfg = small_cfg("tiny_u8_d32", 0.1, rounds=0)
+    wl = synth.Workload(cfg, 3)
+    n = cfg["n"]
+    base = wl.vectors(0, n)
+    o, g = make_pair(dict(cfg, max_build_batch=500, ins=500, dele=500), n)
+    for lo in range(0, n, 250):
+        ids = np.arange(lo, lo + 250, dtype=np.uint32)
+        o.insert_batch(ids, base[ids])
+        g.insert_batch_host(torch.from_numpy(ids).pin_memory(), torch.from_numpy(base[ids]).pin_memory())
+    dele = synth.choose_ids(3, "del", np.arange(n, dtype=np.uint32), 100)
+    o.delete_batch(dele)
+    g.delete_batch_host(torch.from_numpy(dele).pin_memory())
+    assert_same_graph(o, g, "host calls")
+    q = wl.queries()
+    out_i = torch.empty((len(q), 10), dtype=torch.uint32).pin_memory()
+    out_d = torch.empty((len(q), 10), dtype=torch.int32).pin_memory()
+    g.search_host(torch.from_numpy(q).pin_memory(), 10, cfg["L"], out_i, out_d)
+    oi, od = o.search(q, 10, cfg["L"])
+    assert (oi == out_i.numpy()).all() and (od == out_d.numpy().astype(np.float64)).all()
+
+
+def test_run_twice_is_deterministic_and_counters_move():
+    cfg = small_cfg("sift_u8_d128", 0.005, rounds=1)
+    _, g1, wl, _ = run_stream(cfg, seed=7, oracle=False)
+    _, g2, _, _ = run_stream(cfg, seed=7, oracle=False)
+    a, b = gpu_graph(g1), gpu_graph(g2)
+    assert (a[0] == b[0]).all() and (a[1] == b[1]).all() and a[3] == b[3]
+    s = g1.stats()
+    assert s["expansions"] > 0 and s["dist_evals"] > s["expansions"] and s["pair_dists"] > 0
+    assert s["dirty_nodes"] > 0 and s["prunes"] > 0 and s["kernel_launches"] > 0
