@@ -57,6 +57,7 @@ struct grand_index {
   // index state
   uint8_t* store = nullptr;
   uint32_t *adj = nullptr, *deg = nullptr, *live = nullptr;
+  uint8_t* rowpfx = nullptr;
   DevState* d_state = nullptr;
   DevState* h_state = nullptr;  // pinned mirror
   uint32_t entry = GRAND_INVALID_ID;
@@ -133,7 +134,7 @@ int ensure(grand_index* idx, Buf& b, size_t bytes, cudaStream_t s) {
 
 GraphView view(const grand_index* idx) {
   GraphView g;
-  g.store = idx->store; g.adj = idx->adj; g.deg = idx->deg; g.live = idx->live; g.R = idx->R; g.cap = idx->cap;
+  g.store = idx->store; g.adj = idx->adj; g.deg = idx->deg; g.live = idx->live; g.rowpfx = idx->rowpfx; g.R = idx->R; g.cap = idx->cap;
   return g;
 }
 
@@ -183,6 +184,7 @@ int write_state_head(grand_index* idx, cudaStream_t s) {
   idx->h_state->entry = idx->entry;
   idx->h_state->ndirty = 0;
   idx->h_state->cursor = 0;
+  idx->h_state->work = 0;
   idx->h_state->nlive = idx->nlive;
   idx->h_state->total_in = 0;
   CK(cudaMemcpyAsync(idx->d_state, idx->h_state, offsetof(DevState, medoid_key), cudaMemcpyHostToDevice, s));
@@ -261,7 +263,8 @@ int grand_create_ex(uint32_t dim, uint32_t dtype, uint32_t metric, uint32_t R, u
   idx->dev_free = o->dev_free ? o->dev_free : default_free;
   idx->user = o->user;
   if (idx->cap >= (1ull << 31) || idx->cap * R >= (1ull << 32) || idx->P > 256 || idx->c > 8 || idx->k_repair > 128 ||
-      idx->k_repair > L || idx->vmax > 1024 || idx->vmax == 0 || idx->hash_bits < 10 || idx->hash_bits > 13 ||
+      idx->k_repair > L || idx->vmax > 1024 || idx->vmax == 0 || idx->hash_bits < 8 || idx->hash_bits > 13 ||
+      (4u << idx->hash_bits) < lay.row_bytes ||
       idx->max_batch * R >= (1ull << 32)) {
     delete idx;
     return GRAND_ERR_INVALID_ARG;
@@ -275,6 +278,7 @@ int grand_create_ex(uint32_t dim, uint32_t dtype, uint32_t metric, uint32_t R, u
   A(alloc_dev(idx, &idx->adj, (size_t)cap * R, false));
   A(alloc_dev(idx, &idx->deg, cap, true));
   A(alloc_dev(idx, &idx->live, words, true));
+  A(alloc_dev(idx, &idx->rowpfx, cap, true));
   A(alloc_dev(idx, &idx->d_state, 1, true));
   A(alloc_dev(idx, &idx->mark, words, true));
   A(alloc_dev(idx, &idx->cnt, cap, true));
@@ -602,6 +606,8 @@ int grand_import_graph(grand_index* idx, const uint32_t* adj, const uint32_t* de
   CK(cudaMemcpyAsync(idx->deg, deg, idx->cap * 4, cudaMemcpyDeviceToDevice, s));
   CK(cudaMemcpyAsync(idx->live, live, (idx->cap + 31) / 32 * 4, cudaMemcpyDeviceToDevice, s));
   CK(launch_pad_rows(idx->lay, idx->store, vecs, idx->cap, s));
+  CK(cudaMemsetAsync(idx->rowpfx, 0, idx->cap, s));
+  CK(launch_pad_adjacency(idx->adj, idx->deg, idx->cap, idx->R, s));
   idx->entry = entry;
   idx->nlive = 0;
   int rc;

@@ -133,6 +133,34 @@ __device__ __forceinline__ void bitonic_sort_any(K* a, uint32_t n, uint32_t tid,
   }
 }
 
+// the same network ordering 64-bit keys by their clean value (bit 31 of the id word rides along as a tag)
+template <typename SyncFn>
+__device__ __forceinline__ void bitonic_sort_clean(unsigned long long* a, uint32_t n, uint32_t tid, uint32_t nthreads, SyncFn sync) {
+  if (n < 2) return;
+  uint32_t m = 1;
+  while (m < n) m <<= 1;
+  for (uint32_t k = 2; k <= m; k <<= 1) {
+    for (uint32_t i = tid; i < n; i += nthreads) {
+      uint32_t p = i ^ (k - 1);
+      if (p > i && p < n) {
+        unsigned long long x = a[i], y = a[p];
+        if (key_clean(y) < key_clean(x)) { a[i] = y; a[p] = x; }
+      }
+    }
+    sync();
+    for (uint32_t j = k >> 2; j > 0; j >>= 1) {
+      for (uint32_t i = tid; i < n; i += nthreads) {
+        uint32_t p = i ^ j;
+        if (p > i && p < n) {
+          unsigned long long x = a[i], y = a[p];
+          if (key_clean(y) < key_clean(x)) { a[i] = y; a[p] = x; }
+        }
+      }
+      sync();
+    }
+  }
+}
+
 // first index in sorted a[0..n) whose clean key is >= k
 __device__ __forceinline__ uint32_t lower_bound_clean(const unsigned long long* a, uint32_t n, unsigned long long k) {
   uint32_t lo = 0, hi = n;

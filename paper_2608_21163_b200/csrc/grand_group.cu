@@ -361,6 +361,20 @@ cudaError_t launch_count_live(const uint32_t* live, uint64_t cap, DevState* st, 
   return cudaGetLastError();
 }
 
+// rows are read whole by the search kernel: every slot at or beyond deg must hold the invalid id
+__global__ void pad_adjacency_kernel(uint32_t* adj, const uint32_t* deg, uint64_t cap, uint32_t R) {
+  const uint64_t total = cap * R;
+  for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < total; i += (uint64_t)gridDim.x * blockDim.x) {
+    const uint64_t v = i / R;
+    if ((uint32_t)(i - v * R) >= deg[v]) adj[i] = kInvalid;
+  }
+}
+cudaError_t launch_pad_adjacency(uint32_t* adj, const uint32_t* deg, uint64_t cap, uint32_t R, cudaStream_t s) {
+  pad_adjacency_kernel<<<grid_for(cap * R), kThreads, 0, s>>>(adj, deg, cap, R);
+  count_launches(1);
+  return cudaGetLastError();
+}
+
 __global__ void fill_u32_kernel(uint32_t* p, uint32_t v, uint64_t n) {
   for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < n; i += (uint64_t)gridDim.x * blockDim.x) p[i] = v;
 }

@@ -27,6 +27,8 @@ struct DevState {
   uint32_t entry;        // medoid
   uint32_t ndirty;       // length of the dirty list
   uint32_t cursor;       // segment allocator for grouped requests
+  uint32_t work;         // dynamic work counter of the rebuild kernel
+  uint32_t pad_;
   unsigned long long nlive;
   unsigned long long total_in;   // sum of in-degrees of the delete batch
   unsigned long long medoid_key; // argmin scratch
@@ -39,6 +41,8 @@ struct GraphView {
   uint32_t* adj;
   uint32_t* deg;
   uint32_t* live;  // bitmap
+  uint8_t* rowpfx;  // per row: length of the leading run that is a RobustPrune output in ascending key
+                    // order (no member of the run prunes a later member); appended entries follow it
   uint32_t R;
   uint64_t cap;
 };
@@ -185,6 +189,7 @@ cudaError_t launch_pick_medoid(const Layout& lay, const GraphView& g, const uint
                                DevState* st, cudaStream_t s);
 cudaError_t launch_count_live(const uint32_t* live, uint64_t cap, DevState* st, cudaStream_t s);
 cudaError_t launch_pad_rows(const Layout& lay, uint8_t* store, const void* vecs, uint64_t n, cudaStream_t s);
+cudaError_t launch_pad_adjacency(uint32_t* adj, const uint32_t* deg, uint64_t cap, uint32_t R, cudaStream_t s);
 cudaError_t launch_fill_u32(uint32_t* p, uint32_t v, uint64_t n, cudaStream_t s);
 
 }  // namespace grand

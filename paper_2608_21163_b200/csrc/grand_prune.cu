@@ -126,7 +126,10 @@ __global__ void __launch_bounds__(kPruneThreads) forward_prune_kernel(const Prun
       a.req_tgt[i * R + s] = id;
       a.req_key[i * R + s] = rk;
     }
-    if (tid == 0) a.g.deg[p] = cnt;
+    if (tid == 0) {
+      a.g.deg[p] = cnt;
+      a.g.rowpfx[p] = a.fixed_mode ? 0 : (uint8_t)cnt;
+    }
     __syncthreads();
   }
   if (npair) atomicAdd(&a.state->counters[CTR_PAIR], npair);
@@ -162,144 +165,6 @@ __device__ __forceinline__ unsigned long long* sort_segment(unsigned long long* 
   return seg;
 }
 
-// Rebuild of dirty nodes: C = (N_out(u) \ B) ++ (scratch_u \ N_out(u) \ {u}); store C if it fits R,
-// else compute D_u for the old neighbours (requests already carry dist(u, id)) and prune.
-template <typename T, int METRIC, int G, int CPL>
-__global__ void __launch_bounds__(kPruneThreads) rebuild_kernel(const RebuildArgs a) {
-  using Dist = typename Elem<T>::Dist;
-  constexpr unsigned FULL = 0xFFFFFFFFu;
-  __shared__ unsigned long long seg_smem[kSegCap];
-  __shared__ unsigned long long scratch[kMaxP];
-  __shared__ unsigned long long cand[kMaxR + kMaxP];
-  __shared__ uint32_t keep[kMaxR];
-  __shared__ uint32_t validw[(kMaxR + kMaxP) / 32];
-  __shared__ uint32_t out_idx[kMaxR];
-  __shared__ uint32_t sh_sel, sh_ns, sh_nk, sh_nf;
-  const uint32_t tid = threadIdx.x, nthreads = blockDim.x;
-  const int lane = tid & 31, warp = tid >> 5;
-  const int t = lane % G;
-  const uint32_t team_global = tid / G, nteams = nthreads / G;
-  const uint32_t R = a.g.R;
-  const AlphaParam ap{a.A_fix, a.alpha};
-  const uint32_t row_bytes = a.lay.row_bytes, nchunk = a.lay.nchunk;
-  unsigned long long npair = 0;
-  uint32_t nprune = 0, ndone = 0;
-  auto sync = [] { __syncthreads(); };
-  const uint32_t ndirty = a.state->ndirty;
-  for (uint32_t k = blockIdx.x; k < ndirty; k += gridDim.x) {
-    const uint32_t u = a.dirty[k];
-    const uint32_t cntu = a.cnt[u];
-    unsigned long long* seg = sort_segment(a.seg_keys + a.start[u], cntu, seg_smem);
-    // scratch_u: first P distinct requests in key order (equal pairs are adjacent after the sort)
-    if (tid == 0) {
-      uint32_t ns = 0;
-      unsigned long long prev = kKeyMax;
-      for (uint32_t j = 0; j < cntu && ns < a.P; ++j) {
-        const unsigned long long kk = seg[j];
-        if (kk != prev) scratch[ns++] = kk;
-        prev = kk;
-      }
-      sh_ns = ns;
-    }
-    // keep = N_out(u) \ B, stable
-    if (warp == 1 || nthreads == 32) {
-      const uint32_t du = min(a.g.deg[u], R);
-      const uint32_t* row = a.g.adj + (size_t)u * R;
-      uint32_t nk = 0;
-      for (uint32_t sb = 0; sb < du; sb += 32) {
-        const uint32_t s = sb + lane;
-        uint32_t v = kInvalid;
-        bool ok = false;
-        if (s < du) {
-          v = row[s];
-          ok = !(a.delmap && bit_test(a.delmap, v));
-        }
-        const unsigned bal = __ballot_sync(FULL, ok);
-        if (ok) keep[nk + __popc(bal & ((1u << lane) - 1u))] = v;
-        nk += __popc(bal);
-      }
-      if (lane == 0) sh_nk = nk;
-    }
-    __syncthreads();
-    const uint32_t ns = sh_ns, nk = sh_nk;
-    // fresh = scratch \ keep \ {u}, stable, appended after the keep slots of cand
-    if (warp == 0) {
-      uint32_t nf = 0;
-      for (uint32_t jb = 0; jb < ns; jb += 32) {
-        const uint32_t j = jb + lane;
-        bool ok = false;
-        unsigned long long kk = 0;
-        if (j < ns) {
-          kk = scratch[j];
-          const uint32_t id = key_id(kk);
-          ok = id != u;
-          for (uint32_t x = 0; ok && x < nk; ++x) ok = keep[x] != id;
-        }
-        const unsigned bal = __ballot_sync(FULL, ok);
-        if (ok) cand[nk + nf + __popc(bal & ((1u << lane) - 1u))] = kk;
-        nf += __popc(bal);
-      }
-      if (lane == 0) sh_nf = nf;
-    }
-    __syncthreads();
-    const uint32_t nf = sh_nf, nC = nk + nf;
-    uint32_t* row_out = a.g.adj + (size_t)u * R;
-    if (nC <= R) {
-      for (uint32_t s = tid; s < R; s += nthreads)
-        row_out[s] = s < nk ? keep[s] : (s < nC ? key_id(cand[s]) : kInvalid);
-      if (tid == 0) a.g.deg[u] = nC;
-    } else {
-      // D_u for the kept neighbours
-      uint4 ur[CPL];
-      load_row<G, CPL>(a.g.store + (size_t)u * row_bytes, nchunk, t, ur);
-      for (uint32_t jb = 0; jb < nk; jb += nteams) {
-        const uint32_t j = jb + team_global;
-        const bool act = j < nk;
-        uint4 v[CPL];
-        if (act) {
-          load_row<G, CPL>(a.g.store + (size_t)keep[j] * row_bytes, nchunk, t, v);
-        } else {
-#pragma unroll
-          for (int c = 0; c < CPL; ++c) v[c] = make_uint4(0, 0, 0, 0);
-        }
-        const Dist d = team_dist_regs<T, kMetricL2, G, CPL>(ur, v);
-        if (act && t == 0) {
-          cand[j] = make_key(d, keep[j]);
-          ++npair;
-        }
-      }
-      __syncthreads();
-      bitonic_sort_any(cand, nC, tid, nthreads, sync);
-      const uint32_t cnt = block_prune<T, G, CPL>(a.g.store, row_bytes, nchunk, ap, cand, nC, R, validw, out_idx, &sh_sel, npair);
-      ++nprune;
-      for (uint32_t s = tid; s < R; s += nthreads) row_out[s] = s < cnt ? key_id(cand[out_idx[s]]) : kInvalid;
-      if (tid == 0) a.g.deg[u] = cnt;
-    }
-    if (tid == 0) {
-      a.cnt[u] = 0;
-      a.fill[u] = 0;
-      a.flag[u] = 0;
-      ++ndone;
-    }
-    __syncthreads();
-  }
-  if (npair) atomicAdd(&a.state->counters[CTR_PAIR], npair);
-  if (tid == 0) {
-    if (nprune) atomicAdd(&a.state->counters[CTR_PRUNE], (unsigned long long)nprune);
-    if (ndone) atomicAdd(&a.state->counters[CTR_DIRTY], (unsigned long long)ndone);
-  }
-}
-
-template <typename T, int METRIC, int G, int CPL>
-static cudaError_t launch_rebuild_t(const RebuildArgs& a, cudaStream_t s) {
-  rebuild_kernel<T, METRIC, G, CPL><<<a.max_blocks, kPruneThreads, 0, s>>>(a);
-  count_launches(1);
-  return cudaGetLastError();
-}
-cudaError_t launch_rebuild(const RebuildArgs& a, cudaStream_t s) {
-  GRAND_DISPATCH_L2(a.lay, launch_rebuild_t, a, s);
-  return cudaErrorInvalidValue;
-}
 
 // Fixed-degree backward edges (Alg. 7): the owner of target q takes its requests in (dist, id)
 // order; a request from new node p appends while deg(q) < R, else replaces the highest-index slot

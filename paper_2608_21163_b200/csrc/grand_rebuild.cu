@@ -1,0 +1,295 @@
+// Rebuild of dirty nodes (Alg. 5 dirty loop, Alg. 6 rebuild loop): one WARP owns one dirty node.
+//
+// C = (N_out(u) \ B) ++ (scratch_u \ N_out(u) \ {u}); if |C| <= R the row is stored as is, else D_u is
+// computed for the kept neighbours (requests already carry dist(u, id)) and GrANDRobustPrune
+// (Alg. 4) runs on C.  The prune is restructured for the GPU without changing its result:
+//
+//  * p* is always the first valid candidate in key order, so only the outcomes of the tests
+//    alpha * dist(c_i, c_j) <= D_u[c_j] for i < j can ever matter.  They are independent of each
+//    other, so the warp evaluates them in parallel into a bit matrix in shared memory and then
+//    replays the sequential selection on bit masks.
+//  * Every row remembers how long its leading run of prune output is (rowpfx).  Two members of
+//    that run both survived an earlier prune of this very node, which means the earlier one does
+//    not prune the later one; distances and D_u are recomputed to the same bits, so those tests
+//    are known to be false and only pairs with an "uncertain" member (appended since, or fresh)
+//    are evaluated.
+//
+// Dirty nodes are handed out through an atomic work counter because a node that prunes costs far
+// more than one that only appends.
+#include "grand_common.cuh"
+#include "grand_kernels.h"
+
+namespace grand {
+
+constexpr int kRebuildWarps = 4;
+constexpr uint32_t kSegSmem = 128;       // request segments up to this length are sorted in shared memory
+constexpr uint32_t kMaxUncertain = 256;  // capacity of the uncertain-position list (aliases the segment buffer)
+
+static inline uint32_t even_up_h(uint32_t x) { return (x + 1u) & ~1u; }
+static size_t rebuild_smem_per_warp(uint32_t R, uint32_t P) {
+  const size_t NM = R + P, W = (NM + 31) / 32, Rp = even_up_h(R);
+  size_t b = (size_t)kSegSmem * 8 + (size_t)P * 8 + NM * 8 + Rp * 4 * 2 + NM * W * 4;
+  return (b + 15) / 16 * 16;
+}
+
+template <typename T, int METRIC, int G, int CPL>
+__global__ void __launch_bounds__(kRebuildWarps * 32) rebuild_kernel(const RebuildArgs a, const uint32_t per_warp_bytes) {
+  using Dist = typename Elem<T>::Dist;
+  constexpr unsigned FULL = 0xFFFFFFFFu;
+  constexpr int NT = 32 / G;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int t = lane % G, team = lane / G;
+  const uint32_t lt_mask = (1u << lane) - 1u;
+  const uint32_t R = a.g.R, P = a.P, NM = R + P, W = (NM + 31) >> 5, Rp = (R + 1u) & ~1u;
+  unsigned char* base = smem_raw + (size_t)warp * per_warp_bytes;
+  unsigned long long* seg_s = reinterpret_cast<unsigned long long*>(base);
+  unsigned long long* scratch = seg_s + kSegSmem;
+  unsigned long long* cand = scratch + P;
+  uint32_t* keep = reinterpret_cast<uint32_t*>(cand + NM);
+  uint32_t* out_idx = keep + Rp;
+  uint32_t* prune = out_idx + Rp;  // NM rows x W words: bit j of row i = "c_i prunes c_j"
+  uint32_t* upos = reinterpret_cast<uint32_t*>(seg_s);  // positions of uncertain candidates (segment buffer is free by then)
+  const AlphaParam ap{a.A_fix, a.alpha};
+  const uint32_t row_bytes = a.lay.row_bytes, nchunk = a.lay.nchunk;
+  const uint8_t* __restrict__ store = a.g.store;
+  auto wsync = [] { __syncwarp(); };
+  unsigned long long npair = 0;
+  uint32_t nprune = 0, ndone = 0;
+  const uint32_t ndirty = a.state->ndirty;
+
+  // one prune test: rows of candidates i < j (sorted positions), result into the bit matrix
+  auto pair_test = [&](bool act, uint32_t i, uint32_t j, uint32_t& jprev, uint4 (&rj)[CPL]) {
+    uint4 ri[CPL];
+    if (act) {
+      if (j != jprev) {
+        load_row<G, CPL>(store + (size_t)key_id(cand[j]) * row_bytes, nchunk, t, rj);
+        jprev = j;
+      }
+      load_row<G, CPL>(store + (size_t)key_id(cand[i]) * row_bytes, nchunk, t, ri);
+    } else {
+#pragma unroll
+      for (int c = 0; c < CPL; ++c) ri[c] = make_uint4(0, 0, 0, 0);
+    }
+    const Dist d = team_dist_regs<T, kMetricL2, G, CPL>(ri, rj);
+    if (act && t == 0) {
+      ++npair;
+      if (alpha_test(ap, d, key_dist<Dist>(cand[j]))) atomicOr(&prune[i * W + (j >> 5)], 1u << (j & 31));
+    }
+  };
+
+  for (;;) {
+    uint32_t k = 0;
+    if (lane == 0) k = atomicAdd(&a.state->work, 1u);
+    k = __shfl_sync(FULL, k, 0);
+    if (k >= ndirty) break;
+    const uint32_t u = a.dirty[k];
+    const uint32_t cntu = a.cnt[u];
+    // ---- scratch_u: sort the request segment by (dist, id), keep the first P distinct entries
+    unsigned long long* seg = a.seg_keys + a.start[u];
+    if (cntu <= kSegSmem) {
+      for (uint32_t j = lane; j < cntu; j += 32) seg_s[j] = seg[j];
+      seg = seg_s;
+    }
+    __syncwarp();
+    bitonic_sort_any(seg, cntu, (uint32_t)lane, 32u, wsync);
+    uint32_t ns = 0;
+    for (uint32_t jb = 0; jb < cntu && ns < P; jb += 32) {
+      const uint32_t j = jb + lane;
+      bool ok = j < cntu;
+      unsigned long long kk = 0;
+      if (ok) {
+        kk = seg[j];
+        if (j > 0 && seg[j - 1] == kk) ok = false;  // equal requests are adjacent after the sort
+      }
+      const unsigned bal = __ballot_sync(FULL, ok);
+      const uint32_t pos = ns + __popc(bal & lt_mask);
+      if (ok && pos < P) scratch[pos] = kk;
+      ns += __popc(bal);
+    }
+    ns = min(ns, P);
+    // ---- keep = N_out(u) \ B, stable; kp = how many kept entries come from the pruned prefix
+    const uint32_t du = min(a.g.deg[u], R);
+    const uint32_t pfx = min((uint32_t)a.g.rowpfx[u], du);
+    uint32_t* row = a.g.adj + (size_t)u * R;
+    uint32_t nk = 0, kp = 0;
+    for (uint32_t sb = 0; sb < du; sb += 32) {
+      const uint32_t s = sb + lane;
+      uint32_t v = kInvalid;
+      bool ok = false;
+      if (s < du) {
+        v = row[s];
+        ok = !(a.delmap && bit_test(a.delmap, v));
+      }
+      const unsigned bal = __ballot_sync(FULL, ok);
+      if (ok) keep[nk + __popc(bal & lt_mask)] = v;
+      nk += __popc(bal);
+      kp += __popc(__ballot_sync(FULL, ok && s < pfx));
+    }
+    __syncwarp();
+    // ---- fresh = scratch \ keep \ {u}, stable, placed after the keep slots of cand (tagged uncertain)
+    uint32_t nf = 0;
+    for (uint32_t jb = 0; jb < ns; jb += 32) {
+      const uint32_t j = jb + lane;
+      bool ok = false;
+      unsigned long long kk = 0;
+      if (j < ns) {
+        kk = scratch[j];
+        const uint32_t id = key_id(kk);
+        ok = id != u;
+        for (uint32_t x = 0; ok && x < nk; ++x) ok = keep[x] != id;
+      }
+      const unsigned bal = __ballot_sync(FULL, ok);
+      if (ok) cand[nk + nf + __popc(bal & lt_mask)] = kk | kExpandedBit;
+      nf += __popc(bal);
+    }
+    __syncwarp();
+    const uint32_t nC = nk + nf;
+    if (nC <= R) {
+      for (uint32_t s = lane; s < R; s += 32) row[s] = s < nk ? keep[s] : (s < nC ? key_id(cand[s]) : kInvalid);
+      if (lane == 0) {
+        a.g.deg[u] = nC;
+        a.g.rowpfx[u] = (uint8_t)kp;  // the surviving part of the pruned run still leads the row
+      }
+    } else {
+      // ---- D_u for the kept neighbours (those appended after the last prune are tagged uncertain)
+      {
+        uint4 ur[CPL];
+        load_row<G, CPL>(store + (size_t)u * row_bytes, nchunk, t, ur);
+        for (uint32_t jb = 0; jb < nk; jb += NT) {
+          const uint32_t j = jb + team;
+          const bool act = j < nk;
+          uint4 v[CPL];
+          if (act) {
+            load_row<G, CPL>(store + (size_t)keep[j] * row_bytes, nchunk, t, v);
+          } else {
+#pragma unroll
+            for (int c = 0; c < CPL; ++c) v[c] = make_uint4(0, 0, 0, 0);
+          }
+          const Dist d = team_dist_regs<T, kMetricL2, G, CPL>(ur, v);
+          if (act && t == 0) {
+            cand[j] = make_key(d, keep[j]) | (j >= kp ? kExpandedBit : 0ull);
+            ++npair;
+          }
+        }
+      }
+      __syncwarp();
+      bitonic_sort_clean(cand, nC, (uint32_t)lane, 32u, wsync);
+      for (uint32_t w = lane; w < nC * W; w += 32) prune[w] = 0u;
+      // ---- prune tests in parallel: pairs with an uncertain member, or the whole upper triangle
+      const uint32_t nu = nC - kp;
+      uint32_t jprev = kInvalid;
+      uint4 rj[CPL];
+#pragma unroll
+      for (int c = 0; c < CPL; ++c) rj[c] = make_uint4(0, 0, 0, 0);
+      if (nu <= kMaxUncertain && 2 * nu + 1 < nC) {
+        uint32_t nfound = 0;
+        for (uint32_t jb = 0; jb < nC; jb += 32) {
+          const uint32_t j = jb + lane;
+          const bool un = j < nC && (cand[j] & kExpandedBit);
+          const unsigned bal = __ballot_sync(FULL, un);
+          if (un) upos[nfound + __popc(bal & lt_mask)] = j;
+          nfound += __popc(bal);
+        }
+        __syncwarp();
+        const uint32_t nwork = nu * nC;
+        for (uint32_t eb = 0; eb < nwork; eb += NT) {
+          const uint32_t e = eb + team;
+          bool act = e < nwork;
+          uint32_t i = 0, j = 1;
+          if (act) {
+            const uint32_t f = upos[e / nC], x = e % nC;
+            // skip self; a pair of two uncertain members is taken once, from its larger member
+            act = f != x && !(x > f && (cand[x] & kExpandedBit));
+            i = min(f, x);
+            j = max(f, x);
+          }
+          pair_test(act, i, j, jprev, rj);
+        }
+      } else {
+        __syncwarp();
+        const uint32_t npairs = nC * (nC - 1) / 2;
+        for (uint32_t pb = 0; pb < npairs; pb += NT) {
+          const uint32_t p = pb + team;
+          const bool act = p < npairs;
+          uint32_t i = 0, j = 1;
+          if (act) {
+            j = (uint32_t)((1.0f + sqrtf(1.0f + 8.0f * (float)p)) * 0.5f);
+            while (j * (j - 1) / 2 > p) --j;
+            while ((j + 1) * j / 2 <= p) ++j;
+            i = p - j * (j - 1) / 2;
+          }
+          pair_test(act, i, j, jprev, rj);
+        }
+      }
+      __syncwarp();
+      // ---- sequential selection replayed on bit masks (lane w holds word w of the valid set)
+      uint32_t valid = 0;
+      if ((uint32_t)lane < W) {
+        const uint32_t lo = lane * 32;
+        valid = nC >= lo + 32 ? 0xFFFFFFFFu : (nC > lo ? (1u << (nC - lo)) - 1u : 0u);
+      }
+      uint32_t cnt = 0;
+      for (uint32_t i = 0; i < nC; ++i) {
+        const uint32_t word = __shfl_sync(FULL, valid, i >> 5);
+        if (!((word >> (i & 31)) & 1u)) continue;
+        if (lane == 0) out_idx[cnt] = i;
+        ++cnt;
+        if (cnt == R) break;
+        if ((uint32_t)lane < W) valid &= ~prune[i * W + lane];
+      }
+      __syncwarp();
+      for (uint32_t s = lane; s < R; s += 32) row[s] = s < cnt ? key_id(cand[out_idx[s]]) : kInvalid;
+      if (lane == 0) {
+        a.g.deg[u] = cnt;
+        a.g.rowpfx[u] = (uint8_t)cnt;
+      }
+      ++nprune;
+    }
+    if (lane == 0) {
+      a.cnt[u] = 0;
+      a.fill[u] = 0;
+      a.flag[u] = 0;
+    }
+    ++ndone;
+    __syncwarp();
+  }
+  if (npair) atomicAdd(&a.state->counters[CTR_PAIR], npair);
+  if (lane == 0) {
+    if (nprune) atomicAdd(&a.state->counters[CTR_PRUNE], (unsigned long long)nprune);
+    if (ndone) atomicAdd(&a.state->counters[CTR_DIRTY], (unsigned long long)ndone);
+  }
+}
+
+template <typename T, int METRIC, int G, int CPL>
+static cudaError_t launch_rebuild_t(const RebuildArgs& a, cudaStream_t s) {
+  const size_t per_warp = rebuild_smem_per_warp(a.g.R, a.P);
+  const size_t smem = per_warp * kRebuildWarps;
+  auto kern = rebuild_kernel<T, METRIC, G, CPL>;
+  static size_t smem_set = 0;
+  static int sm_count = 0;
+  if (smem > smem_set) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    smem_set = smem;
+  }
+  if (!sm_count) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
+  }
+  int occ = 1;
+  cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, kRebuildWarps * 32, smem);
+  if (occ < 1) occ = 1;
+  uint32_t blocks = (uint32_t)sm_count * occ;
+  if (blocks > a.max_blocks && a.max_blocks) blocks = a.max_blocks;
+  kern<<<blocks, kRebuildWarps * 32, smem, s>>>(a, (uint32_t)per_warp);
+  count_launches(1);
+  return cudaGetLastError();
+}
+cudaError_t launch_rebuild(const RebuildArgs& a, cudaStream_t s) {
+  GRAND_DISPATCH_L2(a.lay, launch_rebuild_t, a, s);
+  return cudaErrorInvalidValue;
+}
+
+}  // namespace grand

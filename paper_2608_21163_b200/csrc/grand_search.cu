@@ -1,15 +1,21 @@
 // Batched greedy beam search (BeamSearch, Alg. 1): one warp per query.
 //
 // Per warp, in shared memory: the sorted worklist C (L keys; the expanded flag rides in bit 31 of
-// the id word), a direct-mapped visited cache that may forget but never lies (full ids), and the
-// candidate staging arrays of one expansion.  One expansion = read the adjacency row of the best
-// unexpanded entry, drop ids the cache has seen, gather the surviving neighbours' vectors with
-// 128-bit loads (a team of G lanes per vector, several vectors in flight per lane), reduce the
-// distances with shuffles, and merge the survivors into the worklist in parallel.
+// the id word), a visited cache that may forget but never lies, and the candidate staging arrays
+// of one expansion.  One expansion = read the adjacency row of the best unexpanded entry, drop ids
+// the cache has seen, gather the surviving neighbours' vectors with 128-bit loads (a team of G
+// lanes per vector, several vectors in flight per lane), reduce the distances with shuffles, and
+// merge the survivors into the worklist in parallel.
 //
 // The worklist always equals the L smallest (dist, id) keys seen so far, so the result does not
 // depend on what the cache forgets: a re-evaluated node either matches an entry exactly (dropped
 // as a duplicate by key equality) or fails the comparison with the worst entry.
+//
+// Visited cache.  When every id fits 16 + (bucket bits) bits, the cache stores 16-bit tags in
+// buckets of 8: an odd multiplier is a bijection on that id range, its high bits pick the bucket
+// and its low 16 bits are the tag, so (bucket, tag) identifies the id exactly and a hit is never
+// false.  That doubles the entries per byte and makes forgetting rare.  Larger capacities fall
+// back to a direct-mapped table of full 32-bit ids.
 #include "grand_common.cuh"
 #include "grand_kernels.h"
 
@@ -24,6 +30,39 @@ size_t beam_search_smem_per_warp(uint32_t L, uint32_t R, uint32_t hash_bits) {
   return Lp * 8 + Rp * 8 + Rp * 8 + Rp * 4 + Rp * 4 + ((size_t)4 << hash_bits);
 }
 
+// Hint: bring one adjacency row (R ids) towards L2; lanes cover its 128-byte lines.
+__device__ __forceinline__ void prefetch_row(const uint32_t* row, uint32_t R, int lane) {
+  if ((uint32_t)lane * 32u < R) asm volatile("prefetch.global.L2 [%0];" ::"l"(row + lane * 32));
+}
+
+// Visited cache probe: returns true if v was not known (and records it).
+__device__ __forceinline__ bool visit_fresh(uint32_t* hash, uint32_t hash_bits, bool tags16, uint32_t v) {
+  if (tags16) {
+    const uint32_t ub = hash_bits + 14;  // bucket bits (hash_bits - 2) + 16 tag bits
+    const uint32_t h = (v * 0x9E3779B1u) & ((1u << ub) - 1u);
+    const uint32_t bucket = h >> 16, tag = h & 0xFFFFu;
+    if (tag == 0xFFFFu) return true;  // the empty marker cannot be stored: always re-evaluate
+    const uint4 b = reinterpret_cast<const uint4*>(hash)[bucket];
+    const uint32_t t2 = tag | (tag << 16);
+    if (__vcmpeq2(b.x, t2) | __vcmpeq2(b.y, t2) | __vcmpeq2(b.z, t2) | __vcmpeq2(b.w, t2)) return false;
+    // first empty half-word, else evict the slot the tag points at
+    const uint32_t e0 = __vcmpeq2(b.x, 0xFFFFFFFFu), e1 = __vcmpeq2(b.y, 0xFFFFFFFFu);
+    const uint32_t e2 = __vcmpeq2(b.z, 0xFFFFFFFFu), e3 = __vcmpeq2(b.w, 0xFFFFFFFFu);
+    uint32_t slot;
+    if (e0) slot = (e0 & 0xFFFFu) ? 0 : 1;
+    else if (e1) slot = (e1 & 0xFFFFu) ? 2 : 3;
+    else if (e2) slot = (e2 & 0xFFFFu) ? 4 : 5;
+    else if (e3) slot = (e3 & 0xFFFFu) ? 6 : 7;
+    else slot = tag & 7u;
+    reinterpret_cast<unsigned short*>(hash)[bucket * 8 + slot] = (unsigned short)tag;
+    return true;
+  }
+  const uint32_t h = (v * 2654435761u) >> (32 - hash_bits);
+  if (hash[h] == v) return false;
+  hash[h] = v;
+  return true;
+}
+
 template <typename T, int METRIC, int G, int CPL>
 __global__ void __launch_bounds__(kSearchWarps * 32) beam_search_kernel(const SearchArgs a, const uint32_t per_warp_bytes) {
   using Dist = typename Elem<T>::Dist;
@@ -34,18 +73,20 @@ __global__ void __launch_bounds__(kSearchWarps * 32) beam_search_kernel(const Se
 
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int t = lane % G, team = lane / G;
+  const uint32_t lt_mask = (1u << lane) - 1u;
   const uint32_t L = a.L, R = a.g.R, H = 1u << a.hash_bits;
   const uint32_t Lp = (L + 1u) & ~1u, Rp = (R + 1u) & ~1u;
   unsigned char* base = smem_raw + (size_t)warp * per_warp_bytes;
   unsigned long long* beam = reinterpret_cast<unsigned long long*>(base);
-  unsigned long long* ckey = beam + Lp;     // candidate keys of this expansion (unsorted)
+  unsigned long long* ckey = beam + Lp;     // candidate keys of this expansion, then the compacted survivors
   unsigned long long* cskey = ckey + Rp;    // surviving candidate keys, ascending
-  uint32_t* cid = reinterpret_cast<uint32_t*>(cskey + Rp);  // candidate ids, later their worklist ranks
+  uint32_t* cid = reinterpret_cast<uint32_t*>(cskey + Rp);  // candidate ids, later the survivors' worklist ranks
   uint32_t* csb = cid + Rp;                 // worklist rank of each sorted survivor
   uint32_t* hash = csb + Rp;                // visited cache (also query staging)
 
   const uint32_t nchunk = a.lay.nchunk, row_bytes = a.lay.row_bytes;
   const uint8_t* __restrict__ store = a.g.store;
+  const bool tags16 = a.g.cap <= (1ull << (a.hash_bits + 14));
   unsigned long long n_exp = 0, n_dist = 0;
 
   const uint64_t wglobal = (uint64_t)blockIdx.x * kSearchWarps + warp;
@@ -74,6 +115,7 @@ __global__ void __launch_bounds__(kSearchWarps * 32) beam_search_kernel(const Se
     __syncwarp();
 
     uint32_t beam_n = 0, nvis = 0, cursor = 0;
+    unsigned long long alt_key = kKeyMax;  // best unexpanded entry besides the one being expanded
 
     // Evaluate cid[0..n) against the query and merge the survivors into the worklist.
     auto process = [&](uint32_t n) {
@@ -100,39 +142,52 @@ __global__ void __launch_bounds__(kSearchWarps * 32) beam_search_kernel(const Se
       }
       n_dist += n;
       __syncwarp();
-      // 2. keep keys below the worst entry that are not already in the worklist
+      // 2. keep keys below the worst entry that are not already in the worklist; compact them in
+      //    place (a write never passes the reader of its own chunk) and remember their ranks
       const unsigned long long worst = beam_n == L ? key_clean(beam[L - 1]) : kKeyMax;
       uint32_t m = 0;
+      unsigned long long best = kKeyMax;
       for (uint32_t jb = 0; jb < n; jb += 32) {
         const uint32_t j = jb + lane;
         bool pass = false;
+        unsigned long long key = 0;
+        uint32_t b = 0;
         if (j < n) {
-          const unsigned long long key = ckey[j];
+          key = ckey[j];
           pass = key < worst;
           if (pass) {
-            const uint32_t b = lower_bound_clean(beam, beam_n, key);
+            b = lower_bound_clean(beam, beam_n, key);
             if (b < beam_n && key_clean(beam[b]) == key) pass = false;
-            cid[j] = b;
           }
-          if (!pass) ckey[j] = kKeyMax;
         }
-        m += __popc(__ballot_sync(FULL, pass));
+        const unsigned bal = __ballot_sync(FULL, pass);
+        if (pass) {
+          const uint32_t pos = m + __popc(bal & lt_mask);
+          ckey[pos] = key;
+          cid[pos] = b;
+          best = min(best, key);
+        }
+        m += __popc(bal);
       }
       __syncwarp();
       if (m == 0) return;
-      // rank survivors among themselves (counting sort by comparison; n <= R is small)
-      for (uint32_t j = lane; j < n; j += 32) {
+      if (!a.boot_ids) {  // a new entry closer than every unexpanded one will be expanded next
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) best = min(best, __shfl_xor_sync(FULL, best, o));
+        if (best < key_clean(alt_key)) prefetch_row(a.g.adj + (size_t)key_id(best) * R, R, lane);
+      }
+      // rank the survivors among themselves (m is small)
+      for (uint32_t j = lane; j < m; j += 32) {
         const unsigned long long key = ckey[j];
-        if (key != kKeyMax) {
-          uint32_t r = 0;
-          for (uint32_t i = 0; i < n; ++i) r += ckey[i] < key;
-          cskey[r] = key;
-          csb[r] = cid[j];
-        }
+        uint32_t r = 0;
+        for (uint32_t i = 0; i < m; ++i) r += ckey[i] < key;
+        cskey[r] = key;
+        csb[r] = cid[j];
       }
       __syncwarp();
       // 3. shift worklist entries to their final places, highest chunk first (a move never goes
-      //    down, so an entry that is still unread is never overwritten)
+      //    down, so an entry that is still unread is never overwritten).  Entry i moves up by the
+      //    number of survivors whose rank is <= i.
       const uint32_t minb = csb[0];
       if (beam_n > minb) {
         const int top = (int)((beam_n - 1) >> 5), low = (int)(minb >> 5);
@@ -142,7 +197,18 @@ __global__ void __launch_bounds__(kSearchWarps * 32) beam_search_kernel(const Se
           uint32_t np = kInvalid;
           if (i < beam_n && i >= minb) {
             e = beam[i];
-            np = i + lower_bound_clean(cskey, m, key_clean(e));
+            uint32_t s = 0;
+            if (m <= 8) {
+              for (uint32_t r = 0; r < m; ++r) s += csb[r] <= i;
+            } else {
+              uint32_t lo = 0, hi = m;  // first r with csb[r] > i
+              while (lo < hi) {
+                const uint32_t mid = (lo + hi) >> 1;
+                if (csb[mid] <= i) lo = mid + 1; else hi = mid;
+              }
+              s = lo;
+            }
+            np = i + s;
           }
           __syncwarp();
           if (np < L) beam[np] = e;
@@ -169,7 +235,7 @@ __global__ void __launch_bounds__(kSearchWarps * 32) beam_search_kernel(const Se
           if (s < R && c0 + s < a.boot_n) v = a.boot_ids[c0 + s];
           const bool ok = v != kInvalid && v != self;
           const unsigned bal = __ballot_sync(FULL, ok);
-          if (ok) cid[n + __popc(bal & ((1u << lane) - 1u))] = v;
+          if (ok) cid[n + __popc(bal & lt_mask)] = v;
           n += __popc(bal);
         }
         __syncwarp();
@@ -178,7 +244,7 @@ __global__ void __launch_bounds__(kSearchWarps * 32) beam_search_kernel(const Se
     } else if (a.entry != kInvalid) {
       if (lane == 0) {
         cid[0] = a.entry;
-        hash[(a.entry * 2654435761u) >> (32 - a.hash_bits)] = a.entry;
+        visit_fresh(hash, a.hash_bits, tags16, a.entry);
       }
       __syncwarp();
       process(1);
@@ -204,24 +270,34 @@ __global__ void __launch_bounds__(kSearchWarps * 32) beam_search_kernel(const Se
         cursor = pos + 1;
         ++nvis;
         const uint32_t u = key_id(ek);
-        const uint32_t du = min(a.g.deg[u], R);
+        // Rows are padded with the invalid id, so the whole row is read without waiting for deg[u].
         const uint32_t* __restrict__ row = a.g.adj + (size_t)u * R;
-        uint32_t n = 0;
-        for (uint32_t sb = 0; sb < du; sb += 32) {
-          const uint32_t s = sb + lane;
-          bool fresh = false;
-          uint32_t v = kInvalid;
-          if (s < du) {
-            v = __ldg(row + s);
-            const uint32_t h = (v * 2654435761u) >> (32 - a.hash_bits);
-            if (hash[h] != v) {
-              hash[h] = v;
-              fresh = true;
-            }
+        uint32_t vrow[4];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) vrow[c] = (uint32_t)(c * 32 + lane) < R ? __ldg(row + c * 32 + lane) : kInvalid;
+        // While that load is in flight: the next unexpanded entry is the likeliest next expansion;
+        // pull its adjacency row towards L2 now (process() does the same for a closer new candidate).
+        alt_key = kKeyMax;
+        for (uint32_t cb = cursor & ~31u; cb < beam_n; cb += 32) {
+          const uint32_t i = cb + lane;
+          const bool un = i < beam_n && i >= cursor && !(beam[i] & kExpandedBit);
+          const unsigned bal = __ballot_sync(FULL, un);
+          if (bal) {
+            alt_key = beam[cb + __ffs(bal) - 1];
+            break;
           }
-          const unsigned bal = __ballot_sync(FULL, fresh);
-          if (fresh) cid[n + __popc(bal & ((1u << lane) - 1u))] = v;
-          n += __popc(bal);
+        }
+        if (alt_key != kKeyMax) prefetch_row(a.g.adj + (size_t)key_id(alt_key) * R, R, lane);
+        uint32_t n = 0;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          if ((uint32_t)(c * 32) < R) {
+            const uint32_t v = vrow[c];
+            const bool fresh = v != kInvalid && visit_fresh(hash, a.hash_bits, tags16, v);
+            const unsigned bal = __ballot_sync(FULL, fresh);
+            if (fresh) cid[n + __popc(bal & lt_mask)] = v;
+            n += __popc(bal);
+          }
         }
         __syncwarp();
         if (n) process(n);
