@@ -62,7 +62,7 @@ typedef struct {
   uint32_t k_repair;  /* repair candidates per deleted node; default min(50, L); <= 128 */
   uint32_t vmax;      /* expansion cap of update searches; default 2*L; <= 1024 */
   uint32_t mode;      /* grand_mode; default GRAND_MODE_VAMANA */
-  uint32_t hash_bits; /* log2 of the per-query visited cache; default 11; 8..13, and 4 << hash_bits >= padded row bytes */
+  uint32_t hash_bits; /* log2 of the per-query visited cache in 4-byte words; default 10; 8..13, and 4 << hash_bits >= padded row bytes */
   /* device allocator hooks (default cudaMalloc / cudaFree); lets a host runtime pool the memory */
   void* (*dev_alloc)(size_t bytes, void* user);
   void (*dev_free)(void* ptr, void* user);

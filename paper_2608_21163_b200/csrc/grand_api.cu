@@ -70,6 +70,8 @@ struct grand_index {
   unsigned long long* Ci = nullptr;
   uint32_t *Ci_n = nullptr, *in_cnt = nullptr, *pair_off = nullptr, *scan_tmp = nullptr;
   uint8_t* mean_row = nullptr;
+  uint32_t* search_ctrs = nullptr;  // ring of work counters, one per in-flight search launch
+  uint32_t ctr_next = 0;
   Buf req_tgt, req_key, seg_keys, dirty;              // grow-only, sized by the number of requests
   Buf t_indeg, t_off, t_fill, t_src;                  // reverse graph, allocated at the first delete
   Buf st_ids, st_vecs, st_out_ids, st_out_d;          // staging of the *_host entry points
@@ -191,8 +193,10 @@ int write_state_head(grand_index* idx, cudaStream_t s) {
   return GRAND_OK;
 }
 
-SearchArgs search_args(const grand_index* idx) {
+SearchArgs search_args(grand_index* idx, cudaStream_t s) {
   SearchArgs a{};
+  a.work_ctr = idx->search_ctrs + (idx->ctr_next++ & 63u);
+  cudaMemsetAsync(a.work_ctr, 0, 4, s);
   a.lay = idx->lay;
   a.g = view(idx);
   a.entry = idx->entry;
@@ -258,7 +262,7 @@ int grand_create_ex(uint32_t dim, uint32_t dtype, uint32_t metric, uint32_t R, u
   idx->k_repair = o->k_repair ? o->k_repair : (L < 50 ? L : 50);
   idx->vmax = o->vmax ? o->vmax : 2 * L;
   idx->mode = o->mode;
-  idx->hash_bits = o->hash_bits ? o->hash_bits : 11;
+  idx->hash_bits = o->hash_bits ? o->hash_bits : 10;
   idx->dev_alloc = o->dev_alloc ? o->dev_alloc : default_alloc;
   idx->dev_free = o->dev_free ? o->dev_free : default_free;
   idx->user = o->user;
@@ -295,6 +299,7 @@ int grand_create_ex(uint32_t dim, uint32_t dtype, uint32_t metric, uint32_t R, u
   A(alloc_dev(idx, &idx->pair_off, mb + 1, true));
   A(alloc_dev(idx, &idx->scan_tmp, (cap + 1) / 2048 + mb / 2048 + 8, true));
   A(alloc_dev(idx, &idx->mean_row, lay.row_bytes, true));
+  A(alloc_dev(idx, &idx->search_ctrs, 64, true));
   if (rc == GRAND_OK && cudaMemset(idx->adj, 0xFF, (size_t)cap * R * 4) != cudaSuccess) rc = GRAND_ERR_CUDA;
   if (rc == GRAND_OK && cudaMallocHost(&idx->h_state, sizeof(DevState)) != cudaSuccess) rc = GRAND_ERR_CUDA;
   if (rc == GRAND_OK) {
@@ -354,7 +359,7 @@ int grand_insert_batch(grand_index* idx, const uint32_t* ids, const void* vecs, 
   {
     // forward candidates: snapshot search (Alg. 5: visited list; Alg. 7: worklist) or bootstrap scan
     PhaseTimer pt(idx, s, PH_SEARCH);
-    SearchArgs a = search_args(idx);
+    SearchArgs a = search_args(idx, s);
     a.qids = ids;
     a.nq = n;
     a.L = idx->L;
@@ -485,7 +490,7 @@ int grand_delete_batch(grand_index* idx, const uint32_t* ids, uint64_t n, grand_
   } else {
     {
       PhaseTimer pt(idx, s, PH_SEARCH);
-      SearchArgs a = search_args(idx);
+      SearchArgs a = search_args(idx, s);
       a.qids = ids; a.nq = n; a.L = idx->L; a.vmax = idx->vmax;
       a.out_beam = idx->wk_keys; a.out_beam_n = idx->wk_n; a.beam_stride = idx->wk_stride;
       CK(launch_beam_search(a, s));
@@ -535,7 +540,7 @@ int grand_search(const grand_index* cidx, const void* queries, uint64_t nq, uint
   cudaStream_t s = (cudaStream_t)stream;
   {
     PhaseTimer pt(idx, s, PH_SEARCH);
-    SearchArgs a = search_args(idx);
+    SearchArgs a = search_args(idx, s);
     a.queries = queries; a.nq = nq; a.L = L; a.vmax = 2 * L; a.k = k;
     a.out_ids = out_ids; a.out_dists = out_dists;
     CK(launch_beam_search(a, s));

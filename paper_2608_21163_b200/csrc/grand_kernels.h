@@ -66,6 +66,7 @@ struct SearchArgs {
   const uint32_t* boot_ids;  // bootstrap: scan these ids (all batch-mates) instead of walking the graph
   uint32_t boot_n;
   uint32_t hash_bits;
+  uint32_t* work_ctr;  // zeroed by the caller before the launch; nullptr = static striding
   DevState* state;
 };
 cudaError_t launch_beam_search(const SearchArgs& a, cudaStream_t s);

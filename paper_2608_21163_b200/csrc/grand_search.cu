@@ -91,7 +91,20 @@ __global__ void __launch_bounds__(kSearchWarps * 32) beam_search_kernel(const Se
 
   const uint64_t wglobal = (uint64_t)blockIdx.x * kSearchWarps + warp;
   const uint64_t wtotal = (uint64_t)gridDim.x * kSearchWarps;
-  for (uint64_t qi = wglobal; qi < a.nq; qi += wtotal) {
+  uint64_t qi_static = wglobal;
+  for (;;) {
+    // queries are handed out through an atomic counter when the caller provides one (search times
+    // vary, and the last partial round would otherwise leave most warps idle)
+    uint64_t qi;
+    if (a.work_ctr) {
+      unsigned k = 0;
+      if (lane == 0) k = atomicAdd(a.work_ctr, 1u);
+      qi = __shfl_sync(FULL, k, 0);
+    } else {
+      qi = qi_static;
+      qi_static += wtotal;
+    }
+    if (qi >= a.nq) break;
     // ---- query into registers: lane t of each team holds chunks t, t+G, ...
     uint4 q[CPL];
     uint32_t self = kInvalid;
