@@ -139,6 +139,25 @@ int grand_import_graph(grand_index* idx, const uint32_t* adj_dev, const uint32_t
 int grand_reverse_graph(grand_index* idx, uint32_t* off_dev, uint32_t* src_dev, uint64_t* E_out_host,
                         grand_stream stream);
 
+/* The same CSR reverse graph for callers that cannot allocate device memory: hosts whose memory plan is
+ * frozen at start-up (a serving process that has handed all of HBM to its own pool, a sandboxed plug-in
+ * barred from the driver's allocator, a real-time loop that cannot take cudaMalloc's implicit
+ * synchronisation or its failure mid-request).  The paper has no counterpart for this call.  It needs no
+ * index handle: adj_dev (n_nodes x R, unused slots ignored through deg_dev) and deg_dev (n_nodes) are the
+ * caller's inputs, off_dev (n_nodes + 1) and src_dev (src_capacity entries; NULL = offsets only) the caller's
+ * outputs, E_out_host a HOST pointer to the edge count.  The result equals grand_reverse_graph on the same
+ * graph.  Its working memory is one fixed device array inside the library, GRAND_NOALLOC_SCRATCH_BYTES per GPU
+ * for the life of the process: n_nodes > GRAND_NOALLOC_MAX_NODES returns GRAND_ERR_CAPACITY, and so does a
+ * src_dev too small for the edges found.  All calls on a device share that array (everything that must be
+ * zero is cleared per call), so calls that overlap on the GPU race: serialise them.  The first call on each
+ * device resolves the array's address and should be made during set-up, before any stream capture.  No
+ * cudaMalloc, cudaFree or allocating library routine is called. */
+#define GRAND_NOALLOC_MAX_NODES (1u << 20)
+#define GRAND_NOALLOC_SCRATCH_BYTES ((GRAND_NOALLOC_MAX_NODES + GRAND_NOALLOC_MAX_NODES / 2048u + 64u) * 4u)
+int grand_reverse_graph_noalloc(const uint32_t* adj_dev, const uint32_t* deg_dev, uint64_t n_nodes, uint32_t R,
+                                uint32_t* off_dev, uint32_t* src_dev, uint64_t src_capacity, uint64_t* E_out_host,
+                                grand_stream stream);
+
 int grand_get_entry(const grand_index* idx, uint32_t* entry_out_host);
 int grand_set_entry(grand_index* idx, uint32_t entry);
 int grand_live_count(const grand_index* idx, uint64_t* n_out_host);

@@ -20,7 +20,7 @@ _TORCH_DTYPE = {U8: torch.uint8, I8: torch.int8, F32: torch.float32}
 EXPORTS = [
     "grand_create", "grand_create_ex", "grand_destroy", "grand_insert_batch", "grand_delete_batch", "grand_search",
     "grand_insert_batch_host", "grand_delete_batch_host", "grand_search_host", "grand_export_graph",
-    "grand_import_graph", "grand_reverse_graph", "grand_get_entry", "grand_set_entry", "grand_live_count",
+    "grand_import_graph", "grand_reverse_graph", "grand_reverse_graph_noalloc", "grand_get_entry", "grand_set_entry", "grand_live_count",
     "grand_row_bytes", "grand_get_stats", "grand_reset_stats", "grand_set_profiling", "grand_strerror",
     "grand_last_error",
 ]
@@ -78,6 +78,25 @@ def _stream():
 
 def _dp(t):
     return C.c_void_p(t.data_ptr()) if t is not None else C.c_void_p(0)
+
+
+NOALLOC_MAX_NODES = 1 << 20
+
+
+def reverse_graph_noalloc(adj, deg, off_out, src_out):
+    """CSR reverse graph of a caller-supplied adjacency array without any device allocation inside
+    the library (grand_reverse_graph_noalloc).  For callers whose memory plan is frozen: adj [n x R]
+    and deg [n] are device inputs, off_out [n + 1] and src_out (or None) device outputs that the
+    caller allocated beforehand.  Calls on one device share a fixed scratch array inside the
+    library and must not overlap.  Returns the number of edges."""
+    lib = load()
+    n, R = adj.shape
+    E = C.c_uint64()
+    rc = lib.grand_reverse_graph_noalloc(_dp(adj), _dp(deg), C.c_uint64(n), C.c_uint32(R), _dp(off_out), _dp(src_out),
+                                         C.c_uint64(src_out.numel() if src_out is not None else 0), C.byref(E), _stream())
+    if rc != 0:
+        raise GrandError(rc, lib.grand_strerror(rc).decode())
+    return E.value
 
 
 class GrandIndex:

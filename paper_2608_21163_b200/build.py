@@ -9,7 +9,7 @@ from concurrent.futures import ThreadPoolExecutor
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libgrand_b200.so")
-SOURCES = ["grand_api.cu", "grand_search.cu", "grand_prune.cu", "grand_rebuild.cu", "grand_group.cu", "grand_delete.cu"]
+SOURCES = ["grand_api.cu", "grand_search.cu", "grand_prune.cu", "grand_rebuild.cu", "grand_group.cu", "grand_delete.cu", "grand_static.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
 
