@@ -63,6 +63,9 @@ typedef struct {
   uint32_t vmax;      /* expansion cap of update searches; default 2*L; <= 1024 */
   uint32_t mode;      /* grand_mode; default GRAND_MODE_VAMANA */
   uint32_t hash_bits; /* log2 of the per-query visited cache in 4-byte words; default 10; 8..13, and 4 << hash_bits >= padded row bytes */
+  uint32_t full_transpose; /* 1: every delete batch builds the whole reverse graph; default 0: only the rows of the
+                              batch's nodes (the only rows the repair reads; identical result) */
+  uint32_t reserved_;
   /* device allocator hooks (default cudaMalloc / cudaFree); lets a host runtime pool the memory */
   void* (*dev_alloc)(size_t bytes, void* user);
   void (*dev_free)(void* ptr, void* user);

@@ -46,7 +46,7 @@ struct Buf {
 
 struct grand_index {
   Layout lay;
-  uint32_t R, L, P, c, k_repair, vmax, mode, hash_bits;
+  uint32_t R, L, P, c, k_repair, vmax, mode, hash_bits, full_transpose;
   float alpha;
   long long A_fix;
   uint64_t cap, max_batch;
@@ -263,6 +263,7 @@ int grand_create_ex(uint32_t dim, uint32_t dtype, uint32_t metric, uint32_t R, u
   idx->vmax = o->vmax ? o->vmax : 2 * L;
   idx->mode = o->mode;
   idx->hash_bits = o->hash_bits ? o->hash_bits : 10;
+  idx->full_transpose = o->full_transpose;
   idx->dev_alloc = o->dev_alloc ? o->dev_alloc : default_alloc;
   idx->dev_free = o->dev_free ? o->dev_free : default_free;
   idx->user = o->user;
@@ -427,7 +428,7 @@ int grand_insert_batch(grand_index* idx, const uint32_t* ids, const void* vecs, 
   return GRAND_OK;
 }
 
-static int build_reverse(grand_index* idx, bool sort_rows, cudaStream_t s) {
+static int build_reverse(grand_index* idx, bool sort_rows, const uint32_t* heads, cudaStream_t s) {
   int rc;
   const uint64_t cap = idx->cap;
   if ((rc = ensure(idx, idx->t_indeg, (cap + 1) * 4, s))) return rc;
@@ -437,7 +438,7 @@ static int build_reverse(grand_index* idx, bool sort_rows, cudaStream_t s) {
   TransposeArgs t{};
   t.g = view(idx);
   t.indeg = (uint32_t*)idx->t_indeg.p; t.off = (uint32_t*)idx->t_off.p; t.fillc = (uint32_t*)idx->t_fill.p;
-  t.src = (uint32_t*)idx->t_src.p; t.scan_tmp = idx->scan_tmp; t.sort_rows = sort_rows;
+  t.src = (uint32_t*)idx->t_src.p; t.scan_tmp = idx->scan_tmp; t.sort_rows = sort_rows; t.heads = heads;
   CK(launch_transpose(t, s));
   return GRAND_OK;
 }
@@ -465,7 +466,8 @@ int grand_delete_batch(grand_index* idx, const uint32_t* ids, uint64_t n, grand_
   {
     // reverse graph of the snapshot: exact in-neighbours, rebuilt per batch and not kept
     PhaseTimer pt(idx, s, PH_TRANSPOSE);
-    if ((rc = build_reverse(idx, false, s))) return rc;
+    // only the in-neighbour rows of the batch are read below, so only those are materialised
+    if ((rc = build_reverse(idx, false, idx->full_transpose ? nullptr : idx->mark, s))) return rc;
     d.off = (uint32_t*)idx->t_off.p; d.src = (uint32_t*)idx->t_src.p;
     CK(launch_delete_prepare(d, s));
   }
@@ -626,7 +628,7 @@ int grand_reverse_graph(grand_index* idx, uint32_t* off, uint32_t* src, uint64_t
   if (!idx) return GRAND_ERR_INVALID_ARG;
   cudaStream_t s = (cudaStream_t)stream;
   int rc;
-  if ((rc = build_reverse(idx, true, s))) return rc;
+  if ((rc = build_reverse(idx, true, nullptr, s))) return rc;
   uint32_t E = 0;
   CK(cudaMemcpyAsync(&E, (uint32_t*)idx->t_off.p + idx->cap, 4, cudaMemcpyDeviceToHost, s));
   CK(cudaStreamSynchronize(s));

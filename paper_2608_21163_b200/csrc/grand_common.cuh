@@ -171,6 +171,19 @@ __device__ __forceinline__ uint32_t lower_bound_clean(const unsigned long long* 
   return lo;
 }
 
+// Append `value` to list[*counter ...] for every lane with `need`: one atomic per warp instead of one
+// per lane (all 32 lanes must call this together).  Counters hit by every dirty node or request would
+// otherwise serialise on a single address.
+__device__ __forceinline__ void warp_append(uint32_t* list, uint32_t* counter, bool need, uint32_t value) {
+  const unsigned bal = __ballot_sync(0xFFFFFFFFu, need);
+  if (!bal) return;
+  const int lane = threadIdx.x & 31, leader = __ffs(bal) - 1;
+  uint32_t base = 0;
+  if (lane == leader) base = atomicAdd(counter, (uint32_t)__popc(bal));
+  base = __shfl_sync(0xFFFFFFFFu, base, leader);
+  if (need) list[base + __popc(bal & ((1u << lane) - 1u))] = value;
+}
+
 __device__ __forceinline__ bool bit_test(const uint32_t* bm, uint32_t v) { return (bm[v >> 5] >> (v & 31)) & 1u; }
 
 // alpha test of RobustPrune (Alg. 4): alpha * dist(p*,p') <= D_p[p'].

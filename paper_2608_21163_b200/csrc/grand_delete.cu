@@ -10,9 +10,6 @@ constexpr int kPickWarps = 4;
 constexpr uint32_t kMaxKRepair = 128;
 constexpr uint32_t kMaxC = 8;
 
-__device__ __forceinline__ void touch_dirty2(uint32_t* flag, uint32_t* dirty, DevState* st, uint32_t u) {
-  if (atomicExch(&flag[u], 1u) == 0u) dirty[atomicAdd(&st->ndirty, 1u)] = u;
-}
 
 // in_cnt[i] = in-degree of p_i in the reverse graph (0 for an id that fails validation), then the
 // prefix over the batch and the total number of (deleted node, in-neighbour) pairs.
@@ -111,26 +108,33 @@ __global__ void __launch_bounds__(kPickWarps * 32) delete_picks_kernel(const Del
       if (lane < c) a.req_tgt[rbase + lane] = kInvalid;
       continue;
     }
-    if (is_in && lane == 0) touch_dirty2(a.flag, a.dirty, a.state, x);  // dirty even without a candidate
     uint4 xr[CPL];
     load_row<G, CPL>(a.g.store + (size_t)x * row_bytes, nchunk, t, xr);
     const uint32_t nc = a.Ci_n[i];
-    for (uint32_t jb = 0; jb < nc; jb += NT) {
-      const uint32_t j = jb + team;
-      uint32_t y = kInvalid;
-      if (j < nc) y = key_id(a.Ci[i * a.k_repair + j]);
-      const bool go = y != kInvalid && y != x;
-      uint4 v[CPL];
-      if (go) {
-        load_row<G, CPL>(a.g.store + (size_t)y * row_bytes, nchunk, t, v);
-      } else {
+    constexpr int U = CPL == 1 ? 4 : (CPL == 2 ? 2 : 1);  // candidate rows in flight per team
+    for (uint32_t jb = 0; jb < nc; jb += NT * U) {
+      uint4 v[U][CPL];
+      uint32_t yv[U];
 #pragma unroll
-        for (int cc = 0; cc < CPL; ++cc) v[cc] = make_uint4(0, 0, 0, 0);
+      for (int uu = 0; uu < U; ++uu) {
+        const uint32_t j = jb + uu * NT + team;
+        yv[uu] = j < nc ? key_id(a.Ci[i * a.k_repair + j]) : kInvalid;
+        if (yv[uu] != kInvalid && yv[uu] != x) {
+          load_row<G, CPL>(a.g.store + (size_t)yv[uu] * row_bytes, nchunk, t, v[uu]);
+        } else {
+#pragma unroll
+          for (int cc = 0; cc < CPL; ++cc) v[uu][cc] = make_uint4(0, 0, 0, 0);
+        }
       }
-      const Dist d = team_dist_regs<T, kMetricL2, G, CPL>(xr, v);
-      if (t == 0 && j < nc) {
-        keys[j] = go ? make_key(d, y) : kKeyMax;
-        npair += go;
+#pragma unroll
+      for (int uu = 0; uu < U; ++uu) {
+        const uint32_t j = jb + uu * NT + team;
+        const Dist d = team_dist_regs<T, kMetricL2, G, CPL>(xr, v[uu]);
+        if (t == 0 && j < nc) {
+          const bool go = yv[uu] != x;
+          keys[j] = go ? make_key(d, yv[uu]) : kKeyMax;
+          npair += go;
+        }
       }
     }
     __syncwarp();
@@ -159,12 +163,38 @@ __global__ void __launch_bounds__(kPickWarps * 32) delete_picks_kernel(const Del
   }
   if (npair) atomicAdd(&a.state->counters[CTR_PAIR], npair);
 }
+// Every surviving in-neighbour of a deleted node is dirty even if it receives no candidate.
+__global__ void delete_touch_kernel(const DeleteArgs a, const uint64_t total_in) {
+  const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  for (uint64_t b = blockIdx.x * (uint64_t)blockDim.x + (threadIdx.x & ~31u); b < total_in; b += stride) {
+    const uint64_t pair = b + (threadIdx.x & 31);
+    bool first = false;
+    uint32_t z = kInvalid;
+    if (pair < total_in) {
+      uint64_t lo = 0, hi = a.n;
+      while (hi - lo > 1) {
+        const uint64_t mid = (lo + hi) >> 1;
+        if (a.pair_off[mid] <= pair) lo = mid; else hi = mid;
+      }
+      z = a.src[a.off[a.ids[lo]] + (uint32_t)(pair - a.pair_off[lo])];
+      first = !bit_test(a.delmap, z) && atomicExch(&a.flag[z], 1u) == 0u;
+    }
+    warp_append(a.dirty, &a.state->ndirty, first, z);
+  }
+}
+
 template <typename T, int METRIC, int G, int CPL>
 static cudaError_t launch_delete_picks_t(const DeleteArgs& a, uint64_t total_in, cudaStream_t s) {
   const uint64_t total = total_in + a.n * a.g.R;
   if (total == 0) return cudaSuccess;
   uint64_t blocks = (total + kPickWarps - 1) / kPickWarps;
   if (blocks > 148u * 16u) blocks = 148u * 16u;
+  if (total_in) {
+    uint64_t tb = (total_in + 255) / 256;
+    if (tb > 148u * 32u) tb = 148u * 32u;
+    delete_touch_kernel<<<(unsigned)tb, 256, 0, s>>>(a, total_in);
+    count_launches(1);
+  }
   delete_picks_kernel<T, METRIC, G, CPL><<<(unsigned)blocks, kPickWarps * 32, 0, s>>>(a, total_in);
   count_launches(1);
   return cudaGetLastError();
@@ -184,7 +214,7 @@ __global__ void fixed_delete_mark_kernel(const FixedDeleteArgs a, const uint64_t
       if (a.pair_off[mid] <= pair) lo = mid; else hi = mid;
     }
     const uint32_t u = a.src[a.off[a.ids[lo]] + (uint32_t)(pair - a.pair_off[lo])];
-    if (!bit_test(a.delmap, u)) touch_dirty2(a.flag, a.dirty, a.state, u);
+    if (!bit_test(a.delmap, u) && atomicExch(&a.flag[u], 1u) == 0u) a.dirty[atomicAdd(&a.state->ndirty, 1u)] = u;
   }
 }
 __global__ void __launch_bounds__(128) fixed_delete_rewire_kernel(const FixedDeleteArgs a) {

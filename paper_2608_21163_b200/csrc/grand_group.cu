@@ -13,28 +13,46 @@ static inline unsigned grid_for(uint64_t n, int threads = kThreads, unsigned max
   return (unsigned)(b > maxb ? maxb : b);
 }
 
-__device__ __forceinline__ void touch_dirty(uint32_t* flag, uint32_t* dirty, DevState* st, uint32_t u) {
-  if (atomicExch(&flag[u], 1u) == 0u) dirty[atomicAdd(&st->ndirty, 1u)] = u;
-}
 
 // ---- request grouping: count per target (first touch appends to the dirty list), allocate one
 // segment per dirty target from a global cursor, scatter keys into the segments.
 __global__ void group_count_kernel(const GroupArgs a) {
   unsigned long long nv = 0;
-  for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < a.nreq; i += (uint64_t)gridDim.x * blockDim.x) {
-    const uint32_t tg = a.req_tgt[i];
-    if (tg == kInvalid) continue;
-    atomicAdd(&a.cnt[tg], 1u);
-    touch_dirty(a.flag, a.dirty, a.state, tg);
-    ++nv;
+  const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  // warp-uniform trip count: every lane takes part in the aggregated append
+  for (uint64_t b = blockIdx.x * (uint64_t)blockDim.x + (threadIdx.x & ~31u); b < a.nreq; b += stride) {
+    const uint64_t i = b + (threadIdx.x & 31);
+    const uint32_t tg = i < a.nreq ? a.req_tgt[i] : kInvalid;
+    bool first = false;
+    if (tg != kInvalid) {
+      ++nv;
+      // first request of this target in the batch, and not already listed by a repair touch
+      first = atomicAdd(&a.cnt[tg], 1u) == 0u && atomicExch(&a.flag[tg], 1u) == 0u;
+    }
+    warp_append(a.dirty, &a.state->ndirty, first, tg);
   }
-  if (nv) atomicAdd(&a.state->counters[CTR_REQ], nv);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) nv += __shfl_xor_sync(0xFFFFFFFFu, nv, o);
+  if ((threadIdx.x & 31) == 0 && nv) atomicAdd(&a.state->counters[CTR_REQ], nv);
 }
 __global__ void group_alloc_kernel(const GroupArgs a) {
   const uint32_t nd = a.state->ndirty;
-  for (uint32_t k = blockIdx.x * blockDim.x + threadIdx.x; k < nd; k += gridDim.x * blockDim.x) {
-    const uint32_t u = a.dirty[k];
-    a.start[u] = atomicAdd(&a.state->cursor, a.cnt[u]);
+  const int lane = threadIdx.x & 31;
+  // one cursor bump per warp: segment sizes are prefix-summed across the lanes
+  for (uint32_t b = blockIdx.x * blockDim.x + (threadIdx.x & ~31u); b < nd; b += gridDim.x * blockDim.x) {
+    const uint32_t k = b + lane;
+    const uint32_t u = k < nd ? a.dirty[k] : 0u;
+    const uint32_t c = k < nd ? a.cnt[u] : 0u;
+    uint32_t inc = c;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+      if (lane >= o) inc += y;
+    }
+    uint32_t base = 0;
+    if (lane == 31) base = atomicAdd(&a.state->cursor, inc);
+    base = __shfl_sync(0xFFFFFFFFu, base, 31);
+    if (k < nd) a.start[u] = base + inc - c;
   }
 }
 __global__ void group_scatter_kernel(const GroupArgs a) {
@@ -134,23 +152,24 @@ cudaError_t launch_exclusive_scan(const uint32_t* in, uint32_t* out, uint64_t n,
 }
 
 // ---- reverse graph
-__global__ void transpose_hist_kernel(const GraphView g, uint32_t* indeg) {
+// `heads` (optional bitmap): only edges whose head is marked are counted / scattered, i.e. only the
+// in-neighbour rows of the marked nodes are materialised (the delete path reads no other row).
+__global__ void transpose_hist_kernel(const GraphView g, uint32_t* indeg, const uint32_t* heads) {
   const uint64_t total = g.cap * g.R;
   for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < total; i += (uint64_t)gridDim.x * blockDim.x) {
     const uint64_t v = i / g.R;
-    const uint32_t s = (uint32_t)(i - v * g.R);
-    if (s < g.deg[v]) atomicAdd(&indeg[g.adj[i]], 1u);
+    if ((uint32_t)(i - v * g.R) >= g.deg[v]) continue;
+    const uint32_t z = g.adj[i];
+    if (!heads || bit_test(heads, z)) atomicAdd(&indeg[z], 1u);
   }
 }
-__global__ void transpose_scatter_kernel(const GraphView g, const uint32_t* off, uint32_t* fillc, uint32_t* src) {
+__global__ void transpose_scatter_kernel(const GraphView g, const uint32_t* off, uint32_t* fillc, uint32_t* src, const uint32_t* heads) {
   const uint64_t total = g.cap * g.R;
   for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < total; i += (uint64_t)gridDim.x * blockDim.x) {
     const uint64_t v = i / g.R;
-    const uint32_t s = (uint32_t)(i - v * g.R);
-    if (s < g.deg[v]) {
-      const uint32_t z = g.adj[i];
-      src[off[z] + atomicAdd(&fillc[z], 1u)] = (uint32_t)v;
-    }
+    if ((uint32_t)(i - v * g.R) >= g.deg[v]) continue;
+    const uint32_t z = g.adj[i];
+    if (!heads || bit_test(heads, z)) src[off[z] + atomicAdd(&fillc[z], 1u)] = (uint32_t)v;
   }
 }
 // ascending rows: shared-memory sort for short rows, in place in global memory for long ones
@@ -175,13 +194,13 @@ __global__ void __launch_bounds__(128) transpose_sort_rows_kernel(uint64_t cap, 
 cudaError_t launch_transpose(const TransposeArgs& a, cudaStream_t s) {
   const uint64_t cap = a.g.cap;
   cudaMemsetAsync(a.indeg, 0, (cap + 1) * 4, s);
-  transpose_hist_kernel<<<grid_for(cap * a.g.R), kThreads, 0, s>>>(a.g, a.indeg);
+  transpose_hist_kernel<<<grid_for(cap * a.g.R), kThreads, 0, s>>>(a.g, a.indeg, a.heads);
   count_launches(1);
   cudaError_t e = launch_exclusive_scan(a.indeg, a.off, cap + 1, a.scan_tmp, s);
   if (e != cudaSuccess) return e;
   if (a.src) {
     cudaMemsetAsync(a.fillc, 0, cap * 4, s);
-    transpose_scatter_kernel<<<grid_for(cap * a.g.R), kThreads, 0, s>>>(a.g, a.off, a.fillc, a.src);
+    transpose_scatter_kernel<<<grid_for(cap * a.g.R), kThreads, 0, s>>>(a.g, a.off, a.fillc, a.src, a.heads);
     count_launches(a.sort_rows ? 2 : 1);
     if (a.sort_rows) transpose_sort_rows_kernel<<<(unsigned)(cap < 148u * 16u ? cap : 148u * 16u), 128, 0, s>>>(cap, a.off, a.src);
   }

@@ -141,6 +141,7 @@ struct TransposeArgs {
   uint32_t* src;    // >= total edges (nullable: offsets only)
   uint32_t* scan_tmp;  // >= ceil((cap+1)/4096)+1
   bool sort_rows;
+  const uint32_t* heads;  // optional bitmap: build only the rows of these nodes
 };
 cudaError_t launch_transpose(const TransposeArgs& a, cudaStream_t s);
 cudaError_t launch_exclusive_scan(const uint32_t* in, uint32_t* out, uint64_t n, uint32_t* tmp, cudaStream_t s);

@@ -23,7 +23,7 @@ namespace grand {
 
 constexpr int kRebuildWarps = 4;
 constexpr uint32_t kSegSmem = 128;       // request segments up to this length are sorted in shared memory
-constexpr uint32_t kMaxUncertain = 256;  // capacity of the uncertain-position list (aliases the segment buffer)
+constexpr uint32_t kWorkChunk = 1;       // dirty nodes taken per work-counter bump
 
 static inline uint32_t even_up_h(uint32_t x) { return (x + 1u) & ~1u; }
 static size_t rebuild_smem_per_warp(uint32_t R, uint32_t P) {
@@ -49,7 +49,8 @@ __global__ void __launch_bounds__(kRebuildWarps * 32) rebuild_kernel(const Rebui
   uint32_t* keep = reinterpret_cast<uint32_t*>(cand + NM);
   uint32_t* out_idx = keep + Rp;
   uint32_t* prune = out_idx + Rp;  // NM rows x W words: bit j of row i = "c_i prunes c_j"
-  uint32_t* upos = reinterpret_cast<uint32_t*>(seg_s);  // positions of uncertain candidates (segment buffer is free by then)
+  uint32_t* upos = reinterpret_cast<uint32_t*>(scratch);  // positions of uncertain candidates (2P entries; scratch is free by then)
+  unsigned long long* cs = cand;  // C in key order: cand itself, or the segment buffer after a rank merge
   const AlphaParam ap{a.A_fix, a.alpha};
   const uint32_t row_bytes = a.lay.row_bytes, nchunk = a.lay.nchunk;
   const uint8_t* __restrict__ store = a.g.store;
@@ -63,10 +64,10 @@ __global__ void __launch_bounds__(kRebuildWarps * 32) rebuild_kernel(const Rebui
     uint4 ri[CPL];
     if (act) {
       if (j != jprev) {
-        load_row<G, CPL>(store + (size_t)key_id(cand[j]) * row_bytes, nchunk, t, rj);
+        load_row<G, CPL>(store + (size_t)key_id(cs[j]) * row_bytes, nchunk, t, rj);
         jprev = j;
       }
-      load_row<G, CPL>(store + (size_t)key_id(cand[i]) * row_bytes, nchunk, t, ri);
+      load_row<G, CPL>(store + (size_t)key_id(cs[i]) * row_bytes, nchunk, t, ri);
     } else {
 #pragma unroll
       for (int c = 0; c < CPL; ++c) ri[c] = make_uint4(0, 0, 0, 0);
@@ -74,15 +75,20 @@ __global__ void __launch_bounds__(kRebuildWarps * 32) rebuild_kernel(const Rebui
     const Dist d = team_dist_regs<T, kMetricL2, G, CPL>(ri, rj);
     if (act && t == 0) {
       ++npair;
-      if (alpha_test(ap, d, key_dist<Dist>(cand[j]))) atomicOr(&prune[i * W + (j >> 5)], 1u << (j & 31));
+      if (alpha_test(ap, d, key_dist<Dist>(cs[j]))) atomicOr(&prune[i * W + (j >> 5)], 1u << (j & 31));
     }
   };
 
+  uint32_t k_next = 0, k_end = 0;
   for (;;) {
-    uint32_t k = 0;
-    if (lane == 0) k = atomicAdd(&a.state->work, 1u);
-    k = __shfl_sync(FULL, k, 0);
-    if (k >= ndirty) break;
+    if (k_next == k_end) {  // fetch a few nodes per atomic: one counter serves every warp of the grid
+      uint32_t kb = 0;
+      if (lane == 0) kb = atomicAdd(&a.state->work, kWorkChunk);
+      k_next = __shfl_sync(FULL, kb, 0);
+      k_end = min(k_next + kWorkChunk, ndirty);
+      if (k_next >= ndirty) break;
+    }
+    const uint32_t k = k_next++;
     const uint32_t u = a.dirty[k];
     const uint32_t cntu = a.cnt[u];
     // ---- scratch_u: sort the request segment by (dist, id), keep the first P distinct entries
@@ -129,19 +135,18 @@ __global__ void __launch_bounds__(kRebuildWarps * 32) rebuild_kernel(const Rebui
     __syncwarp();
     // ---- fresh = scratch \ keep \ {u}, stable, placed after the keep slots of cand (tagged uncertain)
     uint32_t nf = 0;
-    for (uint32_t jb = 0; jb < ns; jb += 32) {
-      const uint32_t j = jb + lane;
-      bool ok = false;
-      unsigned long long kk = 0;
-      if (j < ns) {
-        kk = scratch[j];
+    {
+      uint32_t kreg[4];  // the kept ids, spread over the lanes (R <= 128); the invalid id never matches
+#pragma unroll
+      for (int c = 0; c < 4; ++c) kreg[c] = (uint32_t)(c * 32 + lane) < nk ? keep[c * 32 + lane] : kInvalid;
+      for (uint32_t j = 0; j < ns; ++j) {
+        const unsigned long long kk = scratch[j];
         const uint32_t id = key_id(kk);
-        ok = id != u;
-        for (uint32_t x = 0; ok && x < nk; ++x) ok = keep[x] != id;
+        const bool hit = kreg[0] == id || kreg[1] == id || kreg[2] == id || kreg[3] == id;
+        if (__any_sync(FULL, hit) || id == u) continue;
+        if (lane == 0) cand[nk + nf] = kk | kExpandedBit;
+        ++nf;
       }
-      const unsigned bal = __ballot_sync(FULL, ok);
-      if (ok) cand[nk + nf + __popc(bal & lt_mask)] = kk | kExpandedBit;
-      nf += __popc(bal);
     }
     __syncwarp();
     const uint32_t nC = nk + nf;
@@ -174,19 +179,58 @@ __global__ void __launch_bounds__(kRebuildWarps * 32) rebuild_kernel(const Rebui
         }
       }
       __syncwarp();
-      bitonic_sort_clean(cand, nC, (uint32_t)lane, 32u, wsync);
+      // ---- C in key order.  The kept prefix is prune output and therefore already ascending: sort
+      //      only the uncertain tail and merge the two runs by rank (checked, with a full sort as the
+      //      fallback); long candidate lists take the full sort as well.
+      uint32_t kpe = kp;
+      bool merged = false;
+      if (nC <= kSegSmem && kp > 0) {
+        bool asc = true;
+        for (uint32_t ib = 0; ib + 1 < kp; ib += 32) {
+          const uint32_t i = ib + lane;
+          const bool bad = i + 1 < kp && !(cand[i] < cand[i + 1]);
+          if (__any_sync(FULL, bad)) asc = false;
+        }
+        if (asc) {
+          const uint32_t nt = nC - kp;
+          bitonic_sort_clean(cand + kp, nt, (uint32_t)lane, 32u, wsync);
+          for (uint32_t i = lane; i < kp; i += 32) {
+            const unsigned long long e = cand[i];
+            uint32_t sft = 0;
+            if (nt <= 8) {
+              for (uint32_t r = 0; r < nt; ++r) sft += key_clean(cand[kp + r]) < e;
+            } else {
+              sft = lower_bound_clean(cand + kp, nt, e);
+            }
+            seg_s[i + sft] = e;
+          }
+          for (uint32_t r = lane; r < nt; r += 32) {
+            const unsigned long long tk = cand[kp + r];
+            seg_s[r + lower_bound_clean(cand, kp, key_clean(tk))] = tk;
+          }
+          __syncwarp();
+          cs = seg_s;
+          merged = true;
+        } else {
+          kpe = 0;  // not the expected order: trust nothing, test the whole triangle
+        }
+      }
+      if (!merged) {
+        bitonic_sort_clean(cand, nC, (uint32_t)lane, 32u, wsync);
+        cs = cand;
+      }
       for (uint32_t w = lane; w < nC * W; w += 32) prune[w] = 0u;
       // ---- prune tests in parallel: pairs with an uncertain member, or the whole upper triangle
-      const uint32_t nu = nC - kp;
+      const uint32_t nu = nC - kpe;
       uint32_t jprev = kInvalid;
       uint4 rj[CPL];
 #pragma unroll
       for (int c = 0; c < CPL; ++c) rj[c] = make_uint4(0, 0, 0, 0);
-      if (nu <= kMaxUncertain && 2 * nu + 1 < nC) {
+      if (nu <= 2 * P && 2 * nu + 1 < nC) {
         uint32_t nfound = 0;
         for (uint32_t jb = 0; jb < nC; jb += 32) {
           const uint32_t j = jb + lane;
-          const bool un = j < nC && (cand[j] & kExpandedBit);
+          const bool un = j < nC && (cs[j] & kExpandedBit);
           const unsigned bal = __ballot_sync(FULL, un);
           if (un) upos[nfound + __popc(bal & lt_mask)] = j;
           nfound += __popc(bal);
@@ -200,7 +244,7 @@ __global__ void __launch_bounds__(kRebuildWarps * 32) rebuild_kernel(const Rebui
           if (act) {
             const uint32_t f = upos[e / nC], x = e % nC;
             // skip self; a pair of two uncertain members is taken once, from its larger member
-            act = f != x && !(x > f && (cand[x] & kExpandedBit));
+            act = f != x && !(x > f && (cs[x] & kExpandedBit));
             i = min(f, x);
             j = max(f, x);
           }
@@ -239,7 +283,7 @@ __global__ void __launch_bounds__(kRebuildWarps * 32) rebuild_kernel(const Rebui
         if ((uint32_t)lane < W) valid &= ~prune[i * W + lane];
       }
       __syncwarp();
-      for (uint32_t s = lane; s < R; s += 32) row[s] = s < cnt ? key_id(cand[out_idx[s]]) : kInvalid;
+      for (uint32_t s = lane; s < R; s += 32) row[s] = s < cnt ? key_id(cs[out_idx[s]]) : kInvalid;
       if (lane == 0) {
         a.g.deg[u] = cnt;
         a.g.rowpfx[u] = (uint8_t)cnt;
