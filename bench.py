@@ -93,11 +93,11 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------ oracle arm
-def oracle_run(steps, warmup, seed=0):
+def oracle_run(steps, warmup, seed=0, workload=WORKLOAD):
     """The CPU oracle on a bounded shrink of the stream: build 10,000 points (untimed), then steps of
     insert 250 + delete 250 + search 250.  Returns the JSON-ready dict of the reference arm."""
     from oracle import grand_oracle as go
-    cfg = dict(synth.CONFIGS[WORKLOAD])
+    cfg = dict(synth.CONFIGS[workload])
     per = 250
     cfg.update(n=10_000 + (steps + warmup) * per, build=10_000, first_batch=1_000, max_build_batch=1_000,
                ins=per, dele=per, nq=per, rounds=steps + warmup)
@@ -128,7 +128,7 @@ def oracle_run(steps, warmup, seed=0):
             t_upd += (t1 - t0) + (t3 - t2)
             t_search += t4 - t3
     value = 2 * per * steps / t_upd
-    sample = (f"{WORKLOAD} shrunk: index built on 10,000 points (untimed, {t_build:.1f} s), then {steps} steps of "
+    sample = (f"{workload} shrunk: index built on 10,000 points (untimed, {t_build:.1f} s), then {steps} steps of "
               f"insert {per} + delete {per} + search {per} (k=10, L={cfg['L']})")
     return {"value": value, "unit": UNIT, "cores": o.nthreads, "kind": "oracle", "sample": sample,
             "search_qps": per * steps / t_search, "ms_per_step": 1e3 * (t_upd + t_search) / steps}
@@ -143,6 +143,8 @@ def main():
     ap.add_argument("--scale", type=float, default=1.0, help="shrink the workload (profiling captures, quick checks)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true")
+    ap.add_argument("--workload", default=WORKLOAD, choices=sorted(synth.CONFIGS), help="default: the bench workload; the other "
+                    "configs are exploration runs (their lines carry their own workload name)")
     ap.add_argument("--hash-bits", type=int, default=0, help="log2 size of the per-query visited cache (0 = library default)")
     ap.add_argument("--search-only", type=int, default=0, help="after the build run this many search launches and exit")
     args = ap.parse_args()
@@ -154,11 +156,11 @@ def main():
     if args.impl == "reference":
         if rank != 0:
             return 0
-        r = oracle_run(K, W)
+        r = oracle_run(K, W, workload=args.workload)
         line = {"impl": "reference", "metric": METRIC, "value": r["value"], "unit": UNIT, "n_gpus": args.gpus, "steps": K,
                 "warmup": W, "ms_per_step": r["ms_per_step"], "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "int32", "data": "synthetic",
-                "config": {"workload": WORKLOAD, "sample": r["sample"]},
+                "config": {"workload": args.workload, "sample": r["sample"]},
                 "cpu_baseline": {k: r[k] for k in ("value", "unit", "cores", "kind", "sample")},
                 "e2e": {"value": r["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
                 "search_qps": r["search_qps"], "gpu_launches": 0}
@@ -177,12 +179,15 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
     torch.backends.cuda.matmul.allow_tf32 = False
 
-    cfg = dict(synth.CONFIGS[WORKLOAD])
+    cfg = dict(synth.CONFIGS[args.workload])
+    is_f32 = cfg["dtype"] == synth.F32
+    dist_dtype = torch.float32 if is_f32 else torch.int32
     if args.scale != 1.0:
         cfg = synth.scaled(cfg, args.scale)
     total_steps = W + 2 * K          # device-resident steps, then K end-to-end steps
     cfg["rounds"] = total_steps
     cfg["n"] = cfg["build"] + total_steps * cfg["ins"]
+    cfg["reuse_ids"] = False      # fresh ids every step, whatever the config's own id policy
     seed = rank                       # replicas draw independent streams
     wl = synth.Workload(cfg, seed)
     st = synth.StreamState(wl)
@@ -213,7 +218,7 @@ def main():
 
     if args.search_only:
         out_i = torch.empty((cfg["nq"], 10), dtype=torch.uint32, device=dev)
-        out_d = torch.empty((cfg["nq"], 10), dtype=torch.int32, device=dev)
+        out_d = torch.empty((cfg["nq"], 10), dtype=dist_dtype, device=dev)
         for _ in range(args.search_only):
             g.search(queries, 10, cfg["L"], out_i, out_d)
         torch.cuda.synchronize()
@@ -222,7 +227,7 @@ def main():
 
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)   # > L2 (126 MB)
     out_i = torch.empty((cfg["nq"], 10), dtype=torch.uint32, device=dev)
-    out_d = torch.empty((cfg["nq"], 10), dtype=torch.int32, device=dev)
+    out_d = torch.empty((cfg["nq"], 10), dtype=dist_dtype, device=dev)
     ev = lambda: torch.cuda.Event(enable_timing=True)
 
     def one_step(timed):
@@ -270,7 +275,7 @@ def main():
     pin = lambda a: torch.from_numpy(a).pin_memory()
     q_pin = pin(queries_host)
     oi_pin = torch.empty((cfg["nq"], 10), dtype=torch.uint32).pin_memory()
-    od_pin = torch.empty((cfg["nq"], 10), dtype=torch.int32).pin_memory()
+    od_pin = torch.empty((cfg["nq"], 10), dtype=dist_dtype).pin_memory()
     t_e2e_upd = t_e2e_all = 0.0
     n_e2e = 0
     h2d = d2h = 0
@@ -292,7 +297,7 @@ def main():
         t_e2e_upd += t1 - t0
         t_e2e_all += t2 - t0
         n_e2e += len(ids) + len(dele)
-        h2d = ids_pin.numel() * 4 + vec_pin.numel() + del_pin.numel() * 4 + q_pin.numel()
+        h2d = ids_pin.numel() * 4 + vec_pin.numel() * vec_pin.element_size() + del_pin.numel() * 4 + q_pin.numel() * q_pin.element_size()
         d2h = oi_pin.numel() * 4 + od_pin.numel() * 4 + 4 * 104   # results + four status blocks
     torch.cuda.synchronize()
 
@@ -325,7 +330,7 @@ def main():
     if not args.no_sweep:
         # recall@10 against brute force over the live set, and the smallest L reaching 0.95
         live = np.flatnonzero(st.live)
-        truth = brute_topk_gpu(torch, base, torch.from_numpy(live).to(dev), queries, 10)
+        truth = brute_topk_gpu(torch, base, torch.from_numpy(live).to(dev), queries, 10, cfg["metric"], is_f32)
         sweep = []
         for L in (10, 16, 24, 32, 48, 64, 96, 128):
             reps = []
@@ -345,15 +350,15 @@ def main():
 
     cpu = None
     if not args.no_cpu_baseline:
-        r = oracle_run(steps=12, warmup=1)
+        r = oracle_run(steps=12, warmup=1, workload=args.workload)
         cpu = {k: r[k] for k in ("value", "unit", "cores", "kind", "sample")}
         cpu["search_qps"] = r["search_qps"]
 
     ms_per_step = (t_upd_ms + t_srch_ms) / K
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "int32", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "scale": args.scale, "built_on": cfg["build"], "dim": cfg["dim"], "R": cfg["R"],
+            "dtype": "f32" if is_f32 else "int32", "data": "synthetic",
+            "config": {"workload": args.workload, "scale": args.scale, "built_on": cfg["build"], "dim": cfg["dim"], "R": cfg["R"],
                        "L": cfg["L"], "alpha": cfg["alpha"], "step": f"insert {cfg['ins']} + delete {cfg['dele']} + search {cfg['nq']} (k=10)",
                        "l2": "index (vectors + adjacency) larger than L2, and a 256 MiB flush between steps",
                        "parallelism": f"replicas x{world}"},
@@ -372,8 +377,17 @@ def main():
     return 0
 
 
-def brute_topk_gpu(torch, base, live_ids, queries, k):
-    """Exact top-k of uint8 vectors under squared L2 with ties by id (harness only: ground truth)."""
+def brute_topk_gpu(torch, base, live_ids, queries, k, metric=0, is_f32=False):
+    """Ground truth for recall (harness only).  uint8 + squared L2: exact, ties by id.  fp32: fp32 matmul."""
+    if is_f32:
+        out = []
+        x = base[live_ids]
+        xn = (x * x).sum(1)
+        for lo in range(0, queries.shape[0], 128):
+            q = queries[lo:lo + 128]
+            d = -(q @ x.T) if metric == 1 else (xn[None, :] - 2 * (q @ x.T))
+            out.append(live_ids[torch.topk(d, k, dim=1, largest=False).indices])
+        return torch.cat(out)
     x = base[live_ids].to(torch.float32)
     xn = (x * x).sum(1).to(torch.int64)
     out = []

@@ -44,15 +44,16 @@ __device__ __forceinline__ bool visit_fresh(uint32_t* hash, uint32_t hash_bits, 
     if (tag == 0xFFFFu) return true;  // the empty marker cannot be stored: always re-evaluate
     const uint4 b = reinterpret_cast<const uint4*>(hash)[bucket];
     const uint32_t t2 = tag | (tag << 16);
-    if (__vcmpeq2(b.x, t2) | __vcmpeq2(b.y, t2) | __vcmpeq2(b.z, t2) | __vcmpeq2(b.w, t2)) return false;
-    // first empty half-word, else evict the slot the tag points at
-    const uint32_t e0 = __vcmpeq2(b.x, 0xFFFFFFFFu), e1 = __vcmpeq2(b.y, 0xFFFFFFFFu);
-    const uint32_t e2 = __vcmpeq2(b.z, 0xFFFFFFFFu), e3 = __vcmpeq2(b.w, 0xFFFFFFFFu);
+    // zero-halfword test: z(x) has bit 15 / 31 set where the low / high half of x is zero
+    auto z = [](uint32_t x) { return (x - 0x00010001u) & ~x & 0x80008000u; };
+    if (z(b.x ^ t2) | z(b.y ^ t2) | z(b.z ^ t2) | z(b.w ^ t2)) return false;
+    // first empty half-word (all ones), else evict the slot the tag points at
+    const uint32_t e0 = z(~b.x), e1 = z(~b.y), e2 = z(~b.z), e3 = z(~b.w);
     uint32_t slot;
-    if (e0) slot = (e0 & 0xFFFFu) ? 0 : 1;
-    else if (e1) slot = (e1 & 0xFFFFu) ? 2 : 3;
-    else if (e2) slot = (e2 & 0xFFFFu) ? 4 : 5;
-    else if (e3) slot = (e3 & 0xFFFFu) ? 6 : 7;
+    if (e0) slot = (e0 & 0x8000u) ? 0 : 1;
+    else if (e1) slot = (e1 & 0x8000u) ? 2 : 3;
+    else if (e2) slot = (e2 & 0x8000u) ? 4 : 5;
+    else if (e3) slot = (e3 & 0x8000u) ? 6 : 7;
     else slot = tag & 7u;
     reinterpret_cast<unsigned short*>(hash)[bucket * 8 + slot] = (unsigned short)tag;
     return true;
@@ -139,7 +140,7 @@ __global__ void __launch_bounds__(kSearchWarps * 32) beam_search_kernel(const Se
 #pragma unroll
         for (int u = 0; u < U; ++u) {
           const uint32_t idx = b0 + u * NT + team;
-          idv[u] = idx < n ? cid[idx] : kInvalid;
+          idv[u] = idx < n ? cid[idx] : kInvalid;  // (no early exit here: it would serialise the loads)
           if (idv[u] != kInvalid) {
             load_row<G, CPL>(store + (size_t)idv[u] * row_bytes, nchunk, t, v[u]);
           } else {
@@ -223,10 +224,10 @@ __global__ void __launch_bounds__(kSearchWarps * 32) beam_search_kernel(const Se
             }
             np = i + s;
           }
-          __syncwarp();
+          __syncwarp();  // every read of this chunk precedes its writes; lower chunks are not written from here
           if (np < L) beam[np] = e;
-          __syncwarp();
         }
+        __syncwarp();
       }
       // 4. drop the survivors in
       for (uint32_t r = lane; r < m; r += 32) {
