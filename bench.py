@@ -92,6 +92,16 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def max_over_ranks(values, dist, device):
+    """Element-wise maximum of a list of floats over all ranks (identity when not distributed).
+    Replicas share nothing on the data path; this reduction of the timers is the only collective."""
+    import torch
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    if dist is not None and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
 # ------------------------------------------------------------------ oracle arm
 def oracle_run(steps, warmup, seed=0, workload=WORKLOAD):
     """The CPU oracle on a bounded shrink of the stream: build 10,000 points (untimed), then steps of
@@ -302,10 +312,7 @@ def main():
     torch.cuda.synchronize()
 
     # ---- max over ranks
-    times = torch.tensor([t_ins + t_del, t_srch, t_e2e_upd], dtype=torch.float64, device=dev)
-    if dist:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    t_upd_ms, t_srch_ms, t_e2e_s = times.tolist()
+    t_upd_ms, t_srch_ms, t_e2e_s = max_over_ranks([t_ins + t_del, t_srch, t_e2e_upd], dist, dev)
     value = world * n_upd / (t_upd_ms * 1e-3)
     e2e_value = world * n_e2e / t_e2e_s
     search_qps = world * cfg["nq"] * K / (t_srch_ms * 1e-3)

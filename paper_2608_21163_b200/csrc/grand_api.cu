@@ -58,6 +58,7 @@ struct grand_index {
   uint8_t* store = nullptr;
   uint32_t *adj = nullptr, *deg = nullptr, *live = nullptr;
   uint8_t* rowpfx = nullptr;
+  uint32_t* rowd = nullptr;
   DevState* d_state = nullptr;
   DevState* h_state = nullptr;  // pinned mirror
   uint32_t entry = GRAND_INVALID_ID;
@@ -136,7 +137,7 @@ int ensure(grand_index* idx, Buf& b, size_t bytes, cudaStream_t s) {
 
 GraphView view(const grand_index* idx) {
   GraphView g;
-  g.store = idx->store; g.adj = idx->adj; g.deg = idx->deg; g.live = idx->live; g.rowpfx = idx->rowpfx; g.R = idx->R; g.cap = idx->cap;
+  g.store = idx->store; g.adj = idx->adj; g.deg = idx->deg; g.live = idx->live; g.rowpfx = idx->rowpfx; g.rowd = idx->rowd; g.R = idx->R; g.cap = idx->cap;
   return g;
 }
 
@@ -284,6 +285,7 @@ int grand_create_ex(uint32_t dim, uint32_t dtype, uint32_t metric, uint32_t R, u
   A(alloc_dev(idx, &idx->deg, cap, true));
   A(alloc_dev(idx, &idx->live, words, true));
   A(alloc_dev(idx, &idx->rowpfx, cap, true));
+  if (idx->mode == GRAND_MODE_VAMANA) A(alloc_dev(idx, &idx->rowd, (size_t)cap * R, false));
   A(alloc_dev(idx, &idx->d_state, 1, true));
   A(alloc_dev(idx, &idx->mark, words, true));
   A(alloc_dev(idx, &idx->cnt, cap, true));
@@ -302,6 +304,7 @@ int grand_create_ex(uint32_t dim, uint32_t dtype, uint32_t metric, uint32_t R, u
   A(alloc_dev(idx, &idx->mean_row, lay.row_bytes, true));
   A(alloc_dev(idx, &idx->search_ctrs, 64, true));
   if (rc == GRAND_OK && cudaMemset(idx->adj, 0xFF, (size_t)cap * R * 4) != cudaSuccess) rc = GRAND_ERR_CUDA;
+  if (rc == GRAND_OK && idx->rowd && cudaMemset(idx->rowd, 0xFF, (size_t)cap * R * 4) != cudaSuccess) rc = GRAND_ERR_CUDA;
   if (rc == GRAND_OK && cudaMallocHost(&idx->h_state, sizeof(DevState)) != cudaSuccess) rc = GRAND_ERR_CUDA;
   if (rc == GRAND_OK) {
     memset(idx->h_state, 0, sizeof(DevState));
@@ -614,6 +617,7 @@ int grand_import_graph(grand_index* idx, const uint32_t* adj, const uint32_t* de
   CK(cudaMemcpyAsync(idx->live, live, (idx->cap + 31) / 32 * 4, cudaMemcpyDeviceToDevice, s));
   CK(launch_pad_rows(idx->lay, idx->store, vecs, idx->cap, s));
   CK(cudaMemsetAsync(idx->rowpfx, 0, idx->cap, s));
+  if (idx->rowd) CK(cudaMemsetAsync(idx->rowd, 0xFF, (size_t)idx->cap * idx->R * 4, s));
   CK(launch_pad_adjacency(idx->adj, idx->deg, idx->cap, idx->R, s));
   idx->entry = entry;
   idx->nlive = 0;

@@ -41,6 +41,7 @@ struct GraphView {
   uint32_t* adj;
   uint32_t* deg;
   uint32_t* live;  // bitmap
+  uint32_t* rowd;  // optional, cap x R: order-preserving bits of dist(u, adj[u][s]); 0xFFFFFFFF = not known
   uint8_t* rowpfx;  // per row: length of the leading run that is a RobustPrune output in ascending key
                     // order (no member of the run prunes a later member); appended entries follow it
   uint32_t R;

@@ -17,7 +17,7 @@ constexpr uint32_t kMaxR = 128;
 // block takes part.  Selected candidate indices go to out_idx; returns how many were selected.
 template <typename T, int G, int CPL>
 __device__ uint32_t block_prune(const uint8_t* __restrict__ store, uint32_t row_bytes, uint32_t nchunk, const AlphaParam ap,
-                                const unsigned long long* cand, uint32_t n, uint32_t R, uint32_t* validw,
+                                const unsigned long long* cand, uint32_t n, uint32_t R, uint32_t* validw, uint32_t* vlist,
                                 uint32_t* out_idx, volatile uint32_t* sh_sel, unsigned long long& npair) {
   using Dist = typename Elem<T>::Dist;
   constexpr unsigned FULL = 0xFFFFFFFFu;
@@ -31,21 +31,18 @@ __device__ uint32_t block_prune(const uint8_t* __restrict__ store, uint32_t row_
   __syncthreads();
   uint32_t cnt = 0;
   for (;;) {
-    if (warp == 0) {  // p* = first valid candidate
-      uint32_t s = kInvalid;
-      for (uint32_t wb = 0; wb < nwords; wb += 32) {
-        const uint32_t w = wb + lane;
-        const uint32_t word = w < nwords ? validw[w] : 0u;
-        const unsigned bal = __ballot_sync(FULL, word != 0u);
-        if (bal) {
-          const int srcl = __ffs(bal) - 1;
-          const uint32_t ww = __shfl_sync(FULL, word, srcl);
-          s = (wb + srcl) * 32 + __ffs(ww) - 1;
-          break;
-        }
+    if (warp == 0) {  // compact the valid set (ascending); p* = its head
+      uint32_t nv = 0;
+      for (uint32_t wd = 0; wd < nwords; ++wd) {
+        const uint32_t bits = validw[wd];
+        if ((bits >> lane) & 1u) vlist[nv + __popc(bits & ((1u << lane) - 1u))] = wd * 32 + lane;
+        nv += __popc(bits);
       }
+      __syncwarp();
       if (lane == 0) {
-        *sh_sel = s;
+        const uint32_t s = nv ? vlist[0] : kInvalid;
+        sh_sel[0] = s;
+        sh_sel[1] = nv;
         if (s != kInvalid) {
           out_idx[cnt] = s;
           validw[s >> 5] &= ~(1u << (s & 31));
@@ -53,16 +50,17 @@ __device__ uint32_t block_prune(const uint8_t* __restrict__ store, uint32_t row_
       }
     }
     __syncthreads();
-    const uint32_t s = *sh_sel;
+    const uint32_t s = sh_sel[0], nv = sh_sel[1];
     if (s == kInvalid) break;
     ++cnt;
     if (cnt == R) break;
-    // invalidate every remaining p' with alpha * dist(p*, p') <= D_p[p']
+    // invalidate every remaining p' with alpha * dist(p*, p') <= D_p[p']: only live candidates are visited
     uint4 pstar[CPL];
     load_row<G, CPL>(store + (size_t)key_id(cand[s]) * row_bytes, nchunk, t, pstar);
-    for (uint32_t jb = s + 1; jb < n; jb += nteams) {
-      const uint32_t j = jb + team_global;
-      const bool act = j < n && ((validw[j >> 5] >> (j & 31)) & 1u);
+    for (uint32_t jb = 1; jb < nv; jb += nteams) {
+      const uint32_t kk = jb + team_global;
+      const bool act = kk < nv;
+      const uint32_t j = act ? vlist[kk] : 0u;
       uint4 v[CPL];
       if (act) {
         load_row<G, CPL>(store + (size_t)key_id(cand[j]) * row_bytes, nchunk, t, v);
@@ -86,8 +84,9 @@ template <typename T, int METRIC, int G, int CPL>
 __global__ void __launch_bounds__(kPruneThreads) forward_prune_kernel(const PruneArgs a) {
   __shared__ unsigned long long cand[kMaxCand];
   __shared__ uint32_t validw[kMaxCand / 32];
+  __shared__ uint32_t vlist[kMaxCand];
   __shared__ uint32_t out_idx[kMaxR];
-  __shared__ uint32_t sh_sel;
+  __shared__ uint32_t sh_sel[2];
   const uint32_t tid = threadIdx.x, nthreads = blockDim.x;
   const uint32_t R = a.g.R;
   const AlphaParam ap{a.A_fix, a.alpha};
@@ -111,7 +110,7 @@ __global__ void __launch_bounds__(kPruneThreads) forward_prune_kernel(const Prun
       for (uint32_t j = tid; j < cnt; j += nthreads) out_idx[j] = j;
       __syncthreads();
     } else {
-      cnt = block_prune<T, G, CPL>(a.g.store, a.lay.row_bytes, a.lay.nchunk, ap, cand, n, R, validw, out_idx, &sh_sel, npair);
+      cnt = block_prune<T, G, CPL>(a.g.store, a.lay.row_bytes, a.lay.nchunk, ap, cand, n, R, validw, vlist, out_idx, sh_sel, npair);
       ++nprune;
     }
     for (uint32_t s = tid; s < R; s += nthreads) {
@@ -123,6 +122,7 @@ __global__ void __launch_bounds__(kPruneThreads) forward_prune_kernel(const Prun
         rk = (k & 0xFFFFFFFF00000000ull) | p;  // dist(p, id) is symmetric: the request carries it
       }
       a.g.adj[(size_t)p * R + s] = id;
+      if (a.g.rowd) a.g.rowd[(size_t)p * R + s] = s < cnt ? (uint32_t)(cand[out_idx[s]] >> 32) : kInvalid;
       a.req_tgt[i * R + s] = id;
       a.req_key[i * R + s] = rk;
     }

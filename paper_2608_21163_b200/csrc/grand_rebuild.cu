@@ -28,7 +28,7 @@ constexpr uint32_t kWorkChunk = 1;       // dirty nodes taken per work-counter b
 static inline uint32_t even_up_h(uint32_t x) { return (x + 1u) & ~1u; }
 static size_t rebuild_smem_per_warp(uint32_t R, uint32_t P) {
   const size_t NM = R + P, W = (NM + 31) / 32, Rp = even_up_h(R);
-  size_t b = (size_t)kSegSmem * 8 + (size_t)P * 8 + NM * 8 + Rp * 4 * 2 + NM * W * 4;
+  size_t b = (size_t)kSegSmem * 8 + (size_t)P * 8 + NM * 8 + Rp * 4 * 3 + NM * W * 4;
   return (b + 15) / 16 * 16;
 }
 
@@ -47,7 +47,8 @@ __global__ void __launch_bounds__(kRebuildWarps * 32) rebuild_kernel(const Rebui
   unsigned long long* scratch = seg_s + kSegSmem;
   unsigned long long* cand = scratch + P;
   uint32_t* keep = reinterpret_cast<uint32_t*>(cand + NM);
-  uint32_t* out_idx = keep + Rp;
+  uint32_t* keepd = keep + Rp;     // cached dist(u, keep[j]) bits (0xFFFFFFFF = not cached)
+  uint32_t* out_idx = keepd + Rp;
   uint32_t* prune = out_idx + Rp;  // NM rows x W words: bit j of row i = "c_i prunes c_j"
   uint32_t* upos = reinterpret_cast<uint32_t*>(scratch);  // positions of uncertain candidates (2P entries; scratch is free by then)
   unsigned long long* cs = cand;  // C in key order: cand itself, or the segment buffer after a rank merge
@@ -128,7 +129,11 @@ __global__ void __launch_bounds__(kRebuildWarps * 32) rebuild_kernel(const Rebui
         ok = !(a.delmap && bit_test(a.delmap, v));
       }
       const unsigned bal = __ballot_sync(FULL, ok);
-      if (ok) keep[nk + __popc(bal & lt_mask)] = v;
+      if (ok) {
+        const uint32_t pos = nk + __popc(bal & lt_mask);
+        keep[pos] = v;
+        keepd[pos] = a.g.rowd ? a.g.rowd[(size_t)u * R + s] : kInvalid;
+      }
       nk += __popc(bal);
       kp += __popc(__ballot_sync(FULL, ok && s < pfx));
     }
@@ -151,19 +156,32 @@ __global__ void __launch_bounds__(kRebuildWarps * 32) rebuild_kernel(const Rebui
     __syncwarp();
     const uint32_t nC = nk + nf;
     if (nC <= R) {
-      for (uint32_t s = lane; s < R; s += 32) row[s] = s < nk ? keep[s] : (s < nC ? key_id(cand[s]) : kInvalid);
+      for (uint32_t s = lane; s < R; s += 32) {
+        row[s] = s < nk ? keep[s] : (s < nC ? key_id(cand[s]) : kInvalid);
+        if (a.g.rowd) a.g.rowd[(size_t)u * R + s] = s < nk ? keepd[s] : (s < nC ? (uint32_t)(cand[s] >> 32) : kInvalid);
+      }
       if (lane == 0) {
         a.g.deg[u] = nC;
         a.g.rowpfx[u] = (uint8_t)kp;  // the surviving part of the pruned run still leads the row
       }
     } else {
       // ---- D_u for the kept neighbours (those appended after the last prune are tagged uncertain)
-      {
+      bool all_cached = true;
+      for (uint32_t jb = 0; jb < nk; jb += 32) {
+        const uint32_t j = jb + lane;
+        bool miss = false;
+        if (j < nk) {
+          miss = keepd[j] == kInvalid;
+          if (!miss) cand[j] = ((unsigned long long)keepd[j] << 32) | keep[j] | (j >= kp ? kExpandedBit : 0ull);
+        }
+        if (__any_sync(FULL, miss)) all_cached = false;
+      }
+      if (!all_cached) {
         uint4 ur[CPL];
         load_row<G, CPL>(store + (size_t)u * row_bytes, nchunk, t, ur);
         for (uint32_t jb = 0; jb < nk; jb += NT) {
           const uint32_t j = jb + team;
-          const bool act = j < nk;
+          const bool act = j < nk && keepd[j] == kInvalid;
           uint4 v[CPL];
           if (act) {
             load_row<G, CPL>(store + (size_t)keep[j] * row_bytes, nchunk, t, v);
@@ -179,6 +197,90 @@ __global__ void __launch_bounds__(kRebuildWarps * 32) rebuild_kernel(const Rebui
         }
       }
       __syncwarp();
+      if (kp == nk && nf == 1) {
+        // ---- the common case of an insert batch: a full row that is entirely prune output receives one
+        //      fresh candidate p.  Kept members never prune each other, so the sequential prune reduces to:
+        //      (1) does a kept member closer than p prune p?  then nothing changes;  (2) otherwise p enters
+        //      at its rank and the only other tests that can fire are p against the members behind it.
+        const unsigned long long kf = key_clean(cand[nk]);
+        const Dist Dp = key_dist<Dist>(kf);
+        uint32_t pos = 0;
+        for (uint32_t jb = 0; jb < nk; jb += 32) pos += __popc(__ballot_sync(FULL, jb + lane < nk && cand[jb + lane] < kf));
+        uint4 rf[CPL];
+        load_row<G, CPL>(store + (size_t)key_id(kf) * row_bytes, nchunk, t, rf);
+        bool pruned = false;
+        for (uint32_t ib = 0; ib < pos && !pruned; ib += NT) {
+          const uint32_t i = ib + team;
+          const bool act = i < pos;
+          uint4 rx[CPL];
+          if (act) {
+            load_row<G, CPL>(store + (size_t)key_id(cand[i]) * row_bytes, nchunk, t, rx);
+          } else {
+#pragma unroll
+            for (int c = 0; c < CPL; ++c) rx[c] = make_uint4(0, 0, 0, 0);
+          }
+          const Dist d = team_dist_regs<T, kMetricL2, G, CPL>(rf, rx);
+          if (act && t == 0) ++npair;
+          if (__any_sync(FULL, act && alpha_test(ap, d, Dp))) pruned = true;
+        }
+        if (!pruned) {
+          for (uint32_t w = lane; w < W; w += 32) prune[w] = 0u;  // bit j: kept member j is pruned by p
+          __syncwarp();
+          for (uint32_t jb = pos; jb < nk; jb += NT) {
+            const uint32_t j = jb + team;
+            const bool act = j < nk;
+            uint4 rx[CPL];
+            if (act) {
+              load_row<G, CPL>(store + (size_t)key_id(cand[j]) * row_bytes, nchunk, t, rx);
+            } else {
+#pragma unroll
+              for (int c = 0; c < CPL; ++c) rx[c] = make_uint4(0, 0, 0, 0);
+            }
+            const Dist d = team_dist_regs<T, kMetricL2, G, CPL>(rf, rx);
+            if (act && t == 0) {
+              ++npair;
+              if (alpha_test(ap, d, key_dist<Dist>(cand[j]))) atomicOr(&prune[j >> 5], 1u << (j & 31));
+            }
+          }
+          __syncwarp();
+          // new row: kept[0..pos), p, surviving kept[pos..), cut at R
+          uint32_t wpos = 0;
+          for (uint32_t sb = 0; sb <= nk; sb += 32) {
+            const uint32_t q = sb + lane;
+            bool ok = false;
+            unsigned long long key = 0;
+            if (q <= nk) {
+              if (q < pos) {
+                key = cand[q];
+                ok = true;
+              } else if (q == pos) {
+                key = kf;
+                ok = true;
+              } else {
+                key = cand[q - 1];
+                ok = !((prune[(q - 1) >> 5] >> ((q - 1) & 31)) & 1u);
+              }
+            }
+            const unsigned bal = __ballot_sync(FULL, ok);
+            const uint32_t o = wpos + __popc(bal & lt_mask);
+            if (ok && o < R) {
+              row[o] = key_id(key);
+              if (a.g.rowd) a.g.rowd[(size_t)u * R + o] = (uint32_t)(key >> 32);
+            }
+            wpos += __popc(bal);
+          }
+          const uint32_t cnt = min(wpos, R);
+          for (uint32_t sl = cnt + lane; sl < R; sl += 32) {
+            row[sl] = kInvalid;
+            if (a.g.rowd) a.g.rowd[(size_t)u * R + sl] = kInvalid;
+          }
+          if (lane == 0) {
+            a.g.deg[u] = cnt;
+            a.g.rowpfx[u] = (uint8_t)cnt;
+          }
+        }
+        ++nprune;
+      } else {
       // ---- C in key order.  The kept prefix is prune output and therefore already ascending: sort
       //      only the uncertain tail and merge the two runs by rank (checked, with a full sort as the
       //      fallback); long candidate lists take the full sort as well.
@@ -236,19 +338,31 @@ __global__ void __launch_bounds__(kRebuildWarps * 32) rebuild_kernel(const Rebui
           nfound += __popc(bal);
         }
         __syncwarp();
-        const uint32_t nwork = nu * nC;
-        for (uint32_t eb = 0; eb < nwork; eb += NT) {
-          const uint32_t e = eb + team;
-          bool act = e < nwork;
-          uint32_t i = 0, j = 1;
-          if (act) {
-            const uint32_t f = upos[e / nC], x = e % nC;
+        // each uncertain member f against every other candidate x; its row stays in registers
+        for (uint32_t fi = 0; fi < nu; ++fi) {
+          const uint32_t f = upos[fi];
+          const unsigned long long kf = cs[f];
+          uint4 rf[CPL];
+          load_row<G, CPL>(store + (size_t)key_id(kf) * row_bytes, nchunk, t, rf);
+          for (uint32_t xb = 0; xb < nC; xb += NT) {
+            const uint32_t x = xb + team;
             // skip self; a pair of two uncertain members is taken once, from its larger member
-            act = f != x && !(x > f && (cs[x] & kExpandedBit));
-            i = min(f, x);
-            j = max(f, x);
+            const unsigned long long kx = x < nC ? cs[x] : 0ull;
+            const bool act = x < nC && x != f && !(x > f && (kx & kExpandedBit));
+            uint4 rx[CPL];
+            if (act) {
+              load_row<G, CPL>(store + (size_t)key_id(kx) * row_bytes, nchunk, t, rx);
+            } else {
+#pragma unroll
+              for (int c = 0; c < CPL; ++c) rx[c] = make_uint4(0, 0, 0, 0);
+            }
+            const Dist d = team_dist_regs<T, kMetricL2, G, CPL>(rf, rx);  // bitwise symmetric in its operands
+            if (act && t == 0) {
+              ++npair;
+              const uint32_t i = min(f, x), j = max(f, x);
+              if (alpha_test(ap, d, key_dist<Dist>(x < f ? kf : kx))) atomicOr(&prune[i * W + (j >> 5)], 1u << (j & 31));
+            }
           }
-          pair_test(act, i, j, jprev, rj);
         }
       } else {
         __syncwarp();
@@ -283,12 +397,17 @@ __global__ void __launch_bounds__(kRebuildWarps * 32) rebuild_kernel(const Rebui
         if ((uint32_t)lane < W) valid &= ~prune[i * W + lane];
       }
       __syncwarp();
-      for (uint32_t s = lane; s < R; s += 32) row[s] = s < cnt ? key_id(cs[out_idx[s]]) : kInvalid;
+      for (uint32_t s = lane; s < R; s += 32) {
+        const unsigned long long ks = s < cnt ? cs[out_idx[s]] : kKeyMax;
+        row[s] = s < cnt ? key_id(ks) : kInvalid;
+        if (a.g.rowd) a.g.rowd[(size_t)u * R + s] = (uint32_t)(ks >> 32);
+      }
       if (lane == 0) {
         a.g.deg[u] = cnt;
         a.g.rowpfx[u] = (uint8_t)cnt;
       }
       ++nprune;
+      }  // general prune
     }
     if (lane == 0) {
       a.cnt[u] = 0;
