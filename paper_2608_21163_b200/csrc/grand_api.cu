@@ -24,8 +24,8 @@ Layout make_layout(uint32_t dim, uint32_t dtype, uint32_t metric) {
   l.esize = dtype == GRAND_F32 ? 4 : 1;
   l.row_bytes = (uint32_t)(((uint64_t)dim * l.esize + 15) / 16 * 16);
   l.nchunk = l.row_bytes / 16;
-  static const int Gs[8] = {2, 8, 8, 8, 8, 32, 32, 32};
-  static const int Cs[8] = {1, 1, 2, 3, 4, 2, 4, 8};
+  static const int Gs[8] = {2, 4, 8, 8, 8, 32, 32, 32};
+  static const int Cs[8] = {1, 2, 2, 3, 4, 2, 4, 8};
   static const uint32_t lim[8] = {2, 8, 16, 24, 32, 64, 128, 256};
   l.code = -1;
   for (int i = 0; i < 8; ++i)
@@ -69,7 +69,7 @@ struct grand_index {
   uint32_t* wk_n = nullptr;
   uint32_t wk_stride = 0;
   unsigned long long* Ci = nullptr;
-  uint32_t *Ci_n = nullptr, *in_cnt = nullptr, *pair_off = nullptr, *scan_tmp = nullptr;
+  uint32_t *Ci_n = nullptr, *in_cnt = nullptr, *pair_off = nullptr, *unit_off = nullptr, *scan_tmp = nullptr;
   uint8_t* mean_row = nullptr;
   uint32_t* search_ctrs = nullptr;  // ring of work counters, one per in-flight search launch
   uint32_t ctr_next = 0;
@@ -300,6 +300,7 @@ int grand_create_ex(uint32_t dim, uint32_t dtype, uint32_t metric, uint32_t R, u
   A(alloc_dev(idx, &idx->Ci_n, mb, true));
   A(alloc_dev(idx, &idx->in_cnt, mb + 1, true));
   A(alloc_dev(idx, &idx->pair_off, mb + 1, true));
+  A(alloc_dev(idx, &idx->unit_off, mb + 1, true));
   A(alloc_dev(idx, &idx->scan_tmp, (cap + 1) / 2048 + mb / 2048 + 8, true));
   A(alloc_dev(idx, &idx->mean_row, lay.row_bytes, true));
   A(alloc_dev(idx, &idx->search_ctrs, 64, true));
@@ -464,7 +465,7 @@ int grand_delete_batch(grand_index* idx, const uint32_t* ids, uint64_t n, grand_
   d.lay = idx->lay; d.g = g; d.ids = ids; d.n = n; d.delmap = idx->mark;
   d.beam = idx->wk_keys; d.beam_n = idx->wk_n; d.beam_stride = idx->wk_stride;
   d.Ci = idx->Ci; d.Ci_n = idx->Ci_n; d.k_repair = idx->k_repair; d.c = idx->c;
-  d.in_cnt = idx->in_cnt; d.pair_off = idx->pair_off; d.scan_tmp = idx->scan_tmp;
+  d.in_cnt = idx->in_cnt; d.pair_off = idx->pair_off; d.unit_off = idx->unit_off; d.scan_tmp = idx->scan_tmp;
   d.flag = idx->flag; d.state = idx->d_state;
   {
     // reverse graph of the snapshot: exact in-neighbours, rebuilt per batch and not kept

@@ -183,18 +183,152 @@ __global__ void delete_touch_kernel(const DeleteArgs a, const uint64_t total_in)
   }
 }
 
+// ---- staged variant: C_i is shared by every pair of deleted node i, so a block copies its rows into
+// shared memory once and its warps run the pairs of that node against the copy.  Work units are
+// chunks of kUnitPairs pairs of one node (hubs with long in-neighbour rows are split over blocks).
+constexpr uint32_t kUnitPairs = 256;
+__global__ void delete_units_kernel(const DeleteArgs a) {
+  for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i <= a.n; i += (uint64_t)gridDim.x * blockDim.x) {
+    uint32_t units = 0;
+    if (i < a.n) units = (a.pair_off[i + 1] - a.pair_off[i] + a.g.R + kUnitPairs - 1) / kUnitPairs;
+    a.in_cnt[i] = units;  // the in-degree counts are not needed once their prefix exists
+  }
+}
+
+template <typename T, int METRIC, int G, int CPL>
+__global__ void __launch_bounds__(kPickWarps * 32) delete_picks_staged_kernel(const DeleteArgs a, const uint64_t total_in) {
+  using Dist = typename Elem<T>::Dist;
+  constexpr unsigned FULL = 0xFFFFFFFFu;
+  constexpr int NT = 32 / G;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int t = lane % G, team = lane / G;
+  const uint32_t R = a.g.R, c = a.c, kr = a.k_repair;
+  const uint32_t row_bytes = a.lay.row_bytes, nchunk = a.lay.nchunk;
+  uint8_t* crow = smem_raw;                                                    // k_repair staged rows
+  unsigned long long* ckeys = reinterpret_cast<unsigned long long*>(smem_raw + (size_t)kr * row_bytes);  // their keys
+  unsigned long long* keys = ckeys + kr + (size_t)warp * kMaxKRepair;          // per-warp pick scratch
+  const uint32_t nunits = a.unit_off[a.n];
+  unsigned long long npair = 0;
+  for (uint32_t unit = blockIdx.x; unit < nunits; unit += gridDim.x) {
+    uint32_t lo = 0, hi = (uint32_t)a.n;  // largest i with unit_off[i] <= unit
+    while (hi - lo > 1) {
+      const uint32_t mid = (lo + hi) >> 1;
+      if (a.unit_off[mid] <= unit) lo = mid; else hi = mid;
+    }
+    const uint32_t i = lo, p = a.ids[i];
+    const uint32_t nin = a.pair_off[i + 1] - a.pair_off[i];
+    const uint32_t q0 = (unit - a.unit_off[i]) * kUnitPairs, q1 = min(nin + R, q0 + kUnitPairs);
+    const uint32_t nc = a.Ci_n[i];
+    __syncthreads();  // the previous unit's readers are done with the staged rows
+    for (uint32_t j = threadIdx.x; j < nc; j += blockDim.x) ckeys[j] = a.Ci[(size_t)i * kr + j];
+    for (uint32_t e = threadIdx.x; e < nc * nchunk; e += blockDim.x) {
+      const uint32_t j = e / nchunk, ch = e - j * nchunk;
+      const uint32_t y = key_id(a.Ci[(size_t)i * kr + j]);
+      reinterpret_cast<uint4*>(crow + (size_t)j * row_bytes)[ch] = __ldg(reinterpret_cast<const uint4*>(a.g.store + (size_t)y * row_bytes) + ch);
+    }
+    __syncthreads();
+    for (uint32_t q = q0 + warp; q < q1; q += kPickWarps) {
+      const bool is_in = q < nin;
+      uint32_t x = kInvalid;
+      uint64_t rbase;
+      if (is_in) {
+        x = a.src[a.off[p] + q];
+        rbase = ((uint64_t)a.pair_off[i] + q) * c;
+      } else {
+        const uint32_t sl = q - nin;
+        if (sl < a.g.deg[p]) x = a.g.adj[(size_t)p * R + sl];
+        rbase = (total_in + (uint64_t)i * R + sl) * c;
+      }
+      if (x == kInvalid || bit_test(a.delmap, x)) {
+        if (lane < c) a.req_tgt[rbase + lane] = kInvalid;
+        continue;
+      }
+      uint4 xr[CPL];
+      load_row<G, CPL>(a.g.store + (size_t)x * row_bytes, nchunk, t, xr);
+      for (uint32_t jb = 0; jb < nc; jb += NT) {
+        const uint32_t j = jb + team;
+        unsigned long long kc = 0;
+        uint4 v[CPL];
+        if (j < nc) {
+          kc = ckeys[j];
+#pragma unroll
+          for (int cc = 0; cc < CPL; ++cc) {
+            const uint32_t ch = t + cc * G;
+            v[cc] = ch < nchunk ? reinterpret_cast<const uint4*>(crow + (size_t)j * row_bytes)[ch] : make_uint4(0, 0, 0, 0);
+          }
+        } else {
+#pragma unroll
+          for (int cc = 0; cc < CPL; ++cc) v[cc] = make_uint4(0, 0, 0, 0);
+        }
+        const Dist d = team_dist_regs<T, kMetricL2, G, CPL>(xr, v);
+        if (t == 0 && j < nc) {
+          const uint32_t y = key_id(kc);
+          keys[j] = y != x ? make_key(d, y) : kKeyMax;
+          npair += y != x;
+        }
+      }
+      __syncwarp();
+      for (uint32_t r = 0; r < c; ++r) {  // r-th smallest (dist, id)
+        unsigned long long best = kKeyMax;
+        for (uint32_t j = lane; j < nc; j += 32) best = min(best, keys[j]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) best = min(best, __shfl_xor_sync(FULL, best, o));
+        if (best != kKeyMax) {
+          for (uint32_t j = lane; j < nc; j += 32)
+            if (keys[j] == best) keys[j] = kKeyMax;
+        }
+        if (lane == 0) {
+          if (best == kKeyMax) {
+            a.req_tgt[rbase + r] = kInvalid;
+          } else if (is_in) {
+            a.req_tgt[rbase + r] = x;
+            a.req_key[rbase + r] = best;
+          } else {
+            a.req_tgt[rbase + r] = key_id(best);
+            a.req_key[rbase + r] = (best & 0xFFFFFFFF00000000ull) | x;
+          }
+        }
+        __syncwarp();
+      }
+    }
+  }
+  if (npair) atomicAdd(&a.state->counters[CTR_PAIR], npair);
+}
+
 template <typename T, int METRIC, int G, int CPL>
 static cudaError_t launch_delete_picks_t(const DeleteArgs& a, uint64_t total_in, cudaStream_t s) {
   const uint64_t total = total_in + a.n * a.g.R;
   if (total == 0) return cudaSuccess;
-  uint64_t blocks = (total + kPickWarps - 1) / kPickWarps;
-  if (blocks > 148u * 16u) blocks = 148u * 16u;
   if (total_in) {
     uint64_t tb = (total_in + 255) / 256;
     if (tb > 148u * 32u) tb = 148u * 32u;
     delete_touch_kernel<<<(unsigned)tb, 256, 0, s>>>(a, total_in);
     count_launches(1);
   }
+  const size_t stage = (size_t)a.k_repair * a.lay.row_bytes;
+  if (stage <= 64 * 1024) {
+    // candidate rows fit shared memory: one staged copy per work unit
+    const size_t smem = stage + ((size_t)a.k_repair + (size_t)kPickWarps * kMaxKRepair) * 8;
+    auto kern = delete_picks_staged_kernel<T, METRIC, G, CPL>;
+    static size_t smem_set = 0;
+    if (smem > smem_set) {
+      cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      if (e != cudaSuccess) return e;
+      smem_set = smem;
+    }
+    const unsigned ub = (unsigned)((a.n + 256) / 256 > 148u * 16u ? 148u * 16u : (a.n + 256) / 256);
+    delete_units_kernel<<<ub, 256, 0, s>>>(a);
+    cudaError_t e = launch_exclusive_scan(a.in_cnt, a.unit_off, a.n + 1, a.scan_tmp, s);
+    if (e != cudaSuccess) return e;
+    uint64_t blocks = (total + kUnitPairs - 1) / kUnitPairs + a.n;  // upper bound on the number of units
+    if (blocks > 148u * 16u) blocks = 148u * 16u;
+    kern<<<(unsigned)blocks, kPickWarps * 32, smem, s>>>(a, total_in);
+    count_launches(2);
+    return cudaGetLastError();
+  }
+  uint64_t blocks = (total + kPickWarps - 1) / kPickWarps;
+  if (blocks > 148u * 16u) blocks = 148u * 16u;
   delete_picks_kernel<T, METRIC, G, CPL><<<(unsigned)blocks, kPickWarps * 32, 0, s>>>(a, total_in);
   count_launches(1);
   return cudaGetLastError();

@@ -158,6 +158,7 @@ struct DeleteArgs {
   uint32_t c;
   const uint32_t* off; const uint32_t* src;   // reverse graph
   uint32_t* in_cnt; uint32_t* pair_off;       // n+1
+  uint32_t* unit_off;                         // n+1: work units (chunks of pairs) per deleted node, prefix
   uint32_t* scan_tmp;
   uint32_t* req_tgt; unsigned long long* req_key;   // (total_in + n*R) * c
   uint32_t* flag; uint32_t* dirty;
@@ -197,12 +198,12 @@ cudaError_t launch_fill_u32(uint32_t* p, uint32_t v, uint64_t n, cudaStream_t s)
 
 }  // namespace grand
 
-// ---- (G, CPL) dispatch table.  nchunk <= 2 -> (2,1); <= 8 -> (8,1); <= 16 -> (8,2); <= 24 -> (8,3);
+// ---- (G, CPL) dispatch table.  nchunk <= 2 -> (2,1); <= 8 -> (4,2) (measured best for 128-byte rows); <= 16 -> (8,2); <= 24 -> (8,3);
 // <= 32 -> (8,4); <= 64 -> (32,2); <= 128 -> (32,4); <= 256 -> (32,8).
 #define GRAND_LAYOUT_SWITCH(code, FN, T, M, ...)            \
   switch (code) {                                           \
     case 0: return FN<T, M, 2, 1>(__VA_ARGS__);             \
-    case 1: return FN<T, M, 8, 1>(__VA_ARGS__);             \
+    case 1: return FN<T, M, 4, 2>(__VA_ARGS__);             \
     case 2: return FN<T, M, 8, 2>(__VA_ARGS__);             \
     case 3: return FN<T, M, 8, 3>(__VA_ARGS__);             \
     case 4: return FN<T, M, 8, 4>(__VA_ARGS__);             \
