@@ -8,7 +8,6 @@ namespace grand {
 
 constexpr int kPickWarps = 4;
 constexpr uint32_t kMaxKRepair = 128;
-constexpr uint32_t kMaxC = 8;
 
 
 // in_cnt[i] = in-degree of p_i in the reverse graph (0 for an id that fails validation), then the

@@ -1,7 +1,6 @@
-// RobustPrune kernels: forward edges of new nodes (Alg. 5, first parallel loop), the rebuild of
-// dirty nodes after reverse-edge / repair requests were grouped (Alg. 5 dirty loop, Alg. 6 rebuild
-// loop), and the fixed-degree detour find-and-replace (Alg. 7).  One thread block owns one node, so
-// no two blocks ever write the same adjacency row.
+// Forward RobustPrune of new nodes (Alg. 5, first parallel loop; Alg. 4) and the fixed-degree detour
+// find-and-replace (Alg. 7).  One thread block owns one node, so no two blocks ever write the same
+// adjacency row.  (The rebuild of dirty nodes lives in grand_rebuild.cu.)
 #include "grand_common.cuh"
 #include "grand_kernels.h"
 
@@ -10,17 +9,17 @@ namespace grand {
 constexpr int kPruneThreads = 128;
 constexpr uint32_t kMaxCand = 1024;  // >= vmax limit
 constexpr uint32_t kSegCap = 1024;   // request segment sorted in shared memory up to this length
-constexpr uint32_t kMaxP = 256;
 constexpr uint32_t kMaxR = 128;
 
 // GrANDRobustPrune (Alg. 4) over candidate keys sorted ascending in shared memory.  The whole
-// block takes part.  Selected candidate indices go to out_idx; returns how many were selected.
+// block takes part.  Each iteration compacts the still-valid candidates into an index list, takes
+// its head as p*, and tests only the listed candidates against it (a team of G lanes per pair
+// distance).  Selected candidate indices go to out_idx; returns how many were selected.
 template <typename T, int G, int CPL>
 __device__ uint32_t block_prune(const uint8_t* __restrict__ store, uint32_t row_bytes, uint32_t nchunk, const AlphaParam ap,
                                 const unsigned long long* cand, uint32_t n, uint32_t R, uint32_t* validw, uint32_t* vlist,
                                 uint32_t* out_idx, volatile uint32_t* sh_sel, unsigned long long& npair) {
   using Dist = typename Elem<T>::Dist;
-  constexpr unsigned FULL = 0xFFFFFFFFu;
   const uint32_t tid = threadIdx.x, nthreads = blockDim.x;
   const int lane = tid & 31, warp = tid >> 5;
   const int t = lane % G;
