@@ -28,7 +28,7 @@ constexpr uint32_t kWorkChunk = 1;       // dirty nodes taken per work-counter b
 static inline uint32_t even_up_h(uint32_t x) { return (x + 1u) & ~1u; }
 static size_t rebuild_smem_per_warp(uint32_t R, uint32_t P) {
   const size_t NM = R + P, W = (NM + 31) / 32, Rp = even_up_h(R);
-  size_t b = (size_t)kSegSmem * 8 + (size_t)P * 8 + NM * 8 + Rp * 4 * 3 + NM * W * 4;
+  size_t b = (size_t)kSegSmem * 8 + (size_t)P * 8 + NM * 8 + Rp * 4 * 3 + (NM + 1) * W * 4;
   return (b + 15) / 16 * 16;
 }
 
@@ -50,6 +50,7 @@ __global__ void __launch_bounds__(kRebuildWarps * 32) rebuild_kernel(const Rebui
   uint32_t* keepd = keep + Rp;     // cached dist(u, keep[j]) bits (0xFFFFFFFF = not cached)
   uint32_t* out_idx = keepd + Rp;
   uint32_t* prune = out_idx + Rp;  // NM rows x W words: bit j of row i = "c_i prunes c_j"
+  uint32_t* hasp = prune + NM * W;  // W words: bit i = row i of the matrix is non-zero (c_i prunes something)
   uint32_t* upos = reinterpret_cast<uint32_t*>(scratch);  // positions of uncertain candidates (2P entries; scratch is free by then)
   unsigned long long* cs = cand;  // C in key order: cand itself, or the segment buffer after a rank merge
   const AlphaParam ap{a.A_fix, a.alpha};
@@ -76,7 +77,10 @@ __global__ void __launch_bounds__(kRebuildWarps * 32) rebuild_kernel(const Rebui
     const Dist d = team_dist_regs<T, kMetricL2, G, CPL>(ri, rj);
     if (act && t == 0) {
       ++npair;
-      if (alpha_test(ap, d, key_dist<Dist>(cs[j]))) atomicOr(&prune[i * W + (j >> 5)], 1u << (j & 31));
+      if (alpha_test(ap, d, key_dist<Dist>(cs[j]))) {
+        atomicOr(&prune[i * W + (j >> 5)], 1u << (j & 31));
+        atomicOr(&hasp[i >> 5], 1u << (i & 31));
+      }
     }
   };
 
@@ -322,6 +326,7 @@ __global__ void __launch_bounds__(kRebuildWarps * 32) rebuild_kernel(const Rebui
         cs = cand;
       }
       for (uint32_t w = lane; w < nC * W; w += 32) prune[w] = 0u;
+      if ((uint32_t)lane < W) hasp[lane] = 0u;
       // ---- prune tests in parallel: pairs with an uncertain member, or the whole upper triangle
       const uint32_t nu = nC - kpe;
       uint32_t jprev = kInvalid;
@@ -360,7 +365,10 @@ __global__ void __launch_bounds__(kRebuildWarps * 32) rebuild_kernel(const Rebui
             if (act && t == 0) {
               ++npair;
               const uint32_t i = min(f, x), j = max(f, x);
-              if (alpha_test(ap, d, key_dist<Dist>(x < f ? kf : kx))) atomicOr(&prune[i * W + (j >> 5)], 1u << (j & 31));
+              if (alpha_test(ap, d, key_dist<Dist>(x < f ? kf : kx))) {
+                atomicOr(&prune[i * W + (j >> 5)], 1u << (j & 31));
+                atomicOr(&hasp[i >> 5], 1u << (i & 31));
+              }
             }
           }
         }
@@ -387,20 +395,33 @@ __global__ void __launch_bounds__(kRebuildWarps * 32) rebuild_kernel(const Rebui
         const uint32_t lo = lane * 32;
         valid = nC >= lo + 32 ? 0xFFFFFFFFu : (nC > lo ? (1u << (nC - lo)) - 1u : 0u);
       }
-      uint32_t cnt = 0;
-      for (uint32_t i = 0; i < nC; ++i) {
-        const uint32_t word = __shfl_sync(FULL, valid, i >> 5);
-        if (!((word >> (i & 31)) & 1u)) continue;
-        if (lane == 0) out_idx[cnt] = i;
-        ++cnt;
-        if (cnt == R) break;
-        if ((uint32_t)lane < W) valid &= ~prune[i * W + lane];
+      // The valid set only changes when a still-valid candidate with a non-zero matrix row is reached, so
+      // only those candidates are visited, in ascending order; everything valid in between is selected.
+      for (uint32_t w = 0; w < W; ++w) {
+        uint32_t hw = hasp[w];
+        while (hw) {
+          const uint32_t b = __ffs(hw) - 1;
+          hw &= hw - 1;
+          const uint32_t vw = __shfl_sync(FULL, valid, w);
+          if (((vw >> b) & 1u) && (uint32_t)lane < W) valid &= ~prune[(w * 32 + b) * W + lane];
+        }
       }
-      __syncwarp();
-      for (uint32_t s = lane; s < R; s += 32) {
-        const unsigned long long ks = s < cnt ? cs[out_idx[s]] : kKeyMax;
-        row[s] = s < cnt ? key_id(ks) : kInvalid;
-        if (a.g.rowd) a.g.rowd[(size_t)u * R + s] = (uint32_t)(ks >> 32);
+      // the first R members of the final valid set, in key order, are the new row
+      uint32_t base_rank = 0;
+      for (uint32_t sb = 0; sb < nC; sb += 32) {
+        const uint32_t word = __shfl_sync(FULL, valid, sb >> 5);
+        const uint32_t rank = base_rank + __popc(word & lt_mask);
+        if (((word >> lane) & 1u) && rank < R) {
+          const unsigned long long ks = cs[sb + lane];
+          row[rank] = key_id(ks);
+          if (a.g.rowd) a.g.rowd[(size_t)u * R + rank] = (uint32_t)(ks >> 32);
+        }
+        base_rank += __popc(word);
+      }
+      const uint32_t cnt = min(base_rank, R);
+      for (uint32_t sl = cnt + lane; sl < R; sl += 32) {
+        row[sl] = kInvalid;
+        if (a.g.rowd) a.g.rowd[(size_t)u * R + sl] = kInvalid;
       }
       if (lane == 0) {
         a.g.deg[u] = cnt;
