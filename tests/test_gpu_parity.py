@@ -327,3 +327,46 @@ def test_run_twice_is_deterministic_and_counters_move():
     s = g1.stats()
     assert s["expansions"] > 0 and s["dist_evals"] > s["expansions"] and s["pair_dists"] > 0
     assert s["dirty_nodes"] > 0 and s["prunes"] > 0 and s["kernel_launches"] > 0
+
+
+def test_maximum_parameters_bit_exact():
+    """Limits of the kernels' fast paths: R = 128 (four id chunks per row), L beyond 256, a visited-list cap
+    of 600, P = 200 (candidate lists longer than the rank-merge buffer: full-sort path, 11-word bit
+    matrix rows), c = 8 and k_repair = 128."""
+    torch = torch_()
+    n, dim = 3000, 16
+    base = synth.uniform_u8(21, "base", 0, n, dim)
+    cfg = dict(dim=dim, dtype=go.U8, metric=go.L2, R=128, L=300, alpha=1.2, mode=go.VAMANA, max_build_batch=1000, ins=1, dele=600)
+    o, g = make_pair(cfg, n, P=200, c=8, k_repair=128, vmax=600)
+    for lo in range(0, n, 750):
+        ids = np.arange(lo, lo + 750, dtype=np.uint32)
+        o.insert_batch(ids, base[ids]); g.insert_batch(torch.from_numpy(ids), torch.from_numpy(base[ids]))
+        assert_same_graph(o, g, f"insert at {lo}")
+    dele = synth.choose_ids(21, "del", np.arange(n, dtype=np.uint32), 600)
+    o.delete_batch(dele); g.delete_batch(torch.from_numpy(dele))
+    assert_same_graph(o, g, "delete")
+    q = synth.uniform_u8(21, "query", 0, 100, dim)
+    for k, L in [(10, 300), (100, 512), (1, 257)]:
+        oi, od = o.search(q, k, L)
+        gi, gd = gpu_search(g, q, k, L)
+        assert (oi == gi).all() and (od == gd.astype(np.float64)).all()
+
+
+def test_small_degree_bound_and_alpha_one():
+    """R = 4 with alpha = 1.0: heavy pruning on every dirty node, rows shorter than a warp chunk."""
+    torch = torch_()
+    n, dim = 4000, 8
+    base = synth.uniform_u8(22, "base", 0, n, dim)
+    cfg = dict(dim=dim, dtype=go.U8, metric=go.L2, R=4, L=12, alpha=1.0, mode=go.VAMANA, max_build_batch=500, ins=1, dele=500)
+    o, g = make_pair(cfg, n)
+    for lo in range(0, n, 500):
+        ids = np.arange(lo, lo + 500, dtype=np.uint32)
+        o.insert_batch(ids, base[ids]); g.insert_batch(torch.from_numpy(ids), torch.from_numpy(base[ids]))
+        assert_same_graph(o, g, f"insert at {lo}")
+    for r in range(2):
+        live = np.flatnonzero(go.live_mask(o.export_graph()[2], n)).astype(np.uint32)
+        dele = synth.choose_ids(22, f"del{r}", live, 500)
+        o.delete_batch(dele); g.delete_batch(torch.from_numpy(dele))
+        assert_same_graph(o, g, f"delete {r}")
+        o.insert_batch(dele[:250], base[dele[:250]]); g.insert_batch(torch.from_numpy(dele[:250]), torch.from_numpy(base[dele[:250]]))
+        assert_same_graph(o, g, f"reinsert {r}")
