@@ -104,12 +104,12 @@ def max_over_ranks(values, dist, device):
 
 # ------------------------------------------------------------------ oracle arm
 def oracle_run(steps, warmup, seed=0, workload=WORKLOAD):
-    """The CPU oracle on a bounded shrink of the stream: build 10,000 points (untimed), then steps of
-    insert 250 + delete 250 + search 250.  Returns the JSON-ready dict of the reference arm."""
+    """The CPU oracle on a bounded shrink of the stream: build 20,000 points (untimed), then steps of
+    insert 500 + delete 500 + search 500.  Returns the JSON-ready dict of the reference arm."""
     from oracle import grand_oracle as go
     cfg = dict(synth.CONFIGS[workload])
-    per = 250
-    cfg.update(n=10_000 + (steps + warmup) * per, build=10_000, first_batch=1_000, max_build_batch=1_000,
+    per = 500
+    cfg.update(n=20_000 + (steps + warmup) * per, build=20_000, first_batch=1_000, max_build_batch=2_000,
                ins=per, dele=per, nq=per, rounds=steps + warmup)
     wl = synth.Workload(cfg, seed)
     st = synth.StreamState(wl)
@@ -138,7 +138,7 @@ def oracle_run(steps, warmup, seed=0, workload=WORKLOAD):
             t_upd += (t1 - t0) + (t3 - t2)
             t_search += t4 - t3
     value = 2 * per * steps / t_upd
-    sample = (f"{workload} shrunk: index built on 10,000 points (untimed, {t_build:.1f} s), then {steps} steps of "
+    sample = (f"{workload} shrunk: index built on 20,000 points (untimed, {t_build:.1f} s), then {steps} steps of "
               f"insert {per} + delete {per} + search {per} (k=10, L={cfg['L']})")
     return {"value": value, "unit": UNIT, "cores": o.nthreads, "kind": "oracle", "sample": sample,
             "search_qps": per * steps / t_search, "ms_per_step": 1e3 * (t_upd + t_search) / steps}
@@ -357,7 +357,7 @@ def main():
 
     cpu = None
     if not args.no_cpu_baseline:
-        r = oracle_run(steps=12, warmup=1, workload=args.workload)
+        r = oracle_run(steps=30, warmup=1, workload=args.workload)
         cpu = {k: r[k] for k in ("value", "unit", "cores", "kind", "sample")}
         cpu["search_qps"] = r["search_qps"]
 
