@@ -24,8 +24,8 @@ Layout make_layout(uint32_t dim, uint32_t dtype, uint32_t metric) {
   l.esize = dtype == GRAND_F32 ? 4 : 1;
   l.row_bytes = (uint32_t)(((uint64_t)dim * l.esize + 15) / 16 * 16);
   l.nchunk = l.row_bytes / 16;
-  static const int Gs[8] = {2, 4, 8, 8, 8, 32, 32, 32};
-  static const int Cs[8] = {1, 2, 2, 3, 4, 2, 4, 8};
+  static const int Gs[8] = {2, 4, 4, 4, 8, 32, 32, 32};
+  static const int Cs[8] = {1, 2, 4, 6, 4, 2, 4, 8};
   static const uint32_t lim[8] = {2, 8, 16, 24, 32, 64, 128, 256};
   l.code = -1;
   for (int i = 0; i < 8; ++i)

@@ -198,14 +198,14 @@ cudaError_t launch_fill_u32(uint32_t* p, uint32_t v, uint64_t n, cudaStream_t s)
 
 }  // namespace grand
 
-// ---- (G, CPL) dispatch table.  nchunk <= 2 -> (2,1); <= 8 -> (4,2) (measured best for 128-byte rows); <= 16 -> (8,2); <= 24 -> (8,3);
-// <= 32 -> (8,4); <= 64 -> (32,2); <= 128 -> (32,4); <= 256 -> (32,8).
+// ---- (G, CPL) dispatch table.  nchunk <= 2 -> (2,1); <= 8 -> (4,2); <= 16 -> (4,4); <= 24 -> (4,6) (teams of 4
+// measured best for 128- and 384-byte rows); <= 32 -> (8,4); <= 64 -> (32,2); <= 128 -> (32,4); <= 256 -> (32,8).
 #define GRAND_LAYOUT_SWITCH(code, FN, T, M, ...)            \
   switch (code) {                                           \
     case 0: return FN<T, M, 2, 1>(__VA_ARGS__);             \
     case 1: return FN<T, M, 4, 2>(__VA_ARGS__);             \
-    case 2: return FN<T, M, 8, 2>(__VA_ARGS__);             \
-    case 3: return FN<T, M, 8, 3>(__VA_ARGS__);             \
+    case 2: return FN<T, M, 4, 4>(__VA_ARGS__);             \
+    case 3: return FN<T, M, 4, 6>(__VA_ARGS__);             \
     case 4: return FN<T, M, 8, 4>(__VA_ARGS__);             \
     case 5: return FN<T, M, 32, 2>(__VA_ARGS__);            \
     case 6: return FN<T, M, 32, 4>(__VA_ARGS__);            \
