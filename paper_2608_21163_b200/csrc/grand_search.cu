@@ -68,7 +68,7 @@ template <typename T, int METRIC, int G, int CPL>
 __global__ void __launch_bounds__(kSearchWarps * 32) beam_search_kernel(const SearchArgs a, const uint32_t per_warp_bytes) {
   using Dist = typename Elem<T>::Dist;
   constexpr int NT = 32 / G;                                   // teams per warp
-  constexpr int U = CPL == 1 ? 4 : (CPL == 2 ? 2 : 1);         // vectors in flight per team
+  constexpr int U = CPL == 1 ? 4 : ((CPL == 2 || G == 32) ? 2 : 1);  // vectors in flight per team
   constexpr unsigned FULL = 0xFFFFFFFFu;
   extern __shared__ __align__(16) unsigned char smem_raw[];
 
