@@ -41,7 +41,7 @@ typedef enum {
   GRAND_ERR_DUPLICATE_ID = -3, /* the same id twice in one batch */
   GRAND_ERR_ALREADY_LIVE = -4, /* insert of a live id */
   GRAND_ERR_NOT_LIVE = -5,     /* delete of an id that is not live */
-  GRAND_ERR_UNSUPPORTED = -6,  /* Vamana mode with the IP metric (alpha-pruning needs a metric) */
+  GRAND_ERR_UNSUPPORTED = -6,  /* Vamana mode with the IP metric and no mips_max_norm (alpha-pruning needs a metric) */
   GRAND_ERR_CUDA = -7,         /* a CUDA call failed; text in grand_last_error */
   GRAND_ERR_LIMIT = -8,        /* a bounded device loop hit its bound */
   GRAND_ERR_NOMEM = -9         /* device allocation failed */
@@ -65,7 +65,10 @@ typedef struct {
   uint32_t hash_bits; /* log2 of the per-query visited cache in 4-byte words; default 10; 8..13, and 4 << hash_bits >= padded row bytes */
   uint32_t full_transpose; /* 1: every delete batch builds the whole reverse graph; default 0: only the rows of the
                               batch's nodes (the only rows the repair reads; identical result) */
-  uint32_t reserved_;
+  float mips_max_norm;     /* > 0: Vamana mode accepts the IP metric on fp32 vectors through the MIPS -> L2
+                              reduction of Sec. 5.3, x -> [x, sqrt(M^2 - |x|^2)] with M = this bound on every base
+                              vector's norm (an insert with a larger norm fails with GRAND_ERR_INVALID_ARG);
+                              searches still return negated inner products */
   /* device allocator hooks (default cudaMalloc / cudaFree); lets a host runtime pool the memory */
   void* (*dev_alloc)(size_t bytes, void* user);
   void (*dev_free)(void* ptr, void* user);

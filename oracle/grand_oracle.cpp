@@ -59,7 +59,10 @@ struct Stats {
 };
 
 struct Index {
-  uint32_t dim, dtype, metric, R, L;
+  uint32_t dim, dtype, metric, R, L;  // dim / metric as used internally (see `augment`)
+  uint32_t udim = 0;                  // dimension of the caller's vectors
+  bool augment = false;               // MIPS -> L2 reduction (Sec. 5.3): x -> [x, sqrt(M^2 - |x|^2)], q -> [q, 0]
+  double M2 = 0.0;                    // M^2, M = bound on the base vectors' norms
   float alpha;
   int64_t A_fix;  // round(alpha * 65536): fixed-point alpha for integer vectors
   uint64_t cap;
@@ -127,6 +130,22 @@ double dist_raw(const Index& ix, const void* a, const void* b) {
     else acc -= xv * yv;
   }
   return (double)acc;
+}
+
+// Store one caller vector as an internal row.  With the MIPS->L2 reduction the extra coordinate is
+// sqrt(M^2 - |x|^2) for base vectors and 0 for queries; squared L2 between such rows orders candidates
+// exactly like the negated inner product does.
+void to_row(const Index& ix, const void* src, void* dst, bool is_query) {
+  std::memcpy(dst, src, (size_t)ix.udim * ix.esize);
+  if (!ix.augment) return;
+  double n2 = 0.0;
+  for (uint32_t j = 0; j < ix.udim; ++j) n2 += (double)((const float*)src)[j] * (double)((const float*)src)[j];
+  ((float*)dst)[ix.udim] = is_query ? 0.0f : (float)std::sqrt(std::max(ix.M2 - n2, 0.0));
+}
+double sq_norm(const Index& ix, const void* v) {
+  double n2 = 0.0;
+  for (uint32_t j = 0; j < ix.udim; ++j) n2 += (double)((const float*)v)[j] * (double)((const float*)v)[j];
+  return n2;
 }
 
 // alpha test of GrANDRobustPrune (Alg. 4): alpha * dist(p*,p') <= D_p[p'].
@@ -379,9 +398,12 @@ int insert_batch(Index& ix, const uint32_t* ids, const void* vecs, uint64_t n) {
   if (n == 0) return OK;
   int rc = validate_insert(ix, ids, n);
   if (rc != OK) return rc;
-  const size_t rb = (size_t)ix.dim * ix.esize;
+  const size_t rb = (size_t)ix.dim * ix.esize, urb = (size_t)ix.udim * ix.esize;
+  if (ix.augment)
+    for (uint64_t i = 0; i < n; ++i)
+      if (sq_norm(ix, (const uint8_t*)vecs + i * urb) > ix.M2 * (1.0 + 1e-6)) return ERR_INVALID_ARG;  // norm above the stated bound
   for (uint64_t i = 0; i < n; ++i) {  // write vector, deg <- 0 (Alg. 5 first loop)
-    std::memcpy(ix.store.data() + (size_t)ids[i] * rb, (const uint8_t*)vecs + i * rb, rb);
+    to_row(ix, (const uint8_t*)vecs + i * urb, ix.store.data() + (size_t)ids[i] * rb, false);
     ix.deg[ids[i]] = 0;
   }
   const bool bootstrap = ix.nlive == 0;
@@ -600,10 +622,18 @@ extern "C" {
 
 int grand_oracle_create(uint32_t dim, uint32_t dtype, uint32_t metric, uint32_t R, uint32_t L, float alpha,
                         uint64_t capacity, uint32_t P, uint32_t c, uint32_t k_repair, uint32_t vmax,
-                        uint32_t mode, uint32_t nthreads, void** out) {
+                        uint32_t mode, uint32_t nthreads, float max_norm, void** out) {
   if (!out || dim == 0 || R == 0 || L == 0 || dtype > 2 || metric > 1 || mode > 1 || capacity == 0) return ERR_INVALID_ARG;
-  if (mode == MODE_VAMANA && metric == M_IP) return ERR_UNSUPPORTED;
+  const bool augment = mode == MODE_VAMANA && metric == M_IP && max_norm > 0.0f && dtype == DT_F32;
+  if (mode == MODE_VAMANA && metric == M_IP && !augment) return ERR_UNSUPPORTED;
   Index* ix = new Index();
+  ix->udim = dim;
+  ix->augment = augment;
+  ix->M2 = (double)max_norm * (double)max_norm;
+  if (augment) {
+    dim += 1;
+    metric = M_L2;
+  }
   ix->dim = dim; ix->dtype = dtype; ix->metric = metric; ix->R = R; ix->L = L; ix->alpha = alpha;
   ix->A_fix = std::llround((double)alpha * 65536.0);
   ix->cap = capacity;
@@ -634,14 +664,20 @@ int grand_oracle_search(void* h, const void* queries, uint64_t nq, uint32_t k, u
                         uint32_t* out_ids, double* out_dists) {
   Index& ix = *(Index*)h;
   if (k == 0 || k > L) return ERR_INVALID_ARG;
-  const size_t rb = (size_t)ix.dim * ix.esize;
+  const size_t urb = (size_t)ix.udim * ix.esize;
   parallel_for(ix, nq, [&](size_t i) {
     std::vector<BeamEntry> C;
     std::vector<Key> V;
-    greedy_search(ix, ix.entry, (const uint8_t*)queries + i * rb, L, 2 * L, use_seen_set != 0, C, V, &ix.st);
+    std::vector<uint8_t> qrow((size_t)ix.dim * ix.esize);
+    const uint8_t* qsrc = (const uint8_t*)queries + i * urb;
+    to_row(ix, qsrc, qrow.data(), true);
+    greedy_search(ix, ix.entry, qrow.data(), L, 2 * L, use_seen_set != 0, C, V, &ix.st);
+    const double qn = ix.augment ? sq_norm(ix, qsrc) : 0.0;
     for (uint32_t j = 0; j < k; ++j) {
       out_ids[i * k + j] = j < C.size() ? C[j].k.id : INVALID;
-      out_dists[i * k + j] = j < C.size() ? C[j].k.d : std::numeric_limits<double>::infinity();
+      double d = j < C.size() ? C[j].k.d : std::numeric_limits<double>::infinity();
+      if (ix.augment && j < C.size()) d = (d - qn - ix.M2) * 0.5;  // back to the negated inner product
+      out_dists[i * k + j] = d;
     }
   });
   return OK;
@@ -654,7 +690,9 @@ int grand_oracle_greedy(void* h, const void* q, uint32_t L, uint32_t vmax, uint3
   Index& ix = *(Index*)h;
   std::vector<BeamEntry> C;
   std::vector<Key> V;
-  greedy_search(ix, ix.entry, q, L, vmax, use_seen_set != 0, C, V, &ix.st);
+  std::vector<uint8_t> qrow((size_t)ix.dim * ix.esize);
+  to_row(ix, q, qrow.data(), true);
+  greedy_search(ix, ix.entry, qrow.data(), L, vmax, use_seen_set != 0, C, V, &ix.st);
   for (size_t i = 0; i < C.size(); ++i) {
     beam_ids[i] = C[i].k.id;
     beam_d[i] = C[i].k.d;
@@ -707,7 +745,8 @@ int grand_oracle_import_graph(void* h, const uint32_t* adj, const uint32_t* deg,
     ix.nlive += ix.live[v];
   }
   ix.entry = entry;
-  std::memcpy(ix.store.data(), vecs, ix.store.size());
+  for (uint64_t v = 0; v < ix.cap; ++v)
+    to_row(ix, (const uint8_t*)vecs + v * ix.udim * ix.esize, ix.store.data() + v * ix.dim * ix.esize, false);
   return OK;
 }
 

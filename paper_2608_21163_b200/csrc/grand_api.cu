@@ -20,7 +20,7 @@ unsigned long long launches_so_far() { return g_launches.load(); }
 
 Layout make_layout(uint32_t dim, uint32_t dtype, uint32_t metric) {
   Layout l{};
-  l.dim = dim; l.dtype = dtype; l.metric = metric;
+  l.dim = dim; l.udim = dim; l.dtype = dtype; l.metric = metric;
   l.esize = dtype == GRAND_F32 ? 4 : 1;
   l.row_bytes = (uint32_t)(((uint64_t)dim * l.esize + 15) / 16 * 16);
   l.nchunk = l.row_bytes / 16;
@@ -47,6 +47,8 @@ struct Buf {
 struct grand_index {
   Layout lay;
   uint32_t R, L, P, c, k_repair, vmax, mode, hash_bits, full_transpose;
+  bool mips = false;   // MIPS -> L2 reduction active (Vamana mode, IP metric, fp32)
+  double mips_M2 = 0.0;
   float alpha;
   long long A_fix;
   uint64_t cap, max_batch;
@@ -202,6 +204,8 @@ SearchArgs search_args(grand_index* idx, cudaStream_t s) {
   a.g = view(idx);
   a.entry = idx->entry;
   a.hash_bits = idx->hash_bits;
+  a.mips = idx->mips ? 1u : 0u;
+  a.mips_M2 = (float)idx->mips_M2;
   a.state = idx->d_state;
   return a;
 }
@@ -249,8 +253,11 @@ int grand_create_ex(uint32_t dim, uint32_t dtype, uint32_t metric, uint32_t R, u
   if (dim == 0 || dtype > GRAND_F32 || metric > GRAND_IP || R == 0 || R > GRAND_MAX_R || L == 0 || L > GRAND_MAX_L ||
       o->mode > GRAND_MODE_FIXED_DEGREE || !(alpha >= 1.0f))
     return GRAND_ERR_INVALID_ARG;
-  if (o->mode == GRAND_MODE_VAMANA && metric == GRAND_IP) return GRAND_ERR_UNSUPPORTED;
-  Layout lay = make_layout(dim, dtype, metric);
+  const bool mips = o->mode == GRAND_MODE_VAMANA && metric == GRAND_IP && o->mips_max_norm > 0.0f && dtype == GRAND_F32;
+  if (o->mode == GRAND_MODE_VAMANA && metric == GRAND_IP && !mips) return GRAND_ERR_UNSUPPORTED;
+  // MIPS -> L2 reduction: rows carry one extra coordinate and the index works on squared L2
+  Layout lay = mips ? make_layout(dim + 1, dtype, GRAND_L2) : make_layout(dim, dtype, metric);
+  lay.udim = dim;
   if (lay.code < 0 || lay.row_bytes > GRAND_MAX_ROW_BYTES) return GRAND_ERR_INVALID_ARG;
   grand_index* idx = new grand_index();
   idx->lay = lay;
@@ -265,6 +272,8 @@ int grand_create_ex(uint32_t dim, uint32_t dtype, uint32_t metric, uint32_t R, u
   idx->mode = o->mode;
   idx->hash_bits = o->hash_bits ? o->hash_bits : 10;
   idx->full_transpose = o->full_transpose;
+  idx->mips = mips;
+  idx->mips_M2 = (double)o->mips_max_norm * (double)o->mips_max_norm;
   idx->dev_alloc = o->dev_alloc ? o->dev_alloc : default_alloc;
   idx->dev_free = o->dev_free ? o->dev_free : default_free;
   idx->user = o->user;
@@ -346,6 +355,7 @@ int grand_insert_batch(grand_index* idx, const uint32_t* ids, const void* vecs, 
   {
     PhaseTimer pt(idx, s, PH_OTHER);
     CK(launch_validate(ids, n, idx->cap, idx->live, idx->mark, 0, idx->d_state, s));
+    if (idx->mips) CK(launch_check_norms(idx->lay, vecs, n, idx->mips_M2, idx->d_state, s));
   }
   if ((rc = read_state(idx, s))) return rc;
   if (idx->h_state->status != 0) {
@@ -359,6 +369,7 @@ int grand_insert_batch(grand_index* idx, const uint32_t* ids, const void* vecs, 
   {
     PhaseTimer pt(idx, s, PH_OTHER);
     CK(launch_store_write(idx->lay, idx->store, idx->deg, idx->slot_of, ids, vecs, n, s));
+    if (idx->mips) CK(launch_augment_rows(idx->lay, idx->store, ids, n, idx->mips_M2, s));
   }
   const bool bootstrap = idx->nlive == 0;
   {
@@ -565,7 +576,7 @@ int grand_insert_batch_host(grand_index* idx, const uint32_t* ids, const void* v
   if (n == 0) return GRAND_OK;
   cudaStream_t s = (cudaStream_t)stream;
   int rc;
-  const size_t vb = (size_t)n * idx->lay.dim * idx->lay.esize;
+  const size_t vb = (size_t)n * idx->lay.udim * idx->lay.esize;
   if ((rc = ensure(idx, idx->st_ids, n * 4, s))) return rc;
   if ((rc = ensure(idx, idx->st_vecs, vb, s))) return rc;
   CK(cudaMemcpyAsync(idx->st_ids.p, ids, n * 4, cudaMemcpyHostToDevice, s));
@@ -587,7 +598,7 @@ int grand_search_host(grand_index* idx, const void* queries, uint64_t nq, uint32
   if (nq == 0) return GRAND_OK;
   cudaStream_t s = (cudaStream_t)stream;
   int rc;
-  const size_t qb = (size_t)nq * idx->lay.dim * idx->lay.esize;
+  const size_t qb = (size_t)nq * idx->lay.udim * idx->lay.esize;
   if ((rc = ensure(idx, idx->st_vecs, qb, s))) return rc;
   if ((rc = ensure(idx, idx->st_out_ids, nq * k * 4, s))) return rc;
   if ((rc = ensure(idx, idx->st_out_d, nq * k * 4, s))) return rc;
@@ -617,6 +628,7 @@ int grand_import_graph(grand_index* idx, const uint32_t* adj, const uint32_t* de
   CK(cudaMemcpyAsync(idx->deg, deg, idx->cap * 4, cudaMemcpyDeviceToDevice, s));
   CK(cudaMemcpyAsync(idx->live, live, (idx->cap + 31) / 32 * 4, cudaMemcpyDeviceToDevice, s));
   CK(launch_pad_rows(idx->lay, idx->store, vecs, idx->cap, s));
+  if (idx->mips) CK(launch_augment_rows(idx->lay, idx->store, nullptr, idx->cap, idx->mips_M2, s));
   CK(cudaMemsetAsync(idx->rowpfx, 0, idx->cap, s));
   if (idx->rowd) CK(cudaMemsetAsync(idx->rowd, 0xFF, (size_t)idx->cap * idx->R * 4, s));
   CK(launch_pad_adjacency(idx->adj, idx->deg, idx->cap, idx->R, s));

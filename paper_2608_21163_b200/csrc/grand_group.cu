@@ -275,14 +275,46 @@ cudaError_t launch_store_write(const Layout& lay, uint8_t* store, uint32_t* deg,
   if (n == 0) return cudaSuccess;
   const uint64_t total = n * (lay.row_bytes / lay.esize);
   if (lay.esize == 4)
-    store_write_kernel<float><<<grid_for(total), kThreads, 0, s>>>(store, deg, slot_of, ids, (const float*)vecs, n, lay.dim, lay.row_bytes);
+    store_write_kernel<float><<<grid_for(total), kThreads, 0, s>>>(store, deg, slot_of, ids, (const float*)vecs, n, lay.udim, lay.row_bytes);
   else
-    store_write_kernel<uint8_t><<<grid_for(total), kThreads, 0, s>>>(store, deg, slot_of, ids, (const uint8_t*)vecs, n, lay.dim, lay.row_bytes);
+    store_write_kernel<uint8_t><<<grid_for(total), kThreads, 0, s>>>(store, deg, slot_of, ids, (const uint8_t*)vecs, n, lay.udim, lay.row_bytes);
   count_launches(1);
   return cudaGetLastError();
 }
 cudaError_t launch_pad_rows(const Layout& lay, uint8_t* store, const void* vecs, uint64_t n, cudaStream_t s) {
   return launch_store_write(lay, store, nullptr, nullptr, nullptr, vecs, n, s);
+}
+
+// ---- MIPS -> L2 reduction (Sec. 5.3): one warp per vector sums the squares in double
+__device__ __forceinline__ double warp_sq_norm(const float* v, uint32_t d) {
+  double s = 0.0;
+  for (uint32_t j = threadIdx.x & 31; j < d; j += 32) s += (double)v[j] * (double)v[j];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
+  return s;
+}
+__global__ void check_norms_kernel(const float* vecs, uint64_t n, uint32_t udim, double M2, DevState* st) {
+  const uint64_t w = (blockIdx.x * (uint64_t)blockDim.x + threadIdx.x) >> 5, nw = ((uint64_t)gridDim.x * blockDim.x) >> 5;
+  for (uint64_t i = w; i < n; i += nw)
+    if (warp_sq_norm(vecs + i * udim, udim) > M2 * (1.0 + 1e-6) && (threadIdx.x & 31) == 0) atomicMin(&st->status, -1);
+}
+__global__ void augment_rows_kernel(uint8_t* store, const uint32_t* ids, uint64_t n, uint32_t udim, uint32_t row_bytes, double M2) {
+  const uint64_t w = (blockIdx.x * (uint64_t)blockDim.x + threadIdx.x) >> 5, nw = ((uint64_t)gridDim.x * blockDim.x) >> 5;
+  for (uint64_t i = w; i < n; i += nw) {
+    float* row = reinterpret_cast<float*>(store + (size_t)(ids ? ids[i] : i) * row_bytes);
+    const double n2 = warp_sq_norm(row, udim);
+    if ((threadIdx.x & 31) == 0) row[udim] = (float)sqrt(fmax(M2 - n2, 0.0));
+  }
+}
+cudaError_t launch_check_norms(const Layout& lay, const void* vecs, uint64_t n, double M2, DevState* st, cudaStream_t s) {
+  check_norms_kernel<<<grid_for(n * 32), kThreads, 0, s>>>((const float*)vecs, n, lay.udim, M2, st);
+  count_launches(1);
+  return cudaGetLastError();
+}
+cudaError_t launch_augment_rows(const Layout& lay, uint8_t* store, const uint32_t* ids, uint64_t n, double M2, cudaStream_t s) {
+  augment_rows_kernel<<<grid_for(n * 32), kThreads, 0, s>>>(store, ids, n, lay.udim, lay.row_bytes, M2);
+  count_launches(1);
+  return cudaGetLastError();
 }
 
 // ---- publish (insert epilogue): live bits on, batch marks off

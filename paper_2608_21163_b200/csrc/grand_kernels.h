@@ -14,7 +14,8 @@ unsigned long long launches_so_far();
 // Row layout shared by every distance kernel: a padded row has nchunk 16-byte chunks; a team of G
 // lanes covers it with CPL chunks per lane.  layout_code selects the (G, CPL) instantiation.
 struct Layout {
-  uint32_t dim, dtype, metric;
+  uint32_t dim, dtype, metric;  // as stored (dim includes the extra coordinate of the MIPS -> L2 reduction)
+  uint32_t udim;                // dimension of the caller's vectors and queries
   uint32_t esize, row_bytes, nchunk;
   int code;  // index into the (G, CPL) table, -1 = unsupported
   int G, CPL;
@@ -68,6 +69,8 @@ struct SearchArgs {
   uint32_t boot_n;
   uint32_t hash_bits;
   uint32_t* work_ctr;  // zeroed by the caller before the launch; nullptr = static striding
+  uint32_t mips;       // 1: rows are MIPS -> L2 augmented; reported distances go back to negated inner products
+  float mips_M2;       // M^2 of that reduction
   DevState* state;
 };
 cudaError_t launch_beam_search(const SearchArgs& a, cudaStream_t s);
@@ -193,6 +196,9 @@ cudaError_t launch_pick_medoid(const Layout& lay, const GraphView& g, const uint
                                DevState* st, cudaStream_t s);
 cudaError_t launch_count_live(const uint32_t* live, uint64_t cap, DevState* st, cudaStream_t s);
 cudaError_t launch_pad_rows(const Layout& lay, uint8_t* store, const void* vecs, uint64_t n, cudaStream_t s);
+// MIPS -> L2 reduction: norm check of a batch (status -1 above the bound) and the extra coordinate of stored rows
+cudaError_t launch_check_norms(const Layout& lay, const void* vecs, uint64_t n, double M2, DevState* st, cudaStream_t s);
+cudaError_t launch_augment_rows(const Layout& lay, uint8_t* store, const uint32_t* ids, uint64_t n, double M2, cudaStream_t s);
 cudaError_t launch_pad_adjacency(uint32_t* adj, const uint32_t* deg, uint64_t cap, uint32_t R, cudaStream_t s);
 cudaError_t launch_fill_u32(uint32_t* p, uint32_t v, uint64_t n, cudaStream_t s);
 

@@ -114,9 +114,9 @@ __global__ void __launch_bounds__(kSearchWarps * 32) beam_search_kernel(const Se
       load_row<G, CPL>(store + (size_t)self * row_bytes, nchunk, t, q);
     } else {
       T* stage = reinterpret_cast<T*>(hash);
-      const T* src = reinterpret_cast<const T*>(a.queries) + qi * a.lay.dim;
+      const T* src = reinterpret_cast<const T*>(a.queries) + qi * a.lay.udim;
       const uint32_t npad = row_bytes / sizeof(T);
-      for (uint32_t j = lane; j < npad; j += 32) stage[j] = j < a.lay.dim ? src[j] : T(0);
+      for (uint32_t j = lane; j < npad; j += 32) stage[j] = j < a.lay.udim ? src[j] : T(0);  // extra coordinate of a query: 0
       __syncwarp();
 #pragma unroll
       for (int c = 0; c < CPL; ++c) {
@@ -320,6 +320,17 @@ __global__ void __launch_bounds__(kSearchWarps * 32) beam_search_kernel(const Se
     }
 
     // ---- outputs
+    float qn = 0.0f;  // |q|^2, needed to turn augmented L2 back into a negated inner product
+    if constexpr (sizeof(T) == 4) {
+      if (a.mips && a.out_dists) {
+#pragma unroll
+        for (int c = 0; c < CPL; ++c) {
+          const float* qf = reinterpret_cast<const float*>(&q[c]);
+          qn = fmaf(qf[0], qf[0], fmaf(qf[1], qf[1], fmaf(qf[2], qf[2], fmaf(qf[3], qf[3], qn))));
+        }
+        qn = team_sum<G>(qn);
+      }
+    }
     if (a.out_ids) {
       for (uint32_t j = lane; j < a.k; j += 32) {
         const bool have = j < beam_n;
@@ -327,7 +338,9 @@ __global__ void __launch_bounds__(kSearchWarps * 32) beam_search_kernel(const Se
         a.out_ids[qi * a.k + j] = have ? key_id(key) : kInvalid;
         if (a.out_dists) {
           if constexpr (sizeof(T) == 4) {
-            reinterpret_cast<float*>(a.out_dists)[qi * a.k + j] = have ? key_dist<float>(key) : __int_as_float(0x7f800000);
+            float dv = have ? key_dist<float>(key) : __int_as_float(0x7f800000);
+            if (a.mips && have) dv = (dv - qn - a.mips_M2) * 0.5f;
+            reinterpret_cast<float*>(a.out_dists)[qi * a.k + j] = dv;
           } else {
             reinterpret_cast<int*>(a.out_dists)[qi * a.k + j] = have ? key_dist<int>(key) : 0x7fffffff;
           }

@@ -370,3 +370,45 @@ def test_small_degree_bound_and_alpha_one():
         assert_same_graph(o, g, f"delete {r}")
         o.insert_batch(dele[:250], base[dele[:250]]); g.insert_batch(torch.from_numpy(dele[:250]), torch.from_numpy(base[dele[:250]]))
         assert_same_graph(o, g, f"reinsert {r}")
+
+
+def test_mips_reduction_vamana_ip_matches_oracle():
+    """Vamana mode on the IP metric through the MIPS -> L2 reduction (Sec. 5.3): fp32, so the comparison is
+    recall against brute-force maximum inner product (within 0.005 of the oracle's), negated inner products
+    within 1e-5 of a float64 recomputation, and the graph invariants; a norm above the bound is refused."""
+    torch = torch_()
+    from paper_2608_21163_b200 import binding as gb
+    n, d, R, L = 6000, 48, 24, 64
+    scale = np.linspace(0.4, 1.0, n, dtype=np.float32)[:, None]
+    base = (synth.aniso_unit_f32(5, "base", 0, n, d) * scale).astype(np.float32)
+    q = synth.aniso_unit_f32(5, "query", 0, 300, d)
+    o = go.Oracle(d, go.F32, go.IP, R, L, 1.2, n, max_norm=1.0)
+    g = gb.GrandIndex(d, gb.F32, gb.IP, R, L, 1.2, capacity=n, max_batch=1000, mips_max_norm=1.0)
+    for lo in range(0, n, 750):
+        ids = np.arange(lo, lo + 750, dtype=np.uint32)
+        o.insert_batch(ids, base[ids]); g.insert_batch(torch.from_numpy(ids), torch.from_numpy(base[ids]))
+    dele = synth.choose_ids(5, "del", np.arange(n, dtype=np.uint32), 600)
+    o.delete_batch(dele); g.delete_batch(torch.from_numpy(dele))
+    adj, deg, live, entry = gpu_graph(g)
+    mask = go.live_mask(live, n)
+    assert mask.sum() == n - 600 == g.live_count and (deg <= R).all() and (deg[~mask] == 0).all() and mask[entry]
+    for v in np.flatnonzero(mask)[:1500]:
+        r = adj[v, :deg[v]]
+        assert mask[r].all() and v not in r and len(set(r.tolist())) == len(r)
+    live_ids = np.flatnonzero(mask).astype(np.uint32)
+    truth = brute_force_topk(base, live_ids, q, 10, go.IP)
+    oi, od = o.search(q, 10, L)
+    gi, gd = gpu_search(g, q, 10, L)
+    r_o, r_g = recall_at_k(oi, truth), recall_at_k(gi, truth)
+    assert abs(r_o - r_g) <= 0.005 and r_g > 0.85, (r_o, r_g)
+    for i in range(len(q)):
+        b = base[gi[i]].astype(np.float64)
+        exact = -(b @ q[i].astype(np.float64))
+        assert (np.abs(gd[i] - exact) <= 1e-5 * np.linalg.norm(b, axis=1) * np.linalg.norm(q[i]) + 2e-6).all()
+        assert (np.diff(gd[i]) >= -1e-6).all()
+    with pytest.raises(gb.GrandError) as e:
+        g.insert_batch(torch.from_numpy(dele[:2]), torch.from_numpy((base[:2] * 9).astype(np.float32)))
+    assert e.value.code == -1
+    g.insert_batch(torch.from_numpy(dele[:2]), torch.from_numpy(base[dele[:2]]))   # the index is still usable
+    with pytest.raises(gb.GrandError):
+        gb.GrandIndex(d, gb.U8, gb.IP, R, L, 1.2, capacity=n, mips_max_norm=1.0)  # fp32 only

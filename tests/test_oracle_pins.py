@@ -507,3 +507,58 @@ def test_recall_sanity_band_tiny():
         bi, _ = brute_knn(base, live, q[i], 10)
         hit += len(set(bi.tolist()) & set(ids[i].tolist()))
     assert hit / (10 * len(q)) > 0.9
+
+
+# ------------------------------------------------------------------ MIPS -> L2 reduction (Sec. 5.3)
+def test_mips_reduction_orders_like_inner_product():
+    """x -> [x, sqrt(M^2 - |x|^2)], q -> [q, 0]: |q' - x'|^2 = |q|^2 + M^2 - 2 q.x, so a complete-graph
+    search in Vamana mode with the IP metric must return the brute-force maximum-inner-product set,
+    with the negated inner products as distances."""
+    rng = np.random.default_rng(8)
+    n, d = 50, 7
+    base = rng.standard_normal((n, d)).astype(np.float32)
+    M = float(np.linalg.norm(base, axis=1).max()) * 1.001
+    o = go.Oracle(d, go.F32, go.IP, n - 1, 16, 1.2, n, max_norm=M, nthreads=2)
+    o.insert_batch(np.arange(n, dtype=np.uint32), base)          # bootstrap batch
+    adj = np.array([[w for w in range(n) if w != v] for v in range(n)], np.uint32)
+    o.import_graph(adj, np.full(n, n - 1, np.uint32), go.pack_bitmap(np.ones(n, bool)), 3, base)
+    q = rng.standard_normal((20, d)).astype(np.float32)
+    ids, dist = o.search(q, 5, 16)
+    for i in range(len(q)):
+        ip = -(base.astype(np.float64) @ q[i].astype(np.float64))
+        want = np.lexsort((np.arange(n), ip))[:5]
+        assert (ids[i] == want).all()
+        assert np.allclose(dist[i], ip[want], rtol=0, atol=2e-6 * (M * M + (q[i] ** 2).sum()))
+    # closed form of one augmented distance: query [x, 0] against stored row [y, sqrt(M^2 - |y|^2)]
+    x, y = base[0].astype(np.float64), base[1].astype(np.float64)
+    ey = float(np.float32(np.sqrt(M * M - y @ y)))          # the stored extra coordinate is a float
+    want = ((x - y) ** 2).sum() + ey ** 2
+    (bi, bd), _ = o.greedy(base[0], n, n)
+    assert abs(bd[list(bi).index(1)] - want) <= 2e-7 * want
+    with pytest.raises(go.OracleError):
+        o.insert_batch([0], base[:1])             # already live
+    o.delete_batch([0])
+    with pytest.raises(go.OracleError) as e:
+        o.insert_batch([0], (base[:1] * 50).astype(np.float32))   # norm above the stated bound
+    assert e.value.code == -1
+    with pytest.raises(go.OracleError):
+        go.Oracle(d, go.U8, go.IP, 4, 8, 1.2, 16, max_norm=10.0)  # the reduction is defined for fp32 only
+
+
+def test_mips_vamana_stream_invariants_and_recall():
+    n, d = 3000, 24
+    base = synth.aniso_unit_f32(3, "base", 0, n, d) * np.linspace(0.5, 1.0, n, dtype=np.float32)[:, None]
+    o = go.Oracle(d, go.F32, go.IP, 16, 48, 1.2, n, max_norm=1.0)
+    for lo in range(0, n, 500):
+        o.insert_batch(np.arange(lo, lo + 500, dtype=np.uint32), base[lo:lo + 500])
+    dele = synth.choose_ids(3, "del", np.arange(n, dtype=np.uint32), 300)
+    o.delete_batch(dele)
+    adj, deg, mask, entry = check_invariants(o, n - 300)
+    live = np.setdiff1d(np.arange(n, dtype=np.uint32), dele)
+    q = synth.aniso_unit_f32(3, "query", 0, 100, d)
+    ids, _ = o.search(q, 10, 48)
+    hit = 0
+    for i in range(len(q)):
+        bi, _ = brute_knn(base, live, q[i], 10, metric=go.IP)
+        hit += len(set(bi.tolist()) & set(ids[i].tolist()))
+    assert hit / (10 * len(q)) > 0.85
