@@ -155,6 +155,8 @@ def main():
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--workload", default=WORKLOAD, choices=sorted(synth.CONFIGS), help="default: the bench workload; the other "
                     "configs are exploration runs (their lines carry their own workload name)")
+    ap.add_argument("--pattern", default="", choices=["", "sliding_window", "interleaved", "expiration_time", "clustered", "insert_heavy"],
+                    help="run one of the paper's streaming patterns (Sec. 5.2) on the SIFT-shaped data instead of the step loop")
     ap.add_argument("--hash-bits", type=int, default=0, help="log2 size of the per-query visited cache (0 = library default)")
     ap.add_argument("--search-only", type=int, default=0, help="after the build run this many search launches and exit")
     args = ap.parse_args()
@@ -189,6 +191,8 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
     torch.backends.cuda.matmul.allow_tf32 = False
 
+    if args.pattern:
+        return run_pattern(args, torch, gb, dev)
     cfg = dict(synth.CONFIGS[args.workload])
     is_f32 = cfg["dtype"] == synth.F32
     dist_dtype = torch.float32 if is_f32 else torch.int32
@@ -382,6 +386,67 @@ def main():
     if dist:
         dist.destroy_process_group()
     return 0
+
+
+def run_pattern(args, torch, gb, dev):
+    """One of the streaming patterns of Sec. 5.2 over SIFT-shaped rows (1M x scale), batches of 10k x scale.
+    Every op is timed with CUDA events; the first `warmup` ops are excluded."""
+    cfg = dict(synth.CONFIGS["sift_u8_d128"])
+    n = max(2000, int(round(cfg["n"] * args.scale)))
+    batch = max(100, int(round(10_000 * args.scale)))
+    wl = synth.Workload(cfg, 0)
+    base = torch.from_numpy(wl.vectors(0, n)).to(dev)
+    queries = torch.from_numpy(synth.mixture_u8(0, "query", 0, batch, cfg["dim"])).to(dev)
+    gens = {
+        "sliding_window": lambda: synth.pattern_sliding_window(n, 100, 50, batch),
+        "interleaved": lambda: synth.pattern_interleaved(n, batch, n_ops=100),
+        "expiration_time": lambda: synth.pattern_expiration(n, batch),
+        "clustered": lambda: synth.pattern_clustered(n, batch, synth.mixture_centre_of(0, "base", 0, n) % 64),
+        "insert_heavy": lambda: synth.pattern_insert_heavy(n, batch),
+    }
+    g = gb.GrandIndex(cfg["dim"], cfg["dtype"], cfg["metric"], cfg["R"], cfg["L"], cfg["alpha"], capacity=n, max_batch=batch)
+    out_i = torch.empty((batch, 10), dtype=torch.uint32, device=dev)
+    out_d = torch.empty((batch, 10), dtype=torch.int32, device=dev)
+    t = {"insert": 0.0, "delete": 0.0, "search": 0.0}
+    cnt = {"insert": 0, "delete": 0, "search": 0}
+    launches0 = None
+    nop = 0
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    for op in gens[args.pattern]():
+        ids = torch.from_numpy(op[1]).to(dev) if len(op) > 1 else None
+        a, b = ev(), ev()
+        torch.cuda.synchronize()
+        a.record()
+        if op[0] == "insert":
+            g.insert_batch(ids, base[ids.view(torch.int32).long()] if not _contiguous(op[1]) else base[int(op[1][0]):int(op[1][0]) + len(op[1])])
+        elif op[0] == "delete":
+            g.delete_batch(ids)
+        else:
+            g.search(queries, 10, cfg["L"], out_i, out_d)
+        b.record()
+        torch.cuda.synchronize()
+        nop += 1
+        if nop == args.warmup:
+            launches0 = g.stats()["kernel_launches"]
+        if nop > args.warmup:
+            t[op[0]] += a.elapsed_time(b)
+            cnt[op[0]] += len(op[1]) if len(op) > 1 else batch
+    upd = cnt["insert"] + cnt["delete"]
+    line = {"metric": METRIC, "value": upd / ((t["insert"] + t["delete"]) * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": nop - args.warmup,
+            "warmup": args.warmup, "ms_per_step": sum(t.values()) / max(nop - args.warmup, 1), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
+            "config": {"workload": f"sift_u8_d128/{args.pattern}", "rows": n, "batch": batch, "R": cfg["R"], "L": cfg["L"],
+                       "step": "one op of the pattern's stream"},
+            "insert_vectors_per_sec": cnt["insert"] / (t["insert"] * 1e-3) if t["insert"] else None,
+            "delete_vectors_per_sec": cnt["delete"] / (t["delete"] * 1e-3) if t["delete"] else None,
+            "search_qps": cnt["search"] / (t["search"] * 1e-3) if t["search"] else None,
+            "live_at_end": g.live_count, "gpu_launches": g.stats()["kernel_launches"] - (launches0 or 0)}
+    print(json.dumps(line))
+    return 0
+
+
+def _contiguous(ids):
+    return len(ids) > 0 and int(ids[-1]) - int(ids[0]) + 1 == len(ids)
 
 
 def brute_topk_gpu(torch, base, live_ids, queries, k, metric=0, is_f32=False):

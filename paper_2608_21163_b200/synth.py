@@ -250,3 +250,104 @@ class StreamState:
 
     def end_round(self):
         self.round += 1
+
+
+# ---------------------------------------------------------------------------------------------
+# Streaming patterns of Sec. 5.2.  Each generator yields ops over a base array of `n_rows` vectors
+# that the caller generates with Workload.vectors(0, n_rows); ids equal row numbers (no id reuse):
+#   ("insert", ids)   ids: uint32 array      ("delete", ids)      ("search",)
+# Sizes are parameters so that the same pattern runs as a shrunk parity case and as a benchmark.
+def mixture_centre_of(seed, stream, start, n, n_centres=1000):
+    """Mixture centre index of rows [start, start+n) of mixture_u8 (same draw as the generator)."""
+    return (hash_u64(seed, stream + "/centre", np.arange(start, start + n, dtype=np.uint64)) % np.uint64(n_centres)).astype(np.int64)
+
+
+def _chunks(ids, batch):
+    for lo in range(0, len(ids), batch):
+        yield ids[lo:lo + batch]
+
+
+def pattern_sliding_window(n_rows, segments=100, active=50, batch=1000):
+    """Sliding Window: the rows are cut into `segments`; `active` of them are live; each step inserts the
+    next segment, deletes the oldest and searches."""
+    seg = n_rows // segments
+    ids = np.arange(n_rows, dtype=np.uint32)
+    for s in range(active):
+        for b in _chunks(ids[s * seg:(s + 1) * seg], batch):
+            yield ("insert", b)
+    for s in range(active, segments):
+        for b in _chunks(ids[s * seg:(s + 1) * seg], batch):
+            yield ("insert", b)
+        for b in _chunks(ids[(s - active) * seg:(s - active + 1) * seg], batch):
+            yield ("delete", b)
+        yield ("search",)
+
+
+def pattern_interleaved(n_rows, batch, seed=0, build_frac=0.3, n_ops=60):
+    """Interleaved: after an initial build, a random sequence of 50% insert / 30% search / 20% delete
+    batches (deletes draw uniformly from the live set)."""
+    ids = np.arange(n_rows, dtype=np.uint32)
+    nxt = int(n_rows * build_frac) // batch * batch
+    for b in _chunks(ids[:nxt], batch):
+        yield ("insert", b)
+    live = np.zeros(n_rows, bool)
+    live[:nxt] = True
+    draw = hash_u64(seed, "interleaved/op", np.arange(n_ops, dtype=np.uint64)) % np.uint64(10)
+    for k in range(n_ops):
+        r = int(draw[k])
+        if r < 5 and nxt + batch <= n_rows:
+            b = ids[nxt:nxt + batch]
+            nxt += batch
+            live[b] = True
+            yield ("insert", b)
+        elif r < 8:
+            yield ("search",)
+        else:
+            lv = np.flatnonzero(live).astype(np.uint32)
+            if len(lv) > 2 * batch:
+                d = choose_ids(seed, f"interleaved/del/{k}", lv, batch)
+                live[d] = False
+                yield ("delete", d)
+
+
+def pattern_expiration(n_rows, batch, seed=0):
+    """Expiration Time: every cycle inserts one batch with a lifetime of 10, 100 or unlimited cycles drawn
+    in the ratio 10:2:1, deletes the batches that expire, then searches."""
+    ids = np.arange(n_rows, dtype=np.uint32)
+    n_cycles = n_rows // batch
+    draw = hash_u64(seed, "expiration/life", np.arange(n_cycles, dtype=np.uint64)) % np.uint64(13)
+    expiry = {}
+    for cyc in range(n_cycles):
+        b = ids[cyc * batch:(cyc + 1) * batch]
+        yield ("insert", b)
+        r = int(draw[cyc])
+        life = 10 if r < 10 else (100 if r < 12 else None)
+        if life is not None:
+            expiry.setdefault(cyc + life, []).append(b)
+        for d in expiry.pop(cyc, []):
+            yield ("delete", d)
+        if cyc % 4 == 3:
+            yield ("search",)
+
+
+def pattern_clustered(n_rows, batch, cluster_of, clusters=64, window=32):
+    """Clustered: rows are grouped into `clusters` (here: by mixture centre); a window of `window` clusters is
+    live; each step inserts the next cluster, deletes the oldest one and searches (deletes hit one region of
+    the graph, which maximises the overlap of dirty sets)."""
+    groups = [np.flatnonzero(cluster_of[:n_rows] == c).astype(np.uint32) for c in range(clusters)]
+    for c in range(clusters):
+        for b in _chunks(groups[c], batch):
+            yield ("insert", b)
+        if c >= window:
+            for b in _chunks(groups[c - window], batch):
+                yield ("delete", b)
+            yield ("search",)
+
+
+def pattern_insert_heavy(n_rows, batch):
+    """Insert Heavy: 90% insert batches, 10% searches, no deletes."""
+    ids = np.arange(n_rows, dtype=np.uint32)
+    for k, b in enumerate(_chunks(ids, batch)):
+        yield ("insert", b)
+        if k % 9 == 8:
+            yield ("search",)
