@@ -158,6 +158,8 @@ def main():
     ap.add_argument("--pattern", default="", choices=["", "sliding_window", "interleaved", "expiration_time", "clustered", "insert_heavy"],
                     help="run one of the paper's streaming patterns (Sec. 5.2) on the SIFT-shaped data instead of the step loop")
     ap.add_argument("--hash-bits", type=int, default=0, help="log2 size of the per-query visited cache (0 = library default)")
+    ap.add_argument("--visited-set-delete", action="store_true",
+                    help="run the delete variant that takes in-neighbours from the visited sets (dangling edges allowed)")
     ap.add_argument("--search-only", type=int, default=0, help="after the build run this many search launches and exit")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
@@ -208,7 +210,8 @@ def main():
     cap = wl.capacity()
     max_batch = max(cfg["first_batch"], cfg["max_build_batch"], cfg["ins"], cfg["dele"])
     g = gb.GrandIndex(cfg["dim"], cfg["dtype"], cfg["metric"], cfg["R"], cfg["L"], cfg["alpha"], capacity=cap,
-                      max_batch=max_batch, mode=cfg["mode"], hash_bits=args.hash_bits)
+                      max_batch=max_batch, mode=cfg["mode"], hash_bits=args.hash_bits,
+                      visited_set_delete=int(args.visited_set_delete))
     row_bytes = g.row_bytes
 
     # ---- data: generated on the host, resident on the device before anything is timed
@@ -372,6 +375,7 @@ def main():
             "config": {"workload": args.workload, "scale": args.scale, "built_on": cfg["build"], "dim": cfg["dim"], "R": cfg["R"],
                        "L": cfg["L"], "alpha": cfg["alpha"], "step": f"insert {cfg['ins']} + delete {cfg['dele']} + search {cfg['nq']} (k=10)",
                        "l2": "index (vectors + adjacency) larger than L2, and a 256 MiB flush between steps",
+                       "delete": "visited-set (Alg. 6 as printed)" if args.visited_set_delete else "exact in-neighbours",
                        "parallelism": f"replicas x{world}"},
             "search_qps": search_qps,
             "insert_vectors_per_sec": world * (n_upd / 2) / (t_ins * 1e-3), "delete_vectors_per_sec": world * (n_upd / 2) / (t_del * 1e-3),

@@ -69,6 +69,12 @@ typedef struct {
                               reduction of Sec. 5.3, x -> [x, sqrt(M^2 - |x|^2)] with M = this bound on every base
                               vector's norm (an insert with a larger norm fails with GRAND_ERR_INVALID_ARG);
                               searches still return negated inner products */
+  uint32_t visited_set_delete; /* 1: Alg. 6 exactly as printed - the in-neighbours of a deleted node are looked for
+                              only in the visited set of its search (no reverse graph).  Edges from nodes that
+                              the search did not visit stay behind; searches and rebuilds skip neighbours that
+                              are not live.  Default 0: exact in-neighbours, no edge to a deleted node survives.
+                              Vamana mode only. */
+  uint32_t reserved_;
   /* device allocator hooks (default cudaMalloc / cudaFree); lets a host runtime pool the memory */
   void* (*dev_alloc)(size_t bytes, void* user);
   void (*dev_free)(void* ptr, void* user);

@@ -63,6 +63,9 @@ struct Index {
   uint32_t udim = 0;                  // dimension of the caller's vectors
   bool augment = false;               // MIPS -> L2 reduction (Sec. 5.3): x -> [x, sqrt(M^2 - |x|^2)], q -> [q, 0]
   double M2 = 0.0;                    // M^2, M = bound on the base vectors' norms
+  bool approx_delete = false;         // Alg. 6 as printed: in-neighbours of a deleted node are looked for in the
+                                      // visited set of its search only; edges from other nodes stay behind
+                                      // ("dangling") and every traversal skips neighbours that are not live
   float alpha;
   int64_t A_fix;  // round(alpha * 65536): fixed-point alpha for integer vectors
   uint64_t cap;
@@ -309,11 +312,12 @@ Grouped group_requests(std::vector<Request>& rq, uint32_t cap_p) {
 
 // Rebuild of one dirty node u (Alg. 5 dirty loop / Alg. 6 rebuild loop): C = (N_out(u) u scratch_u) \ B;
 // if |C| <= R store it (old order, then new in key order), else compute D_u and prune.
-void rebuild_dirty(Index& ix, uint32_t u, const std::vector<Key>& scratch, const std::vector<uint8_t>* inB) {
+void rebuild_dirty(Index& ix, uint32_t u, const std::vector<Key>& scratch, const std::vector<uint8_t>* inB,
+                   const std::vector<uint8_t>* alive = nullptr) {
   std::vector<uint32_t> keep;
   uint32_t* r = ix.row(u);
   for (uint32_t s = 0; s < ix.deg[u]; ++s)
-    if (!inB || !(*inB)[r[s]]) keep.push_back(r[s]);
+    if ((!inB || !(*inB)[r[s]]) && (!alive || (*alive)[r[s]])) keep.push_back(r[s]);  // `alive`: drops dangling edges
   std::vector<Key> fresh;
   for (const auto& k : scratch) {
     if (k.id == u) continue;
@@ -441,7 +445,14 @@ int insert_batch(Index& ix, const uint32_t* ids, const void* vecs, uint64_t n) {
     for (const auto& k : fwd[i]) rq.push_back({k.id, {k.d, ids[i]}});  // dist is symmetric: reuse D_{p_i}[u]
   if (!fixed) {
     Grouped g = group_requests(rq, ix.P);
-    parallel_for(ix, g.targets.size(), [&](size_t t) { rebuild_dirty(ix, g.targets[t], g.scratch[t], nullptr); });
+    std::vector<uint8_t> alive;  // visited-set delete mode: rows may hold dangling edges; batch members count as alive
+    if (ix.approx_delete) {
+      alive = ix.live;
+      for (uint64_t i = 0; i < n; ++i) alive[ids[i]] = 1;
+    }
+    parallel_for(ix, g.targets.size(), [&](size_t t) {
+      rebuild_dirty(ix, g.targets[t], g.scratch[t], nullptr, ix.approx_delete ? &alive : nullptr);
+    });
   } else {
     // Alg. 7 backward edges: detour find-and-replace, one owner per target, requests in key order.
     Grouped g = group_requests(rq, 0);
@@ -504,7 +515,8 @@ int delete_batch(Index& ix, const uint32_t* ids, uint64_t n) {
   for (uint64_t i = 0; i < n; ++i) inB[ids[i]] = 1;
   std::vector<uint64_t> off;
   std::vector<uint32_t> src;
-  transpose(ix, off, src);  // exact in-neighbours, rebuilt per delete batch and not kept
+  const bool approx = ix.approx_delete && ix.mode == MODE_VAMANA;
+  if (!approx) transpose(ix, off, src);  // exact in-neighbours, rebuilt per delete batch and not kept
 
   uint32_t new_entry = INVALID;  // replacement medoid, used only if the medoid is in B
   if (ix.mode == MODE_FIXED) {
@@ -547,10 +559,13 @@ int delete_batch(Index& ix, const uint32_t* ids, uint64_t n) {
   } else {
     // Alg. 6: per-deleted search on the snapshot; C_i = first k_r of the final worklist minus B.
     std::vector<std::vector<Key>> Ci(n);
+    std::vector<std::vector<uint32_t>> Vi(n);  // visited sets, used by the visited-set variant only
     parallel_for(ix, n, [&](size_t i) {
       std::vector<BeamEntry> C;
       std::vector<Key> V;
       greedy_search(ix, ix.entry, ix.vec(ids[i]), ix.L, ix.vmax, false, C, V, &ix.st);
+      if (approx)
+        for (const auto& k : V) Vi[i].push_back(k.id);
       for (const auto& e : C) {
         if (inB[e.k.id]) continue;
         if (Ci[i].size() == ix.k_repair) break;
@@ -571,15 +586,25 @@ int delete_batch(Index& ix, const uint32_t* ids, uint64_t n) {
     std::vector<std::vector<uint32_t>> touched(n);
     parallel_for(ix, n, [&](size_t i) {
       const uint32_t p = ids[i];
-      for (uint64_t e = off[p]; e < off[p + 1]; ++e) {  // in-neighbour repair: z -> y
-        const uint32_t z = src[e];
-        if (inB[z]) continue;
-        touched[i].push_back(z);
-        for (const auto& k : closest_c(z, Ci[i])) per[i].push_back({z, k});
+      if (approx) {  // Alg. 6 as printed: z in V_i where p_i in N_out(z)
+        for (uint32_t z : Vi[i]) {
+          if (inB[z]) continue;
+          const uint32_t* zr = ix.row(z);
+          if (std::find(zr, zr + ix.deg[z], p) == zr + ix.deg[z]) continue;
+          touched[i].push_back(z);
+          for (const auto& k : closest_c(z, Ci[i])) per[i].push_back({z, k});
+        }
+      } else {
+        for (uint64_t e = off[p]; e < off[p + 1]; ++e) {  // in-neighbour repair: z -> y
+          const uint32_t z = src[e];
+          if (inB[z]) continue;
+          touched[i].push_back(z);
+          for (const auto& k : closest_c(z, Ci[i])) per[i].push_back({z, k});
+        }
       }
       for (uint32_t s = 0; s < ix.deg[p]; ++s) {  // out-neighbour repair: y -> w
         const uint32_t w = ix.row(p)[s];
-        if (inB[w]) continue;
+        if (inB[w] || !ix.live[w]) continue;  // (a dangling edge of p itself: nothing to reconnect)
         for (const auto& k : closest_c(w, Ci[i])) per[i].push_back({k.id, {k.d, w}});
       }
     });
@@ -593,7 +618,9 @@ int delete_batch(Index& ix, const uint32_t* ids, uint64_t n) {
       s.erase(std::remove_if(s.begin(), s.end(), [](const Key& k) { return k.id == INVALID; }), s.end());
       if (s.size() > ix.P) s.resize(ix.P);
     }
-    parallel_for(ix, g.targets.size(), [&](size_t t) { rebuild_dirty(ix, g.targets[t], g.scratch[t], &inB); });
+    parallel_for(ix, g.targets.size(), [&](size_t t) {
+      rebuild_dirty(ix, g.targets[t], g.scratch[t], &inB, approx ? &ix.live : nullptr);
+    });
     if (inB[ix.entry]) {  // medoid deleted: first repair candidate of the old medoid
       for (uint64_t i = 0; i < n; ++i)
         if (ids[i] == ix.entry && !Ci[i].empty()) new_entry = Ci[i][0].id;
@@ -622,12 +649,13 @@ extern "C" {
 
 int grand_oracle_create(uint32_t dim, uint32_t dtype, uint32_t metric, uint32_t R, uint32_t L, float alpha,
                         uint64_t capacity, uint32_t P, uint32_t c, uint32_t k_repair, uint32_t vmax,
-                        uint32_t mode, uint32_t nthreads, float max_norm, void** out) {
+                        uint32_t mode, uint32_t nthreads, float max_norm, uint32_t approx_delete, void** out) {
   if (!out || dim == 0 || R == 0 || L == 0 || dtype > 2 || metric > 1 || mode > 1 || capacity == 0) return ERR_INVALID_ARG;
   const bool augment = mode == MODE_VAMANA && metric == M_IP && max_norm > 0.0f && dtype == DT_F32;
   if (mode == MODE_VAMANA && metric == M_IP && !augment) return ERR_UNSUPPORTED;
   Index* ix = new Index();
   ix->udim = dim;
+  ix->approx_delete = approx_delete != 0 && mode == MODE_VAMANA;
   ix->augment = augment;
   ix->M2 = (double)max_norm * (double)max_norm;
   if (augment) {

@@ -60,7 +60,7 @@ class OracleError(RuntimeError):
 
 class Oracle:
     def __init__(self, dim, dtype, metric, R, L, alpha, capacity, P=0, c=0, k_repair=0, vmax=0,
-                 mode=VAMANA, nthreads=0, max_norm=0.0):
+                 mode=VAMANA, nthreads=0, max_norm=0.0, approx_delete=0):
         self.dim, self.dtype, self.metric, self.R, self.L = dim, dtype, metric, R, L
         self.capacity = int(capacity)
         self.np_dtype = _NP[dtype]
@@ -71,7 +71,7 @@ class Oracle:
         rc = lib().grand_oracle_create(C.c_uint32(dim), C.c_uint32(dtype), C.c_uint32(metric), C.c_uint32(R),
                                        C.c_uint32(L), C.c_float(alpha), C.c_uint64(capacity), C.c_uint32(P),
                                        C.c_uint32(c), C.c_uint32(k_repair), C.c_uint32(vmax), C.c_uint32(mode),
-                                       C.c_uint32(nthreads), C.c_float(max_norm), C.byref(h))
+                                       C.c_uint32(nthreads), C.c_float(max_norm), C.c_uint32(approx_delete), C.byref(h))
         if rc != 0:
             raise OracleError(rc)
         self.h = h

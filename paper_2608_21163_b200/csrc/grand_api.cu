@@ -47,6 +47,11 @@ struct Buf {
 struct grand_index {
   Layout lay;
   uint32_t R, L, P, c, k_repair, vmax, mode, hash_bits, full_transpose;
+  bool approx = false; // visited-set delete mode (Alg. 6 as printed): rows may hold dangling edges
+  unsigned long long* vis_keys = nullptr;  // max_batch x vmax visited lists of the per-deleted searches (that mode only)
+  uint32_t *vis_n = nullptr, *vis_in = nullptr;
+  uint32_t *birth = nullptr, *rowepoch = nullptr;  // per node: batch number of its insertion / of its row's last write
+  uint32_t epoch = 0;                              // batches applied so far
   bool mips = false;   // MIPS -> L2 reduction active (Vamana mode, IP metric, fp32)
   double mips_M2 = 0.0;
   float alpha;
@@ -140,6 +145,7 @@ int ensure(grand_index* idx, Buf& b, size_t bytes, cudaStream_t s) {
 GraphView view(const grand_index* idx) {
   GraphView g;
   g.store = idx->store; g.adj = idx->adj; g.deg = idx->deg; g.live = idx->live; g.rowpfx = idx->rowpfx; g.rowd = idx->rowd; g.R = idx->R; g.cap = idx->cap;
+  g.birth = idx->birth; g.rowepoch = idx->rowepoch; g.epoch = idx->epoch;
   return g;
 }
 
@@ -204,6 +210,7 @@ SearchArgs search_args(grand_index* idx, cudaStream_t s) {
   a.g = view(idx);
   a.entry = idx->entry;
   a.hash_bits = idx->hash_bits;
+  a.check_live = idx->approx ? 1u : 0u;
   a.mips = idx->mips ? 1u : 0u;
   a.mips_M2 = (float)idx->mips_M2;
   a.state = idx->d_state;
@@ -272,6 +279,7 @@ int grand_create_ex(uint32_t dim, uint32_t dtype, uint32_t metric, uint32_t R, u
   idx->mode = o->mode;
   idx->hash_bits = o->hash_bits ? o->hash_bits : 10;
   idx->full_transpose = o->full_transpose;
+  idx->approx = o->visited_set_delete != 0 && o->mode == GRAND_MODE_VAMANA;
   idx->mips = mips;
   idx->mips_M2 = (double)o->mips_max_norm * (double)o->mips_max_norm;
   idx->dev_alloc = o->dev_alloc ? o->dev_alloc : default_alloc;
@@ -312,6 +320,13 @@ int grand_create_ex(uint32_t dim, uint32_t dtype, uint32_t metric, uint32_t R, u
   A(alloc_dev(idx, &idx->unit_off, mb + 1, true));
   A(alloc_dev(idx, &idx->scan_tmp, (cap + 1) / 2048 + mb / 2048 + 8, true));
   A(alloc_dev(idx, &idx->mean_row, lay.row_bytes, true));
+  if (idx->approx) {
+    A(alloc_dev(idx, &idx->vis_keys, (size_t)mb * idx->vmax, false));
+    A(alloc_dev(idx, &idx->vis_n, mb, true));
+    A(alloc_dev(idx, &idx->vis_in, (size_t)mb * idx->vmax, false));
+    A(alloc_dev(idx, &idx->birth, cap, true));
+    A(alloc_dev(idx, &idx->rowepoch, cap, true));
+  }
   A(alloc_dev(idx, &idx->search_ctrs, 64, true));
   if (rc == GRAND_OK && cudaMemset(idx->adj, 0xFF, (size_t)cap * R * 4) != cudaSuccess) rc = GRAND_ERR_CUDA;
   if (rc == GRAND_OK && idx->rowd && cudaMemset(idx->rowd, 0xFF, (size_t)cap * R * 4) != cudaSuccess) rc = GRAND_ERR_CUDA;
@@ -365,6 +380,7 @@ int grand_insert_batch(grand_index* idx, const uint32_t* ids, const void* vecs, 
     return fail(idx, idx->h_state->status, grand_strerror(idx->h_state->status));
   }
   if ((rc = ensure_requests(idx, n * R, s))) return rc;
+  ++idx->epoch;
   GraphView g = view(idx);
   {
     PhaseTimer pt(idx, s, PH_OTHER);
@@ -424,6 +440,7 @@ int grand_insert_batch(grand_index* idx, const uint32_t* ids, const void* vecs, 
     } else {
       RebuildArgs a{};
       a.lay = idx->lay; a.g = g; a.A_fix = idx->A_fix; a.alpha = idx->alpha; a.P = idx->P; a.delmap = nullptr;
+      if (idx->approx) { a.livemap = idx->live; a.newmap = idx->mark; }  // rows may hold dangling edges: drop them
       a.cnt = idx->cnt; a.fill = idx->fill; a.start = idx->start; a.flag = idx->flag;
       a.dirty = (uint32_t*)idx->dirty.p; a.seg_keys = (unsigned long long*)idx->seg_keys.p;
       a.max_blocks = (uint32_t)mbk; a.state = idx->d_state;
@@ -471,6 +488,7 @@ int grand_delete_batch(grand_index* idx, const uint32_t* ids, uint64_t n, grand_
     PhaseTimer pt(idx, s, PH_OTHER);
     CK(launch_validate(ids, n, idx->cap, idx->live, idx->mark, 1, idx->d_state, s));
   }
+  ++idx->epoch;
   GraphView g = view(idx);
   DeleteArgs d{};
   d.lay = idx->lay; d.g = g; d.ids = ids; d.n = n; d.delmap = idx->mark;
@@ -478,7 +496,8 @@ int grand_delete_batch(grand_index* idx, const uint32_t* ids, uint64_t n, grand_
   d.Ci = idx->Ci; d.Ci_n = idx->Ci_n; d.k_repair = idx->k_repair; d.c = idx->c;
   d.in_cnt = idx->in_cnt; d.pair_off = idx->pair_off; d.unit_off = idx->unit_off; d.scan_tmp = idx->scan_tmp;
   d.flag = idx->flag; d.state = idx->d_state;
-  {
+  const bool approx = idx->approx && !fixed;
+  if (!approx) {
     // reverse graph of the snapshot: exact in-neighbours, rebuilt per batch and not kept
     PhaseTimer pt(idx, s, PH_TRANSPOSE);
     // only the in-neighbour rows of the batch are read below, so only those are materialised
@@ -493,6 +512,24 @@ int grand_delete_batch(grand_index* idx, const uint32_t* ids, uint64_t n, grand_
     collect_spans(idx);
     return fail(idx, idx->h_state->status, grand_strerror(idx->h_state->status));
   }
+  if (approx) {
+    // Alg. 6 as printed: the searches come first, their visited sets are the only place where
+    // in-neighbours are looked for
+    {
+      PhaseTimer pt(idx, s, PH_SEARCH);
+      SearchArgs a = search_args(idx, s);
+      a.qids = ids; a.nq = n; a.L = idx->L; a.vmax = idx->vmax;
+      a.out_beam = idx->wk_keys; a.out_beam_n = idx->wk_n; a.beam_stride = idx->wk_stride;
+      a.out_vis = idx->vis_keys; a.out_vis_n = idx->vis_n; a.vis_stride = idx->vmax;
+      CK(launch_beam_search(a, s));
+      idx->stats.n_search_launches++;
+    }
+    PhaseTimer pt(idx, s, PH_TRANSPOSE);
+    d.vis = idx->vis_keys; d.vis_n = idx->vis_n; d.vis_stride = idx->vmax;
+    d.src = idx->vis_in; d.src_stride = idx->vmax; d.livemap = idx->live;
+    CK(launch_delete_visited_in(d, idx->vis_in, s));
+  }
+  if (approx && (rc = read_state(idx, s))) return rc;
   const uint64_t total_in = idx->h_state->total_in;
   const uint64_t nreq = fixed ? total_in + 1 : (total_in + n * R) * idx->c;
   if (nreq >= (1ull << 32)) return fail(idx, GRAND_ERR_CAPACITY, "delete batch touches too many edges");
@@ -505,7 +542,7 @@ int grand_delete_batch(grand_index* idx, const uint32_t* ids, uint64_t n, grand_
     f.flag = idx->flag; f.dirty = (uint32_t*)idx->dirty.p; f.state = idx->d_state;
     CK(launch_fixed_delete(f, total_in, s));
   } else {
-    {
+    if (!approx) {
       PhaseTimer pt(idx, s, PH_SEARCH);
       SearchArgs a = search_args(idx, s);
       a.qids = ids; a.nq = n; a.L = idx->L; a.vmax = idx->vmax;
@@ -530,6 +567,7 @@ int grand_delete_batch(grand_index* idx, const uint32_t* ids, uint64_t n, grand_
       PhaseTimer pt(idx, s, PH_REBUILD);
       RebuildArgs a{};
       a.lay = idx->lay; a.g = g; a.A_fix = idx->A_fix; a.alpha = idx->alpha; a.P = idx->P; a.delmap = idx->mark;
+      if (approx) a.livemap = idx->live;
       a.cnt = idx->cnt; a.fill = idx->fill; a.start = idx->start; a.flag = idx->flag;
       a.dirty = d.dirty; a.seg_keys = (unsigned long long*)idx->seg_keys.p;
       a.max_blocks = (uint32_t)(nreq < 148u * 16u ? nreq : 148u * 16u); a.state = idx->d_state;
@@ -630,6 +668,10 @@ int grand_import_graph(grand_index* idx, const uint32_t* adj, const uint32_t* de
   CK(launch_pad_rows(idx->lay, idx->store, vecs, idx->cap, s));
   if (idx->mips) CK(launch_augment_rows(idx->lay, idx->store, nullptr, idx->cap, idx->mips_M2, s));
   CK(cudaMemsetAsync(idx->rowpfx, 0, idx->cap, s));
+  if (idx->birth) {
+    CK(cudaMemsetAsync(idx->birth, 0, idx->cap * 4, s));
+    CK(cudaMemsetAsync(idx->rowepoch, 0, idx->cap * 4, s));
+  }
   if (idx->rowd) CK(cudaMemsetAsync(idx->rowd, 0xFF, (size_t)idx->cap * idx->R * 4, s));
   CK(launch_pad_adjacency(idx->adj, idx->deg, idx->cap, idx->R, s));
   idx->entry = entry;

@@ -10,6 +10,11 @@ constexpr int kPickWarps = 4;
 constexpr uint32_t kMaxKRepair = 128;
 
 
+// start of the in-neighbour list of batch member i (reverse-graph row, or its slice of the visited-set list)
+__device__ __forceinline__ uint32_t in_base(const DeleteArgs& a, uint64_t i) {
+  return a.src_stride ? (uint32_t)i * a.src_stride : a.off[a.ids[i]];
+}
+
 // in_cnt[i] = in-degree of p_i in the reverse graph (0 for an id that fails validation), then the
 // prefix over the batch and the total number of (deleted node, in-neighbour) pairs.
 __global__ void delete_incnt_kernel(const DeleteArgs a) {
@@ -27,6 +32,40 @@ __global__ void delete_total_kernel(const uint32_t* pair_off, uint64_t n, DevSta
 cudaError_t launch_delete_prepare(const DeleteArgs& a, cudaStream_t s) {
   const unsigned blocks = (unsigned)((a.n + 256) / 256 > 148u * 16u ? 148u * 16u : (a.n + 256) / 256);
   delete_incnt_kernel<<<blocks, 256, 0, s>>>(a);
+  cudaError_t e = launch_exclusive_scan(a.in_cnt, a.pair_off, a.n + 1, a.scan_tmp, s);
+  if (e != cudaSuccess) return e;
+  delete_total_kernel<<<1, 1, 0, s>>>(a.pair_off, a.n, a.state);
+  count_launches(2);
+  return cudaGetLastError();
+}
+
+// Alg. 6 as printed: the in-neighbours of p_i are the visited nodes z whose row holds p_i.  One warp per
+// (batch member, visited entry); hits are appended to the member's slice of `inlist` (order is irrelevant:
+// requests are grouped and sorted later) and counted in in_cnt, whose prefix then drives the pair loop.
+__global__ void delete_visited_in_kernel(const DeleteArgs a, uint32_t* inlist) {
+  const int lane = threadIdx.x & 31;
+  const uint32_t R = a.g.R;
+  const uint64_t total = a.n * a.vis_stride;
+  const uint64_t wglobal = (blockIdx.x * (uint64_t)blockDim.x + threadIdx.x) >> 5;
+  const uint64_t wtotal = ((uint64_t)gridDim.x * blockDim.x) >> 5;
+  for (uint64_t e = wglobal; e < total; e += wtotal) {
+    const uint64_t i = e / a.vis_stride;
+    const uint32_t j = (uint32_t)(e - i * a.vis_stride);
+    if (j >= min(a.vis_n[i], a.vis_stride)) continue;
+    const uint32_t z = key_id(a.vis[i * a.vis_stride + j]);
+    if (bit_test(a.delmap, z)) continue;
+    const uint32_t p = a.ids[i];
+    const uint32_t dz = min(a.g.deg[z], R);
+    bool hit = false;
+    for (uint32_t sb = 0; sb < dz; sb += 32) hit |= sb + lane < dz && a.g.adj[(size_t)z * R + sb + lane] == p;
+    if (__any_sync(0xFFFFFFFFu, hit) && lane == 0) inlist[i * a.vis_stride + atomicAdd(&a.in_cnt[i], 1u)] = z;
+  }
+}
+cudaError_t launch_delete_visited_in(const DeleteArgs& a, uint32_t* inlist, cudaStream_t s) {
+  cudaMemsetAsync(a.in_cnt, 0, (a.n + 1) * 4, s);
+  uint64_t blocks = (a.n * a.vis_stride + 3) / 4;
+  if (blocks > 148u * 32u) blocks = 148u * 32u;
+  delete_visited_in_kernel<<<(unsigned)blocks, 128, 0, s>>>(a, inlist);
   cudaError_t e = launch_exclusive_scan(a.in_cnt, a.pair_off, a.n + 1, a.scan_tmp, s);
   if (e != cudaSuccess) return e;
   delete_total_kernel<<<1, 1, 0, s>>>(a.pair_off, a.n, a.state);
@@ -93,7 +132,7 @@ __global__ void __launch_bounds__(kPickWarps * 32) delete_picks_kernel(const Del
         if (a.pair_off[mid] <= pair) lo = mid; else hi = mid;
       }
       i = lo;
-      x = a.src[a.off[a.ids[i]] + (uint32_t)(pair - a.pair_off[i])];
+      x = a.src[in_base(a, i) + (uint32_t)(pair - a.pair_off[i])];
     } else {
       const uint64_t o = pair - total_in;
       i = o / R;
@@ -101,7 +140,7 @@ __global__ void __launch_bounds__(kPickWarps * 32) delete_picks_kernel(const Del
       const uint32_t p = a.ids[i];
       if (s < a.g.deg[p]) x = a.g.adj[(size_t)p * R + s];
     }
-    const bool act = x != kInvalid && !bit_test(a.delmap, x);
+    const bool act = x != kInvalid && !bit_test(a.delmap, x) && (!a.livemap || bit_test(a.livemap, x));
     const uint64_t rbase = pair * c;
     if (!act) {
       if (lane < c) a.req_tgt[rbase + lane] = kInvalid;
@@ -175,7 +214,7 @@ __global__ void delete_touch_kernel(const DeleteArgs a, const uint64_t total_in)
         const uint64_t mid = (lo + hi) >> 1;
         if (a.pair_off[mid] <= pair) lo = mid; else hi = mid;
       }
-      z = a.src[a.off[a.ids[lo]] + (uint32_t)(pair - a.pair_off[lo])];
+      z = a.src[in_base(a, lo) + (uint32_t)(pair - a.pair_off[lo])];
       first = !bit_test(a.delmap, z) && atomicExch(&a.flag[z], 1u) == 0u;
     }
     warp_append(a.dirty, &a.state->ndirty, first, z);
@@ -232,14 +271,14 @@ __global__ void __launch_bounds__(kPickWarps * 32) delete_picks_staged_kernel(co
       uint32_t x = kInvalid;
       uint64_t rbase;
       if (is_in) {
-        x = a.src[a.off[p] + q];
+        x = a.src[in_base(a, i) + q];
         rbase = ((uint64_t)a.pair_off[i] + q) * c;
       } else {
         const uint32_t sl = q - nin;
         if (sl < a.g.deg[p]) x = a.g.adj[(size_t)p * R + sl];
         rbase = (total_in + (uint64_t)i * R + sl) * c;
       }
-      if (x == kInvalid || bit_test(a.delmap, x)) {
+      if (x == kInvalid || bit_test(a.delmap, x) || (a.livemap && !bit_test(a.livemap, x))) {
         if (lane < c) a.req_tgt[rbase + lane] = kInvalid;
         continue;
       }

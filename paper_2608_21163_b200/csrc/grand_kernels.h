@@ -45,6 +45,13 @@ struct GraphView {
   uint32_t* rowd;  // optional, cap x R: order-preserving bits of dist(u, adj[u][s]); 0xFFFFFFFF = not known
   uint8_t* rowpfx;  // per row: length of the leading run that is a RobustPrune output in ascending key
                     // order (no member of the run prunes a later member); appended entries follow it
+  // visited-set delete mode only (else nullptr): rows may hold edges to ids that were deleted and later came
+  // back with another vector.  birth[v] = batch number of v's latest insertion, rowepoch[u] = batch number of
+  // the latest write of row u; an entry with birth[v] > rowepoch[u] predates v's present vector, so its
+  // cached distance and its place in the pruned run are void.
+  uint32_t* birth;
+  uint32_t* rowepoch;
+  uint32_t epoch;  // number of the running batch
   uint32_t R;
   uint64_t cap;
 };
@@ -69,6 +76,7 @@ struct SearchArgs {
   uint32_t boot_n;
   uint32_t hash_bits;
   uint32_t* work_ctr;  // zeroed by the caller before the launch; nullptr = static striding
+  uint32_t check_live; // 1: skip neighbours that are not live (rows may hold dangling edges)
   uint32_t mips;       // 1: rows are MIPS -> L2 augmented; reported distances go back to negated inner products
   float mips_M2;       // M^2 of that reduction
   DevState* state;
@@ -115,6 +123,8 @@ struct RebuildArgs {
   float alpha;
   uint32_t P;
   const uint32_t* delmap;  // bitmap of the delete batch, or nullptr on insert
+  const uint32_t* livemap; // visited-set delete mode: kept neighbours must be live ...
+  const uint32_t* newmap;  // ... or members of the running insert batch (not published yet)
   uint32_t* cnt; uint32_t* fill; uint32_t* start; uint32_t* flag;
   const uint32_t* dirty;
   unsigned long long* seg_keys;
@@ -159,7 +169,10 @@ struct DeleteArgs {
   const unsigned long long* beam; const uint32_t* beam_n; uint32_t beam_stride;  // per-deleted search result
   unsigned long long* Ci; uint32_t* Ci_n; uint32_t k_repair;                    // repair candidates
   uint32_t c;
-  const uint32_t* off; const uint32_t* src;   // reverse graph
+  const uint32_t* off; const uint32_t* src;   // reverse graph (exact mode): in-neighbours of p at src[off[p] ..]
+  uint32_t src_stride;                        // visited-set mode: in-neighbours of batch member i at src[i * src_stride ..]
+  const uint32_t* livemap;                    // visited-set mode: out-neighbours that are not live are skipped
+  const unsigned long long* vis; const uint32_t* vis_n; uint32_t vis_stride;  // visited lists of the per-deleted searches
   uint32_t* in_cnt; uint32_t* pair_off;       // n+1
   uint32_t* unit_off;                         // n+1: work units (chunks of pairs) per deleted node, prefix
   uint32_t* scan_tmp;
@@ -169,6 +182,7 @@ struct DeleteArgs {
 };
 cudaError_t launch_delete_prepare(const DeleteArgs& a, cudaStream_t s);   // in-degree prefix, total_in
 cudaError_t launch_delete_ci(const DeleteArgs& a, cudaStream_t s);        // repair candidates C_i
+cudaError_t launch_delete_visited_in(const DeleteArgs& a, uint32_t* inlist, cudaStream_t s);  // Alg. 6 as printed: z in V_i with p_i in N_out(z)
 cudaError_t launch_delete_picks(const DeleteArgs& a, uint64_t total_in, cudaStream_t s);
 
 struct FixedDeleteArgs {

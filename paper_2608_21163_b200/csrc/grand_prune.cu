@@ -128,6 +128,10 @@ __global__ void __launch_bounds__(kPruneThreads) forward_prune_kernel(const Prun
     if (tid == 0) {
       a.g.deg[p] = cnt;
       a.g.rowpfx[p] = a.fixed_mode ? 0 : (uint8_t)cnt;
+      if (a.g.birth) {
+        a.g.birth[p] = a.g.epoch;
+        a.g.rowepoch[p] = a.g.epoch;
+      }
     }
     __syncthreads();
   }

@@ -121,22 +121,29 @@ __global__ void __launch_bounds__(kRebuildWarps * 32) rebuild_kernel(const Rebui
     ns = min(ns, P);
     // ---- keep = N_out(u) \ B, stable; kp = how many kept entries come from the pruned prefix
     const uint32_t du = min(a.g.deg[u], R);
-    const uint32_t pfx = min((uint32_t)a.g.rowpfx[u], du);
+    uint32_t pfx = min((uint32_t)a.g.rowpfx[u], du);
+    const uint32_t rowep = a.g.birth ? a.g.rowepoch[u] : 0u;
     uint32_t* row = a.g.adj + (size_t)u * R;
     uint32_t nk = 0, kp = 0;
     for (uint32_t sb = 0; sb < du; sb += 32) {
       const uint32_t s = sb + lane;
       uint32_t v = kInvalid;
-      bool ok = false;
+      bool ok = false, reborn = false;
       if (s < du) {
         v = row[s];
         ok = !(a.delmap && bit_test(a.delmap, v));
+        if (ok && a.livemap) ok = bit_test(a.livemap, v) || (a.newmap && bit_test(a.newmap, v));  // drops dangling edges
+        // an old edge to an id that has come back since this row was written: a legal edge to the new node, but
+        // nothing cached about it holds, and the pruned run ends in front of it
+        reborn = ok && a.g.birth && a.g.birth[v] > rowep;
       }
       const unsigned bal = __ballot_sync(FULL, ok);
+      const unsigned rbal = __ballot_sync(FULL, reborn);
+      if (rbal) pfx = min(pfx, sb + (uint32_t)__ffs(rbal) - 1u);
       if (ok) {
         const uint32_t pos = nk + __popc(bal & lt_mask);
         keep[pos] = v;
-        keepd[pos] = a.g.rowd ? a.g.rowd[(size_t)u * R + s] : kInvalid;
+        keepd[pos] = a.g.rowd && !reborn ? a.g.rowd[(size_t)u * R + s] : kInvalid;
       }
       nk += __popc(bal);
       kp += __popc(__ballot_sync(FULL, ok && s < pfx));
@@ -434,6 +441,7 @@ __global__ void __launch_bounds__(kRebuildWarps * 32) rebuild_kernel(const Rebui
       a.cnt[u] = 0;
       a.fill[u] = 0;
       a.flag[u] = 0;
+      if (a.g.birth) a.g.rowepoch[u] = a.g.epoch;  // every kept entry now refers to its target's present vector
     }
     ++ndone;
     __syncwarp();

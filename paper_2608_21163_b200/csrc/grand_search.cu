@@ -307,7 +307,7 @@ __global__ void __launch_bounds__(kSearchWarps * 32) beam_search_kernel(const Se
         for (int c = 0; c < 4; ++c) {
           if ((uint32_t)(c * 32) < R) {
             const uint32_t v = vrow[c];
-            const bool fresh = v != kInvalid && visit_fresh(hash, a.hash_bits, tags16, v);
+            const bool fresh = v != kInvalid && (!a.check_live || bit_test(a.g.live, v)) && visit_fresh(hash, a.hash_bits, tags16, v);
             const unsigned bal = __ballot_sync(FULL, fresh);
             if (fresh) cid[n + __popc(bal & lt_mask)] = v;
             n += __popc(bal);

@@ -8,11 +8,19 @@ from paper_2608_21163_b200 import synth
 INV = 0xFFFFFFFF
 
 
+def oracle_opts(opts):
+    """The library's option names, translated to the oracle's constructor arguments."""
+    o = dict(opts)
+    if "visited_set_delete" in o:
+        o["approx_delete"] = o.pop("visited_set_delete")
+    return o
+
+
 def make_pair(cfg, capacity, **opts):
     """(oracle, gpu index) with identical parameters."""
     from paper_2608_21163_b200 import binding as gb
     o = go.Oracle(cfg["dim"], cfg["dtype"], cfg["metric"], cfg["R"], cfg["L"], cfg["alpha"], capacity,
-                  mode=cfg["mode"], **opts)
+                  mode=cfg["mode"], **oracle_opts(opts))
     g = gb.GrandIndex(cfg["dim"], cfg["dtype"], cfg["metric"], cfg["R"], cfg["L"], cfg["alpha"], capacity=capacity,
                       max_batch=max(cfg.get("first_batch", 1), cfg["max_build_batch"], cfg["ins"], cfg["dele"], 1), mode=cfg["mode"], **opts)
     return o, g
@@ -52,7 +60,7 @@ def run_stream(cfg, seed=0, check_each=True, oracle=True, gpu=True, opts=None, o
     if oracle and gpu:
         o, g = make_pair(cfg, cap, **opts)
     elif oracle:
-        o = go.Oracle(cfg["dim"], cfg["dtype"], cfg["metric"], cfg["R"], cfg["L"], cfg["alpha"], cap, mode=cfg["mode"], **opts)
+        o = go.Oracle(cfg["dim"], cfg["dtype"], cfg["metric"], cfg["R"], cfg["L"], cfg["alpha"], cap, mode=cfg["mode"], **oracle_opts(opts))
     else:
         g = gb.GrandIndex(cfg["dim"], cfg["dtype"], cfg["metric"], cfg["R"], cfg["L"], cfg["alpha"], capacity=cap,
                           max_batch=max(cfg.get("first_batch", 1), cfg["max_build_batch"], cfg["ins"], cfg["dele"], 1), mode=cfg["mode"], **opts)

@@ -41,6 +41,6 @@ def test_strerror_and_argument_checks_need_no_gpu():
 
 
 def test_options_struct_layout_matches_header():
-    # 2 x u64, 8 x u32, 3 pointers
-    assert ctypes.sizeof(binding.GrandOptions) == 16 + 32 + 24
+    # 2 x u64, 10 x 32-bit fields, 3 pointers
+    assert ctypes.sizeof(binding.GrandOptions) == 16 + 40 + 24
     assert ctypes.sizeof(binding.GrandStats) == 8 * 8 + 7 * 8 + 8

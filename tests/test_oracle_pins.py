@@ -562,3 +562,72 @@ def test_mips_vamana_stream_invariants_and_recall():
         bi, _ = brute_knn(base, live, q[i], 10, metric=go.IP)
         hit += len(set(bi.tolist()) & set(ids[i].tolist()))
     assert hit / (10 * len(q)) > 0.85
+
+
+# ------------------------------------------------------------------ Alg. 6 as printed: visited-set in-neighbours
+def test_visited_set_delete_hand_case_leaves_a_dangling_edge():
+    """1-D points at x = 10*id (ids 0..5), medoid 0.  Rows: 0->[1], 1->[0,2], 2->[1,3], 3->[2,4], 4->[3], and
+    node 5 (x=50) -> [2] although nothing points to 5.  Deleting id 2 searches for x=20 from node 0: the walk
+    visits 0,1,2,3,4 but never 5, so with the visited-set rule node 5 keeps its edge to the deleted node
+    (the exact reverse graph would have repaired it) while 1 and 3 are repaired.  A later search skips the
+    dangling edge, and the edge disappears when node 5 is rebuilt for another reason."""
+    base = (10 * np.arange(6))[:, None].astype(np.uint8)
+    rows = {0: [1], 1: [0, 2], 2: [1, 3], 3: [2, 4], 4: [3], 5: [2]}
+    o = mk(1, R=2, L=8, alpha=1.2, cap=6, c=2, k_repair=4, approx_delete=1)
+    load_graph(o, base, rows, entry=0)
+    o.delete_batch([2])
+    adj, deg, live, entry = o.export_graph()
+    assert adj[1, :deg[1]].tolist() == [0, 3] and adj[3, :deg[3]].tolist() == [4, 1]
+    assert adj[5, :deg[5]].tolist() == [2] and not go.live_mask(live, 6)[2]          # dangling
+    ex = mk(1, R=2, L=8, alpha=1.2, cap=6, c=2, k_repair=4)
+    load_graph(ex, base, rows, entry=0)
+    ex.delete_batch([2])
+    a2, d2, _, _ = ex.export_graph()
+    assert 2 not in a2[5, :d2[5]].tolist()                                           # exact mode repairs node 5
+    ids, _ = o.search(np.array([[50]], np.uint8), 3, 8)
+    assert 2 not in ids[0].tolist()
+    assert o.stats()["dead_edges_seen"] == 0            # node 5 is unreachable, so no traversal met the edge
+    # id 2 comes back with a new vector: node 5's old edge now points at the new node (a legal edge)
+    o.insert_batch([2], np.array([[55]], np.uint8))
+    adj, deg, live, entry = o.export_graph()
+    assert go.live_mask(live, 6)[2] and adj[5, :deg[5]].tolist() == [2]
+
+
+def test_visited_set_delete_stream_invariants():
+    n = 3000
+    base = synth.uniform_u8(0, "base", 0, n, 32)
+    o = go.Oracle(32, go.U8, go.L2, 16, 32, 1.2, n, approx_delete=1)
+    e = go.Oracle(32, go.U8, go.L2, 16, 32, 1.2, n)
+    for lo in range(0, n, 500):
+        ids = np.arange(lo, lo + 500, dtype=np.uint32)
+        o.insert_batch(ids, base[ids]); e.insert_batch(ids, base[ids])
+    ga, gb_ = o.export_graph(), e.export_graph()
+    assert (ga[0] == gb_[0]).all() and (ga[1] == gb_[1]).all()        # identical until the first delete
+    q = synth.uniform_u8(0, "query", 0, 200, 32)
+    alive = np.ones(n, bool)
+    for r in range(3):
+        dele = synth.choose_ids(0, f"del/{r}", np.flatnonzero(alive).astype(np.uint32), 300)
+        o.delete_batch(dele); e.delete_batch(dele)
+        alive[dele] = False
+        back = dele[:100]
+        o.insert_batch(back, base[back]); e.insert_batch(back, base[back])
+        alive[back] = True
+        adj, deg, live, entry = o.export_graph()
+        mask = go.live_mask(live, n)
+        assert (mask == alive).all() and mask[entry] and (deg <= 16).all() and (deg[~mask] == 0).all()
+        dangling = 0
+        for v in np.flatnonzero(mask):
+            row = adj[v, :deg[v]]
+            assert v not in row and len(set(row.tolist())) == len(row)
+            dangling += int((~mask[row]).sum())
+        ids, _ = o.search(q, 10, 32)
+        assert mask[ids[ids != INV]].all()                            # a search never returns a deleted id
+    assert dangling > 0 and o.stats()["dead_edges_seen"] > 0           # the variant really leaves edges behind
+    # recall stays close to the exact-reverse-graph path
+    live_ids = np.flatnonzero(alive).astype(np.uint32)
+    ia, _ = o.search(q, 10, 32); ib, _ = e.search(q, 10, 32)
+    ra = rb = 0
+    for i in range(len(q)):
+        t, _ = brute_knn(base, live_ids, q[i], 10)
+        ra += len(set(t.tolist()) & set(ia[i].tolist())); rb += len(set(t.tolist()) & set(ib[i].tolist()))
+    assert ra / 2000 > 0.85 and abs(ra - rb) / 2000 < 0.05
