@@ -47,15 +47,13 @@ __device__ __forceinline__ bool visit_fresh(uint32_t* hash, uint32_t hash_bits, 
     // zero-halfword test: z(x) has bit 15 / 31 set where the low / high half of x is zero
     auto z = [](uint32_t x) { return (x - 0x00010001u) & ~x & 0x80008000u; };
     if (z(b.x ^ t2) | z(b.y ^ t2) | z(b.z ^ t2) | z(b.w ^ t2)) return false;
-    // first empty half-word (all ones), else evict the slot the tag points at
-    const uint32_t e0 = z(~b.x), e1 = z(~b.y), e2 = z(~b.z), e3 = z(~b.w);
-    uint32_t slot;
-    if (e0) slot = (e0 & 0x8000u) ? 0 : 1;
-    else if (e1) slot = (e1 & 0x8000u) ? 2 : 3;
-    else if (e2) slot = (e2 & 0x8000u) ? 4 : 5;
-    else if (e3) slot = (e3 & 0x8000u) ? 6 : 7;
-    else slot = tag & 7u;
-    reinterpret_cast<unsigned short*>(hash)[bucket * 8 + slot] = (unsigned short)tag;
+    // the bucket is a queue: the new tag enters in front and the oldest one (or an empty marker) falls out
+    uint4 nb;
+    nb.w = __funnelshift_l(b.z, b.w, 16);
+    nb.z = __funnelshift_l(b.y, b.z, 16);
+    nb.y = __funnelshift_l(b.x, b.y, 16);
+    nb.x = (b.x << 16) | tag;
+    reinterpret_cast<uint4*>(hash)[bucket] = nb;
     return true;
   }
   const uint32_t h = (v * 2654435761u) >> (32 - hash_bits);
@@ -140,7 +138,9 @@ __global__ void __launch_bounds__(kSearchWarps * 32) beam_search_kernel(const Se
 #pragma unroll
         for (int u = 0; u < U; ++u) {
           const uint32_t idx = b0 + u * NT + team;
-          idv[u] = idx < n ? cid[idx] : kInvalid;  // (no early exit here: it would serialise the loads)
+          idv[u] = kInvalid;
+          if (u > 0 && b0 + u * NT >= n) continue;  // warp-uniform: this slice of the pass is empty
+          if (idx < n) idv[u] = cid[idx];            // (no per-team early exit here: it would serialise the loads)
           if (idv[u] != kInvalid) {
             load_row<G, CPL>(store + (size_t)idv[u] * row_bytes, nchunk, t, v[u]);
           } else {
@@ -150,6 +150,7 @@ __global__ void __launch_bounds__(kSearchWarps * 32) beam_search_kernel(const Se
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) {
+          if (u > 0 && b0 + u * NT >= n) continue;
           const Dist d = team_dist_regs<T, METRIC, G, CPL>(q, v[u]);
           if (t == 0 && idv[u] != kInvalid) ckey[b0 + u * NT + team] = make_key(d, idv[u]);
         }
@@ -186,8 +187,9 @@ __global__ void __launch_bounds__(kSearchWarps * 32) beam_search_kernel(const Se
       __syncwarp();
       if (m == 0) return;
       if (!a.boot_ids) {  // a new entry closer than every unexpanded one will be expanded next
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) best = min(best, __shfl_xor_sync(FULL, best, o));
+        const uint32_t bhi = __reduce_min_sync(FULL, (uint32_t)(best >> 32));
+        const uint32_t blo = __reduce_min_sync(FULL, (uint32_t)(best >> 32) == bhi ? (uint32_t)best : 0xFFFFFFFFu);
+        best = ((unsigned long long)bhi << 32) | blo;
         if (best < key_clean(alt_key)) prefetch_row(a.g.adj + (size_t)key_id(best) * R, R, lane);
       }
       // rank the survivors among themselves (m is small)
@@ -264,18 +266,24 @@ __global__ void __launch_bounds__(kSearchWarps * 32) beam_search_kernel(const Se
       process(1);
       while (nvis < a.vmax) {
         // closest unexpanded entry; everything before `cursor` is expanded
-        uint32_t pos = kInvalid;
+        // ... and the one after it, the likeliest next expansion
+        uint32_t pos = kInvalid, apos = kInvalid;
         for (uint32_t cb = cursor & ~31u; cb < beam_n; cb += 32) {
           const uint32_t i = cb + lane;
           const bool un = i < beam_n && i >= cursor && !(beam[i] & kExpandedBit);
-          const unsigned bal = __ballot_sync(FULL, un);
-          if (bal) {
+          unsigned bal = __ballot_sync(FULL, un);
+          if (pos == kInvalid && bal) {
             pos = cb + __ffs(bal) - 1;
+            bal &= bal - 1u;
+          }
+          if (pos != kInvalid && bal) {
+            apos = cb + __ffs(bal) - 1;
             break;
           }
         }
         if (pos == kInvalid) break;
         const unsigned long long ek = beam[pos];
+        alt_key = apos != kInvalid ? beam[apos] : kKeyMax;
         __syncwarp();
         if (lane == 0) {
           beam[pos] = ek | kExpandedBit;
@@ -289,18 +297,8 @@ __global__ void __launch_bounds__(kSearchWarps * 32) beam_search_kernel(const Se
         uint32_t vrow[4];
 #pragma unroll
         for (int c = 0; c < 4; ++c) vrow[c] = (uint32_t)(c * 32 + lane) < R ? __ldg(row + c * 32 + lane) : kInvalid;
-        // While that load is in flight: the next unexpanded entry is the likeliest next expansion;
-        // pull its adjacency row towards L2 now (process() does the same for a closer new candidate).
-        alt_key = kKeyMax;
-        for (uint32_t cb = cursor & ~31u; cb < beam_n; cb += 32) {
-          const uint32_t i = cb + lane;
-          const bool un = i < beam_n && i >= cursor && !(beam[i] & kExpandedBit);
-          const unsigned bal = __ballot_sync(FULL, un);
-          if (bal) {
-            alt_key = beam[cb + __ffs(bal) - 1];
-            break;
-          }
-        }
+        // While that load is in flight: pull the adjacency row of the likeliest next expansion towards L2
+        // (process() does the same for a closer new candidate).
         if (alt_key != kKeyMax) prefetch_row(a.g.adj + (size_t)key_id(alt_key) * R, R, lane);
         uint32_t n = 0;
 #pragma unroll
