@@ -171,6 +171,13 @@ __device__ __forceinline__ uint32_t lower_bound_clean(const unsigned long long* 
   return lo;
 }
 
+// Smallest 64-bit key over the warp (all lanes call this): two 32-bit min reductions, high word first.
+__device__ __forceinline__ unsigned long long warp_min_key(unsigned long long k) {
+  const uint32_t hi = __reduce_min_sync(0xFFFFFFFFu, (uint32_t)(k >> 32));
+  const uint32_t lo = __reduce_min_sync(0xFFFFFFFFu, (uint32_t)(k >> 32) == hi ? (uint32_t)k : 0xFFFFFFFFu);
+  return ((unsigned long long)hi << 32) | lo;
+}
+
 // Append `value` to list[*counter ...] for every lane with `need`: one atomic per warp instead of one
 // per lane (all 32 lanes must call this together).  Counters hit by every dirty node or request would
 // otherwise serialise on a single address.

@@ -179,8 +179,7 @@ __global__ void __launch_bounds__(kPickWarps * 32) delete_picks_kernel(const Del
     for (uint32_t r = 0; r < c; ++r) {  // r-th smallest (dist, id)
       unsigned long long best = kKeyMax;
       for (uint32_t j = lane; j < nc; j += 32) best = min(best, keys[j]);
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) best = min(best, __shfl_xor_sync(FULL, best, o));
+      best = warp_min_key(best);
       if (best != kKeyMax) {
         for (uint32_t j = lane; j < nc; j += 32)
           if (keys[j] == best) keys[j] = kKeyMax;
@@ -243,9 +242,13 @@ __global__ void __launch_bounds__(kPickWarps * 32) delete_picks_staged_kernel(co
   const int t = lane % G, team = lane / G;
   const uint32_t R = a.g.R, c = a.c, kr = a.k_repair;
   const uint32_t row_bytes = a.lay.row_bytes, nchunk = a.lay.nchunk;
+  // staged rows sit on an odd number of 16-byte chunks, so that lanes reading the same chunk of 32 different
+  // rows fall on different banks
+  const uint32_t rs = (nchunk | 1u) * 16u;
   uint8_t* crow = smem_raw;                                                    // k_repair staged rows
-  unsigned long long* ckeys = reinterpret_cast<unsigned long long*>(smem_raw + (size_t)kr * row_bytes);  // their keys
+  unsigned long long* ckeys = reinterpret_cast<unsigned long long*>(smem_raw + (size_t)kr * rs);  // their keys
   unsigned long long* keys = ckeys + kr + (size_t)warp * kMaxKRepair;          // per-warp pick scratch
+  uint4* xb = reinterpret_cast<uint4*>(ckeys + ((kr + 1u) & ~1u) + (size_t)kPickWarps * kMaxKRepair) + (size_t)warp * nchunk;  // x's row
   const uint32_t nunits = a.unit_off[a.n];
   unsigned long long npair = 0;
   for (uint32_t unit = blockIdx.x; unit < nunits; unit += gridDim.x) {
@@ -263,7 +266,7 @@ __global__ void __launch_bounds__(kPickWarps * 32) delete_picks_staged_kernel(co
     for (uint32_t e = threadIdx.x; e < nc * nchunk; e += blockDim.x) {
       const uint32_t j = e / nchunk, ch = e - j * nchunk;
       const uint32_t y = key_id(a.Ci[(size_t)i * kr + j]);
-      reinterpret_cast<uint4*>(crow + (size_t)j * row_bytes)[ch] = __ldg(reinterpret_cast<const uint4*>(a.g.store + (size_t)y * row_bytes) + ch);
+      reinterpret_cast<uint4*>(crow + (size_t)j * rs)[ch] = __ldg(reinterpret_cast<const uint4*>(a.g.store + (size_t)y * row_bytes) + ch);
     }
     __syncthreads();
     for (uint32_t q = q0 + warp; q < q1; q += kPickWarps) {
@@ -282,6 +285,53 @@ __global__ void __launch_bounds__(kPickWarps * 32) delete_picks_staged_kernel(co
         if (lane < c) a.req_tgt[rbase + lane] = kInvalid;
         continue;
       }
+      if constexpr (sizeof(T) == 1) {
+        // integer rows: any summation order gives the same distance, so one lane takes one candidate and walks
+        // its staged row against x's row (a broadcast read); the keys stay in registers
+        for (uint32_t ch = lane; ch < nchunk; ch += 32) xb[ch] = __ldg(reinterpret_cast<const uint4*>(a.g.store + (size_t)x * row_bytes) + ch);
+        __syncwarp();
+        unsigned long long k[kMaxKRepair / 32];
+#pragma unroll
+        for (int ps = 0; ps < (int)(kMaxKRepair / 32); ++ps) {
+          k[ps] = kKeyMax;
+          if ((uint32_t)ps * 32u < nc) {
+            const uint32_t j = (uint32_t)ps * 32u + lane;
+            const uint4* cr = reinterpret_cast<const uint4*>(crow + (size_t)min(j, nc - 1u) * rs);
+            int acc = 0;
+#pragma unroll 2
+            for (uint32_t ch = 0; ch < nchunk; ++ch) acc_chunk<T, kMetricL2>(xb[ch], cr[ch], acc);
+            if (j < nc) {
+              const uint32_t y = key_id(ckeys[j]);
+              if (y != x) {
+                k[ps] = make_key(acc, y);
+                ++npair;
+              }
+            }
+          }
+        }
+        __syncwarp();
+        for (uint32_t r = 0; r < c; ++r) {  // r-th smallest (dist, id)
+          unsigned long long mine = k[0];
+#pragma unroll
+          for (int ps = 1; ps < (int)(kMaxKRepair / 32); ++ps) mine = min(mine, k[ps]);
+          const unsigned long long best = warp_min_key(mine);
+#pragma unroll
+          for (int ps = 0; ps < (int)(kMaxKRepair / 32); ++ps)
+            if (k[ps] == best) k[ps] = kKeyMax;
+          if (lane == 0) {
+            if (best == kKeyMax) {
+              a.req_tgt[rbase + r] = kInvalid;
+            } else if (is_in) {
+              a.req_tgt[rbase + r] = x;
+              a.req_key[rbase + r] = best;
+            } else {
+              a.req_tgt[rbase + r] = key_id(best);
+              a.req_key[rbase + r] = (best & 0xFFFFFFFF00000000ull) | x;
+            }
+          }
+        }
+        continue;
+      }
       uint4 xr[CPL];
       load_row<G, CPL>(a.g.store + (size_t)x * row_bytes, nchunk, t, xr);
       for (uint32_t jb = 0; jb < nc; jb += NT) {
@@ -293,7 +343,7 @@ __global__ void __launch_bounds__(kPickWarps * 32) delete_picks_staged_kernel(co
 #pragma unroll
           for (int cc = 0; cc < CPL; ++cc) {
             const uint32_t ch = t + cc * G;
-            v[cc] = ch < nchunk ? reinterpret_cast<const uint4*>(crow + (size_t)j * row_bytes)[ch] : make_uint4(0, 0, 0, 0);
+            v[cc] = ch < nchunk ? reinterpret_cast<const uint4*>(crow + (size_t)j * rs)[ch] : make_uint4(0, 0, 0, 0);
           }
         } else {
 #pragma unroll
@@ -310,8 +360,7 @@ __global__ void __launch_bounds__(kPickWarps * 32) delete_picks_staged_kernel(co
       for (uint32_t r = 0; r < c; ++r) {  // r-th smallest (dist, id)
         unsigned long long best = kKeyMax;
         for (uint32_t j = lane; j < nc; j += 32) best = min(best, keys[j]);
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) best = min(best, __shfl_xor_sync(FULL, best, o));
+        best = warp_min_key(best);
         if (best != kKeyMax) {
           for (uint32_t j = lane; j < nc; j += 32)
             if (keys[j] == best) keys[j] = kKeyMax;
@@ -344,10 +393,10 @@ static cudaError_t launch_delete_picks_t(const DeleteArgs& a, uint64_t total_in,
     delete_touch_kernel<<<(unsigned)tb, 256, 0, s>>>(a, total_in);
     count_launches(1);
   }
-  const size_t stage = (size_t)a.k_repair * a.lay.row_bytes;
+  const size_t stage = (size_t)a.k_repair * ((a.lay.nchunk | 1u) * 16u);
   if (stage <= 64 * 1024) {
     // candidate rows fit shared memory: one staged copy per work unit
-    const size_t smem = stage + ((size_t)a.k_repair + (size_t)kPickWarps * kMaxKRepair) * 8;
+    const size_t smem = stage + ((size_t)((a.k_repair + 1u) & ~1u) + (size_t)kPickWarps * kMaxKRepair) * 8 + (size_t)kPickWarps * a.lay.row_bytes;
     auto kern = delete_picks_staged_kernel<T, METRIC, G, CPL>;
     static size_t smem_set = 0;
     if (smem > smem_set) {

@@ -187,9 +187,7 @@ __global__ void __launch_bounds__(kSearchWarps * 32) beam_search_kernel(const Se
       __syncwarp();
       if (m == 0) return;
       if (!a.boot_ids) {  // a new entry closer than every unexpanded one will be expanded next
-        const uint32_t bhi = __reduce_min_sync(FULL, (uint32_t)(best >> 32));
-        const uint32_t blo = __reduce_min_sync(FULL, (uint32_t)(best >> 32) == bhi ? (uint32_t)best : 0xFFFFFFFFu);
-        best = ((unsigned long long)bhi << 32) | blo;
+        best = warp_min_key(best);
         if (best < key_clean(alt_key)) prefetch_row(a.g.adj + (size_t)key_id(best) * R, R, lane);
       }
       // rank the survivors among themselves (m is small)
