@@ -95,12 +95,41 @@ __global__ void __launch_bounds__(kRebuildWarps * 32) rebuild_kernel(const Rebui
     }
     const uint32_t k = k_next++;
     const uint32_t u = a.dirty[k];
+    // the node some warp will take about one generation of warps from now: its id is fetched here and its row,
+    // cached distances and counters are pulled towards L2 once this node is done
+    const uint32_t k_ahead = k + gridDim.x * kRebuildWarps;
+    const uint32_t u_ahead = k_ahead < ndirty ? a.dirty[k_ahead] : kInvalid;
+    // Everything the node needs from global memory is requested up front, in two rounds (what depends only on
+    // u; then the request segment and the batch-membership bits of the row's entries), so that the latencies
+    // overlap instead of following one another through the phases below.
     const uint32_t cntu = a.cnt[u];
+    const uint32_t startu = a.start[u];
+    const uint32_t du = min(a.g.deg[u], R);
+    uint32_t pfx = min((uint32_t)a.g.rowpfx[u], du);
+    const uint32_t rowep = a.g.birth ? a.g.rowepoch[u] : 0u;
+    uint32_t* row = a.g.adj + (size_t)u * R;
+    uint32_t vrow[4], vrd[4];  // the row and its cached distances, spread over the lanes (R <= 128)
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const uint32_t sl = (uint32_t)c * 32u + lane;
+      vrow[c] = sl < R ? row[sl] : kInvalid;
+      vrd[c] = a.g.rowd && sl < R ? a.g.rowd[(size_t)u * R + sl] : kInvalid;
+    }
     // ---- scratch_u: sort the request segment by (dist, id), keep the first P distinct entries
-    unsigned long long* seg = a.seg_keys + a.start[u];
+    unsigned long long* seg = a.seg_keys + startu;
     if (cntu <= kSegSmem) {
       for (uint32_t j = lane; j < cntu; j += 32) seg_s[j] = seg[j];
       seg = seg_s;
+    }
+    uint32_t okbits = 0;  // bit c: entry c * 32 + lane of the row stays
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const uint32_t sl = (uint32_t)c * 32u + lane, v = vrow[c];
+      if (sl < du) {
+        bool ok = !(a.delmap && bit_test(a.delmap, v));
+        if (ok && a.livemap) ok = bit_test(a.livemap, v) || (a.newmap && bit_test(a.newmap, v));  // drops dangling edges
+        okbits |= (uint32_t)ok << c;
+      }
     }
     __syncwarp();
     bitonic_sort_any(seg, cntu, (uint32_t)lane, 32u, wsync);
@@ -120,33 +149,29 @@ __global__ void __launch_bounds__(kRebuildWarps * 32) rebuild_kernel(const Rebui
     }
     ns = min(ns, P);
     // ---- keep = N_out(u) \ B, stable; kp = how many kept entries come from the pruned prefix
-    const uint32_t du = min(a.g.deg[u], R);
-    uint32_t pfx = min((uint32_t)a.g.rowpfx[u], du);
-    const uint32_t rowep = a.g.birth ? a.g.rowepoch[u] : 0u;
-    uint32_t* row = a.g.adj + (size_t)u * R;
     uint32_t nk = 0, kp = 0;
-    for (uint32_t sb = 0; sb < du; sb += 32) {
-      const uint32_t s = sb + lane;
-      uint32_t v = kInvalid;
-      bool ok = false, reborn = false;
-      if (s < du) {
-        v = row[s];
-        ok = !(a.delmap && bit_test(a.delmap, v));
-        if (ok && a.livemap) ok = bit_test(a.livemap, v) || (a.newmap && bit_test(a.newmap, v));  // drops dangling edges
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const uint32_t sb = (uint32_t)c * 32u;
+      if (sb < du) {
+        const uint32_t s = sb + lane, v = vrow[c];
+        const bool ok = (okbits >> c) & 1u;
         // an old edge to an id that has come back since this row was written: a legal edge to the new node, but
         // nothing cached about it holds, and the pruned run ends in front of it
-        reborn = ok && a.g.birth && a.g.birth[v] > rowep;
+        const bool reborn = ok && a.g.birth && a.g.birth[v] > rowep;
+        const unsigned bal = __ballot_sync(FULL, ok);
+        if (a.g.birth) {
+          const unsigned rbal = __ballot_sync(FULL, reborn);
+          if (rbal) pfx = min(pfx, sb + (uint32_t)__ffs(rbal) - 1u);
+        }
+        if (ok) {
+          const uint32_t pos = nk + __popc(bal & lt_mask);
+          keep[pos] = v;
+          keepd[pos] = reborn ? kInvalid : vrd[c];
+        }
+        nk += __popc(bal);
+        kp += __popc(bal & (pfx > sb ? (pfx - sb >= 32u ? FULL : (1u << (pfx - sb)) - 1u) : 0u));
       }
-      const unsigned bal = __ballot_sync(FULL, ok);
-      const unsigned rbal = __ballot_sync(FULL, reborn);
-      if (rbal) pfx = min(pfx, sb + (uint32_t)__ffs(rbal) - 1u);
-      if (ok) {
-        const uint32_t pos = nk + __popc(bal & lt_mask);
-        keep[pos] = v;
-        keepd[pos] = a.g.rowd && !reborn ? a.g.rowd[(size_t)u * R + s] : kInvalid;
-      }
-      nk += __popc(bal);
-      kp += __popc(__ballot_sync(FULL, ok && s < pfx));
     }
     __syncwarp();
     // ---- fresh = scratch \ keep \ {u}, stable, placed after the keep slots of cand (tagged uncertain)
@@ -444,6 +469,17 @@ __global__ void __launch_bounds__(kRebuildWarps * 32) rebuild_kernel(const Rebui
       if (a.g.birth) a.g.rowepoch[u] = a.g.epoch;  // every kept entry now refers to its target's present vector
     }
     ++ndone;
+    if (u_ahead != kInvalid) {
+      const uint32_t lines = (R + 31u) >> 5;  // 128-byte lines of a row
+      const void* pa = nullptr;
+      if ((uint32_t)lane < lines) pa = a.g.adj + (size_t)u_ahead * R + lane * 32;
+      else if ((uint32_t)lane < 2 * lines) pa = a.g.rowd ? a.g.rowd + (size_t)u_ahead * R + (lane - lines) * 32 : nullptr;
+      else if ((uint32_t)lane == 2 * lines) pa = a.cnt + u_ahead;
+      else if ((uint32_t)lane == 2 * lines + 1) pa = a.start + u_ahead;
+      else if ((uint32_t)lane == 2 * lines + 2) pa = a.g.deg + u_ahead;
+      else if ((uint32_t)lane == 2 * lines + 3) pa = a.g.rowpfx + u_ahead;
+      if (pa) asm volatile("prefetch.global.L2 [%0];" ::"l"(pa));
+    }
     __syncwarp();
   }
   if (npair) atomicAdd(&a.state->counters[CTR_PAIR], npair);
