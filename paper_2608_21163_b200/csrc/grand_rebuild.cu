@@ -23,7 +23,6 @@ namespace grand {
 
 constexpr int kRebuildWarps = 4;
 constexpr uint32_t kSegSmem = 128;       // request segments up to this length are sorted in shared memory
-constexpr uint32_t kWorkChunk = 1;       // dirty nodes taken per work-counter bump
 
 static inline uint32_t even_up_h(uint32_t x) { return (x + 1u) & ~1u; }
 static size_t rebuild_smem_per_warp(uint32_t R, uint32_t P) {
@@ -84,16 +83,14 @@ __global__ void __launch_bounds__(kRebuildWarps * 32) rebuild_kernel(const Rebui
     }
   };
 
-  uint32_t k_next = 0, k_end = 0;
+  // One counter serves every warp of the grid.  The ticket for the node after this one is drawn while this one
+  // is processed, so the atomic's round trip is never waited for.
+  uint32_t ticket = 0;
+  if (lane == 0) ticket = atomicAdd(&a.state->work, 1u);
   for (;;) {
-    if (k_next == k_end) {  // fetch a few nodes per atomic: one counter serves every warp of the grid
-      uint32_t kb = 0;
-      if (lane == 0) kb = atomicAdd(&a.state->work, kWorkChunk);
-      k_next = __shfl_sync(FULL, kb, 0);
-      k_end = min(k_next + kWorkChunk, ndirty);
-      if (k_next >= ndirty) break;
-    }
-    const uint32_t k = k_next++;
+    const uint32_t k = __shfl_sync(FULL, ticket, 0);
+    if (k >= ndirty) break;
+    if (lane == 0) ticket = atomicAdd(&a.state->work, 1u);
     const uint32_t u = a.dirty[k];
     // the node some warp will take about one generation of warps from now: its id is fetched here and its row,
     // cached distances and counters are pulled towards L2 once this node is done
