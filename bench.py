@@ -160,6 +160,8 @@ def main():
     ap.add_argument("--hash-bits", type=int, default=0, help="log2 size of the per-query visited cache (0 = library default)")
     ap.add_argument("--visited-set-delete", action="store_true",
                     help="run the delete variant that takes in-neighbours from the visited sets (dangling edges allowed)")
+    ap.add_argument("--snapshot-search", action="store_true",
+                    help="keep the adjacency twice so that searches may overlap update batches; adds an 'overlap' measurement")
     ap.add_argument("--search-only", type=int, default=0, help="after the build run this many search launches and exit")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
@@ -201,6 +203,8 @@ def main():
     if args.scale != 1.0:
         cfg = synth.scaled(cfg, args.scale)
     total_steps = W + 2 * K + 1      # device-resident steps, then one untimed and K timed end-to-end steps
+    if args.snapshot_search:
+        total_steps += K + 1         # and the same steps once more with the searches on a second stream
     cfg["rounds"] = total_steps
     cfg["n"] = cfg["build"] + total_steps * cfg["ins"]
     cfg["reuse_ids"] = False      # fresh ids every step, whatever the config's own id policy
@@ -211,7 +215,7 @@ def main():
     max_batch = max(cfg["first_batch"], cfg["max_build_batch"], cfg["ins"], cfg["dele"])
     g = gb.GrandIndex(cfg["dim"], cfg["dtype"], cfg["metric"], cfg["R"], cfg["L"], cfg["alpha"], capacity=cap,
                       max_batch=max_batch, mode=cfg["mode"], hash_bits=args.hash_bits,
-                      visited_set_delete=int(args.visited_set_delete))
+                      visited_set_delete=int(args.visited_set_delete), snapshot_search=int(args.snapshot_search))
     row_bytes = g.row_bytes
 
     # ---- data: generated on the host, resident on the device before anything is timed
@@ -287,6 +291,36 @@ def main():
     stats = g.stats()
     launches = stats["kernel_launches"] - launches0
     g.set_profiling(False)
+
+    # ---- snapshot mode: the step's search on a second stream, overlapping the step's update batches
+    overlap = None
+    if args.snapshot_search:
+        side = torch.cuda.Stream()
+        main = torch.cuda.current_stream()
+        t_ov = 0.0
+        for it in range(K + 1):
+            ids, rows = st.insert_ids()
+            d_ins = ids_dev(ids)
+            vec = base[rows[0]:rows[0] + rows[1]]
+            d_del = ids_dev(st.delete_ids())
+            st.end_round()
+            flush.zero_()
+            e0, e1, es = ev(), ev(), ev()
+            torch.cuda.synchronize()
+            e0.record()
+            side.wait_event(e0)
+            with torch.cuda.stream(side):
+                g.search(queries, 10, cfg["L"], out_i, out_d)     # sees the graph of the previous step
+                es.record()
+            g.insert_batch(d_ins, vec)
+            g.delete_batch(d_del)
+            main.wait_event(es)
+            e1.record()
+            torch.cuda.synchronize()
+            if it:
+                t_ov += e0.elapsed_time(e1)
+        overlap = {"ms_per_step_overlapped": t_ov / K, "ms_per_step_in_sequence": (t_ins + t_del + t_srch) / K,
+                   "what": "insert + delete on one stream, the step's search on another (it reads the last published graph)"}
 
     # ---- end to end: host buffers through the host entry points, copies inside the timed region
     pin = lambda a: torch.from_numpy(a).pin_memory()
@@ -379,6 +413,7 @@ def main():
                        "l2": "index (vectors + adjacency) larger than L2, and a 256 MiB flush between steps",
                        "delete": "visited-set (Alg. 6 as printed)" if args.visited_set_delete else "exact in-neighbours",
                        "parallelism": f"replicas x{world}"},
+            "overlap": overlap,
             "search_qps": search_qps,
             "insert_vectors_per_sec": world * (n_upd / 2) / (t_ins * 1e-3), "delete_vectors_per_sec": world * (n_upd / 2) / (t_del * 1e-3),
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,

@@ -74,7 +74,12 @@ typedef struct {
                               the search did not visit stay behind; searches and rebuilds skip neighbours that
                               are not live.  Default 0: exact in-neighbours, no edge to a deleted node survives.
                               Vamana mode only. */
-  uint32_t reserved_;
+  uint32_t snapshot_search;    /* 1: searches may run on other streams (and from other host threads) WHILE an update
+                              batch runs.  The adjacency is kept twice; a batch works on the unpublished copy and
+                              publishes it when it returns, so a search sees exactly the graph of the last batch
+                              that had returned when the search was issued.  Costs capacity*R*4 bytes and one
+                              copy of the changed rows per batch.  Default 0: one copy, and a search must not
+                              overlap an update.  Not combinable with visited_set_delete. */
   /* device allocator hooks (default cudaMalloc / cudaFree); lets a host runtime pool the memory */
   void* (*dev_alloc)(size_t bytes, void* user);
   void (*dev_free)(void* ptr, void* user);

@@ -30,7 +30,7 @@ class GrandOptions(C.Structure):
     _fields_ = [("capacity", C.c_uint64), ("max_batch", C.c_uint64), ("P", C.c_uint32), ("c", C.c_uint32),
                 ("k_repair", C.c_uint32), ("vmax", C.c_uint32), ("mode", C.c_uint32), ("hash_bits", C.c_uint32),
                 ("full_transpose", C.c_uint32), ("mips_max_norm", C.c_float),
-                ("visited_set_delete", C.c_uint32), ("reserved_", C.c_uint32),
+                ("visited_set_delete", C.c_uint32), ("snapshot_search", C.c_uint32),
                 ("dev_alloc", C.c_void_p), ("dev_free", C.c_void_p), ("user", C.c_void_p)]
 
 
@@ -105,7 +105,8 @@ class GrandIndex:
     """One index on the current CUDA device.  Methods mirror the C entry points one to one."""
 
     def __init__(self, dim, dtype, metric, R, L, alpha, capacity=0, max_batch=0, P=0, c=0, k_repair=0, vmax=0,
-                 mode=VAMANA, hash_bits=0, full_transpose=0, mips_max_norm=0.0, visited_set_delete=0):
+                 mode=VAMANA, hash_bits=0, full_transpose=0, mips_max_norm=0.0, visited_set_delete=0,
+                 snapshot_search=0):
         if not torch.cuda.is_available():
             raise RuntimeError("a CUDA device is required (no CPU fallback)")
         self.lib = load()
@@ -114,7 +115,7 @@ class GrandIndex:
         self.dist_dtype = torch.float32 if dtype == F32 else torch.int32
         o = GrandOptions(capacity=capacity, max_batch=max_batch, P=P, c=c, k_repair=k_repair, vmax=vmax, mode=mode,
                          hash_bits=hash_bits, full_transpose=full_transpose, mips_max_norm=mips_max_norm,
-                         visited_set_delete=visited_set_delete)
+                         visited_set_delete=visited_set_delete, snapshot_search=snapshot_search)
         h = C.c_void_p()
         rc = self.lib.grand_create_ex(C.c_uint32(dim), C.c_uint32(dtype), C.c_uint32(metric), C.c_uint32(R),
                                       C.c_uint32(L), C.c_float(alpha), C.byref(o), C.byref(h))

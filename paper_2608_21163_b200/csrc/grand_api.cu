@@ -6,6 +6,7 @@
 #include <cstddef>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <string>
 #include <vector>
 
@@ -52,6 +53,17 @@ struct grand_index {
   uint32_t *vis_n = nullptr, *vis_in = nullptr;
   uint32_t *birth = nullptr, *rowepoch = nullptr;  // per node: batch number of its insertion / of its row's last write
   uint32_t epoch = 0;                              // batches applied so far
+  // snapshot mode: searches read the published adjacency buffer while an update batch works on the other one
+  bool snap = false;
+  uint32_t* adj_alt = nullptr;
+  int pub = 0;                         // 0: adj is published, 1: adj_alt
+  uint32_t* sync_ids = nullptr;        // ids of the last applied batch ...
+  uint64_t sync_n = 0;
+  Buf sync_dirty;                      // ... and its dirty list: the rows the unpublished buffer still lacks
+  uint64_t sync_ndirty = 0;
+  std::mutex pub_mu;                   // guards pub, entry and the reader lists against searches from other threads
+  std::vector<cudaEvent_t> readers[2]; // end-of-search events of the searches launched on each buffer
+  std::vector<cudaEvent_t> reader_pool;
   bool mips = false;   // MIPS -> L2 reduction active (Vamana mode, IP metric, fp32)
   double mips_M2 = 0.0;
   float alpha;
@@ -79,7 +91,7 @@ struct grand_index {
   uint32_t *Ci_n = nullptr, *in_cnt = nullptr, *pair_off = nullptr, *unit_off = nullptr, *scan_tmp = nullptr;
   uint8_t* mean_row = nullptr;
   uint32_t* search_ctrs = nullptr;  // ring of work counters, one per in-flight search launch
-  uint32_t ctr_next = 0;
+  std::atomic<uint32_t> ctr_next{0};
   Buf req_tgt, req_key, seg_keys, dirty;              // grow-only, sized by the number of requests
   Buf t_indeg, t_off, t_fill, t_src;                  // reverse graph, allocated at the first delete
   Buf st_ids, st_vecs, st_out_ids, st_out_d;          // staging of the *_host entry points
@@ -142,9 +154,15 @@ int ensure(grand_index* idx, Buf& b, size_t bytes, cudaStream_t s) {
   return GRAND_OK;
 }
 
-GraphView view(const grand_index* idx) {
+// work = true: the buffer an update batch reads and writes; false: the published one
+uint32_t* adj_of(const grand_index* idx, bool work) {
+  if (!idx->snap) return idx->adj;
+  const int b = work ? 1 - idx->pub : idx->pub;
+  return b == 0 ? idx->adj : idx->adj_alt;
+}
+GraphView view(const grand_index* idx, bool work) {
   GraphView g;
-  g.store = idx->store; g.adj = idx->adj; g.deg = idx->deg; g.live = idx->live; g.rowpfx = idx->rowpfx; g.rowd = idx->rowd; g.R = idx->R; g.cap = idx->cap;
+  g.store = idx->store; g.adj = adj_of(idx, work); g.deg = idx->deg; g.live = idx->live; g.rowpfx = idx->rowpfx; g.rowd = idx->rowd; g.R = idx->R; g.cap = idx->cap;
   g.birth = idx->birth; g.rowepoch = idx->rowepoch; g.epoch = idx->epoch;
   return g;
 }
@@ -202,12 +220,12 @@ int write_state_head(grand_index* idx, cudaStream_t s) {
   return GRAND_OK;
 }
 
-SearchArgs search_args(grand_index* idx, cudaStream_t s) {
+SearchArgs search_args(grand_index* idx, cudaStream_t s, bool work) {
   SearchArgs a{};
-  a.work_ctr = idx->search_ctrs + (idx->ctr_next++ & 63u);
+  a.work_ctr = idx->search_ctrs + (idx->ctr_next.fetch_add(1u) & 63u);
   cudaMemsetAsync(a.work_ctr, 0, 4, s);
   a.lay = idx->lay;
-  a.g = view(idx);
+  a.g = view(idx, work);
   a.entry = idx->entry;
   a.hash_bits = idx->hash_bits;
   a.check_live = idx->approx ? 1u : 0u;
@@ -224,6 +242,43 @@ int ensure_requests(grand_index* idx, uint64_t nreq, cudaStream_t s) {
   if ((rc = ensure(idx, idx->seg_keys, nreq * 8, s))) return rc;
   if ((rc = ensure(idx, idx->dirty, nreq * 4, s))) return rc;
   return GRAND_OK;
+}
+
+// Snapshot mode, start of an update batch: the batch works on the unpublished buffer.  Searches that were
+// launched while that buffer was the published one must have finished, and the rows the previous batch
+// changed are carried over from the published buffer first.
+int begin_update(grand_index* idx, const uint32_t* ids, uint64_t n, cudaStream_t s) {
+  if (!idx->snap) return GRAND_OK;
+  const int w = 1 - idx->pub;
+  {
+    std::lock_guard<std::mutex> lk(idx->pub_mu);
+    for (cudaEvent_t ev : idx->readers[w]) {
+      CK(cudaStreamWaitEvent(s, ev, 0));
+      idx->reader_pool.push_back(ev);
+    }
+    idx->readers[w].clear();
+  }
+  const uint32_t* from = adj_of(idx, false);
+  uint32_t* to = adj_of(idx, true);
+  if (idx->sync_n) CK(launch_copy_rows(from, to, idx->sync_ids, idx->sync_n, idx->R, idx->cap, s));
+  if (idx->sync_ndirty) CK(launch_copy_rows(from, to, (const uint32_t*)idx->sync_dirty.p, idx->sync_ndirty, idx->R, idx->cap, s));
+  idx->sync_n = idx->sync_ndirty = 0;
+  CK(cudaMemcpyAsync(idx->sync_ids, ids, n * 4, cudaMemcpyDeviceToDevice, s));  // the caller's array need not outlive the call
+  return GRAND_OK;
+}
+// End of a successful batch (its kernels have completed): remember which rows the other buffer lacks, publish.
+// A batch that failed after it had started to write (a device loop hit its limit) is not published; the same
+// lists then bring its buffer back to the published state at the start of the next batch.
+void end_update(grand_index* idx, uint64_t n) {
+  const bool ok = idx->h_state->status == 0;
+  std::lock_guard<std::mutex> lk(idx->pub_mu);
+  idx->entry = idx->h_state->entry;
+  idx->nlive = idx->h_state->nlive;
+  if (!idx->snap) return;
+  std::swap(idx->dirty, idx->sync_dirty);
+  idx->sync_ndirty = idx->h_state->ndirty;
+  idx->sync_n = n;
+  if (ok) idx->pub = 1 - idx->pub;
 }
 
 }  // namespace
@@ -262,6 +317,7 @@ int grand_create_ex(uint32_t dim, uint32_t dtype, uint32_t metric, uint32_t R, u
     return GRAND_ERR_INVALID_ARG;
   const bool mips = o->mode == GRAND_MODE_VAMANA && metric == GRAND_IP && o->mips_max_norm > 0.0f && dtype == GRAND_F32;
   if (o->mode == GRAND_MODE_VAMANA && metric == GRAND_IP && !mips) return GRAND_ERR_UNSUPPORTED;
+  if (o->snapshot_search && o->visited_set_delete) return GRAND_ERR_UNSUPPORTED;  // those searches read the live bitmap, which has one copy
   // MIPS -> L2 reduction: rows carry one extra coordinate and the index works on squared L2
   Layout lay = mips ? make_layout(dim + 1, dtype, GRAND_L2) : make_layout(dim, dtype, metric);
   lay.udim = dim;
@@ -280,6 +336,7 @@ int grand_create_ex(uint32_t dim, uint32_t dtype, uint32_t metric, uint32_t R, u
   idx->hash_bits = o->hash_bits ? o->hash_bits : 10;
   idx->full_transpose = o->full_transpose;
   idx->approx = o->visited_set_delete != 0 && o->mode == GRAND_MODE_VAMANA;
+  idx->snap = o->snapshot_search != 0;
   idx->mips = mips;
   idx->mips_M2 = (double)o->mips_max_norm * (double)o->mips_max_norm;
   idx->dev_alloc = o->dev_alloc ? o->dev_alloc : default_alloc;
@@ -299,6 +356,10 @@ int grand_create_ex(uint32_t dim, uint32_t dtype, uint32_t metric, uint32_t R, u
   auto A = [&](int r) { if (rc == GRAND_OK) rc = r; };
   A(alloc_dev(idx, &idx->store, (size_t)cap * lay.row_bytes, true));
   A(alloc_dev(idx, &idx->adj, (size_t)cap * R, false));
+  if (idx->snap) {
+    A(alloc_dev(idx, &idx->adj_alt, (size_t)cap * R, false));
+    A(alloc_dev(idx, &idx->sync_ids, mb, false));
+  }
   A(alloc_dev(idx, &idx->deg, cap, true));
   A(alloc_dev(idx, &idx->live, words, true));
   A(alloc_dev(idx, &idx->rowpfx, cap, true));
@@ -329,6 +390,7 @@ int grand_create_ex(uint32_t dim, uint32_t dtype, uint32_t metric, uint32_t R, u
   }
   A(alloc_dev(idx, &idx->search_ctrs, 64, true));
   if (rc == GRAND_OK && cudaMemset(idx->adj, 0xFF, (size_t)cap * R * 4) != cudaSuccess) rc = GRAND_ERR_CUDA;
+  if (rc == GRAND_OK && idx->snap && cudaMemset(idx->adj_alt, 0xFF, (size_t)cap * R * 4) != cudaSuccess) rc = GRAND_ERR_CUDA;
   if (rc == GRAND_OK && idx->rowd && cudaMemset(idx->rowd, 0xFF, (size_t)cap * R * 4) != cudaSuccess) rc = GRAND_ERR_CUDA;
   if (rc == GRAND_OK && cudaMallocHost(&idx->h_state, sizeof(DevState)) != cudaSuccess) rc = GRAND_ERR_CUDA;
   if (rc == GRAND_OK) {
@@ -349,11 +411,13 @@ int grand_destroy(grand_index* idx) {
   if (!idx) return GRAND_OK;
   cudaDeviceSynchronize();
   for (void* p : idx->owned) idx->dev_free(p, idx->user);
-  for (Buf* b : {&idx->req_tgt, &idx->req_key, &idx->seg_keys, &idx->dirty, &idx->t_indeg, &idx->t_off, &idx->t_fill, &idx->t_src,
+  for (Buf* b : {&idx->req_tgt, &idx->req_key, &idx->seg_keys, &idx->dirty, &idx->sync_dirty, &idx->t_indeg, &idx->t_off, &idx->t_fill, &idx->t_src,
                  &idx->st_ids, &idx->st_vecs, &idx->st_out_ids, &idx->st_out_d})
     if (b->p) idx->dev_free(b->p, idx->user);
   if (idx->h_state) cudaFreeHost(idx->h_state);
   for (auto e : idx->ev_pool) cudaEventDestroy(e);
+  for (auto e : idx->reader_pool) cudaEventDestroy(e);
+  for (auto& rd : idx->readers) for (auto e : rd) cudaEventDestroy(e);
   delete idx;
   return GRAND_OK;
 }
@@ -367,6 +431,7 @@ int grand_insert_batch(grand_index* idx, const uint32_t* ids, const void* vecs, 
   const uint32_t R = idx->R;
   int rc;
   if ((rc = write_state_head(idx, s))) return rc;
+  if ((rc = begin_update(idx, ids, n, s))) return rc;
   {
     PhaseTimer pt(idx, s, PH_OTHER);
     CK(launch_validate(ids, n, idx->cap, idx->live, idx->mark, 0, idx->d_state, s));
@@ -381,7 +446,7 @@ int grand_insert_batch(grand_index* idx, const uint32_t* ids, const void* vecs, 
   }
   if ((rc = ensure_requests(idx, n * R, s))) return rc;
   ++idx->epoch;
-  GraphView g = view(idx);
+  GraphView g = view(idx, true);
   {
     PhaseTimer pt(idx, s, PH_OTHER);
     CK(launch_store_write(idx->lay, idx->store, idx->deg, idx->slot_of, ids, vecs, n, s));
@@ -391,7 +456,7 @@ int grand_insert_batch(grand_index* idx, const uint32_t* ids, const void* vecs, 
   {
     // forward candidates: snapshot search (Alg. 5: visited list; Alg. 7: worklist) or bootstrap scan
     PhaseTimer pt(idx, s, PH_SEARCH);
-    SearchArgs a = search_args(idx, s);
+    SearchArgs a = search_args(idx, s, true);
     a.qids = ids;
     a.nq = n;
     a.L = idx->L;
@@ -454,13 +519,12 @@ int grand_insert_batch(grand_index* idx, const uint32_t* ids, const void* vecs, 
   }
   if ((rc = read_state(idx, s))) return rc;
   collect_spans(idx);
-  idx->entry = idx->h_state->entry;
-  idx->nlive = idx->h_state->nlive;
+  end_update(idx, n);
   if (idx->h_state->status != 0) return fail(idx, idx->h_state->status, grand_strerror(idx->h_state->status));
   return GRAND_OK;
 }
 
-static int build_reverse(grand_index* idx, bool sort_rows, const uint32_t* heads, cudaStream_t s) {
+static int build_reverse(grand_index* idx, bool sort_rows, const uint32_t* heads, bool work, cudaStream_t s) {
   int rc;
   const uint64_t cap = idx->cap;
   if ((rc = ensure(idx, idx->t_indeg, (cap + 1) * 4, s))) return rc;
@@ -468,7 +532,7 @@ static int build_reverse(grand_index* idx, bool sort_rows, const uint32_t* heads
   if ((rc = ensure(idx, idx->t_fill, cap * 4, s))) return rc;
   if ((rc = ensure(idx, idx->t_src, cap * idx->R * 4, s))) return rc;
   TransposeArgs t{};
-  t.g = view(idx);
+  t.g = view(idx, work);
   t.indeg = (uint32_t*)idx->t_indeg.p; t.off = (uint32_t*)idx->t_off.p; t.fillc = (uint32_t*)idx->t_fill.p;
   t.src = (uint32_t*)idx->t_src.p; t.scan_tmp = idx->scan_tmp; t.sort_rows = sort_rows; t.heads = heads;
   CK(launch_transpose(t, s));
@@ -484,12 +548,13 @@ int grand_delete_batch(grand_index* idx, const uint32_t* ids, uint64_t n, grand_
   const uint32_t R = idx->R;
   int rc;
   if ((rc = write_state_head(idx, s))) return rc;
+  if ((rc = begin_update(idx, ids, n, s))) return rc;
   {
     PhaseTimer pt(idx, s, PH_OTHER);
     CK(launch_validate(ids, n, idx->cap, idx->live, idx->mark, 1, idx->d_state, s));
   }
   ++idx->epoch;
-  GraphView g = view(idx);
+  GraphView g = view(idx, true);
   DeleteArgs d{};
   d.lay = idx->lay; d.g = g; d.ids = ids; d.n = n; d.delmap = idx->mark;
   d.beam = idx->wk_keys; d.beam_n = idx->wk_n; d.beam_stride = idx->wk_stride;
@@ -501,7 +566,7 @@ int grand_delete_batch(grand_index* idx, const uint32_t* ids, uint64_t n, grand_
     // reverse graph of the snapshot: exact in-neighbours, rebuilt per batch and not kept
     PhaseTimer pt(idx, s, PH_TRANSPOSE);
     // only the in-neighbour rows of the batch are read below, so only those are materialised
-    if ((rc = build_reverse(idx, false, idx->full_transpose ? nullptr : idx->mark, s))) return rc;
+    if ((rc = build_reverse(idx, false, idx->full_transpose ? nullptr : idx->mark, true, s))) return rc;
     d.off = (uint32_t*)idx->t_off.p; d.src = (uint32_t*)idx->t_src.p;
     CK(launch_delete_prepare(d, s));
   }
@@ -517,7 +582,7 @@ int grand_delete_batch(grand_index* idx, const uint32_t* ids, uint64_t n, grand_
     // in-neighbours are looked for
     {
       PhaseTimer pt(idx, s, PH_SEARCH);
-      SearchArgs a = search_args(idx, s);
+      SearchArgs a = search_args(idx, s, true);
       a.qids = ids; a.nq = n; a.L = idx->L; a.vmax = idx->vmax;
       a.out_beam = idx->wk_keys; a.out_beam_n = idx->wk_n; a.beam_stride = idx->wk_stride;
       a.out_vis = idx->vis_keys; a.out_vis_n = idx->vis_n; a.vis_stride = idx->vmax;
@@ -544,7 +609,7 @@ int grand_delete_batch(grand_index* idx, const uint32_t* ids, uint64_t n, grand_
   } else {
     if (!approx) {
       PhaseTimer pt(idx, s, PH_SEARCH);
-      SearchArgs a = search_args(idx, s);
+      SearchArgs a = search_args(idx, s, true);
       a.qids = ids; a.nq = n; a.L = idx->L; a.vmax = idx->vmax;
       a.out_beam = idx->wk_keys; a.out_beam_n = idx->wk_n; a.beam_stride = idx->wk_stride;
       CK(launch_beam_search(a, s));
@@ -580,8 +645,7 @@ int grand_delete_batch(grand_index* idx, const uint32_t* ids, uint64_t n, grand_
   }
   if ((rc = read_state(idx, s))) return rc;
   collect_spans(idx);
-  idx->entry = idx->h_state->entry;
-  idx->nlive = idx->h_state->nlive;
+  end_update(idx, n);
   if (idx->h_state->status != 0) return fail(idx, idx->h_state->status, grand_strerror(idx->h_state->status));
   return GRAND_OK;
 }
@@ -594,12 +658,35 @@ int grand_search(const grand_index* cidx, const void* queries, uint64_t nq, uint
   if (nq == 0) return GRAND_OK;
   cudaStream_t s = (cudaStream_t)stream;
   {
+    // the lock keeps the choice of the published buffer, the launch and the registration of the launch's end
+    // as a reader of that buffer together (an update batch on another host thread may publish at any time)
+    std::lock_guard<std::mutex> lk(idx->pub_mu);
     PhaseTimer pt(idx, s, PH_SEARCH);
-    SearchArgs a = search_args(idx, s);
+    SearchArgs a = search_args(idx, s, false);
     a.queries = queries; a.nq = nq; a.L = L; a.vmax = 2 * L; a.k = k;
     a.out_ids = out_ids; a.out_dists = out_dists;
     CK(launch_beam_search(a, s));
     idx->stats.n_search_launches++;
+    if (idx->snap) {
+      std::vector<cudaEvent_t>& rd = idx->readers[idx->pub];
+      if (rd.size() >= 256) {  // searches only, no update in between: recycle the events that have completed
+        size_t w = 0;
+        for (cudaEvent_t ev : rd) {
+          if (cudaEventQuery(ev) == cudaSuccess) idx->reader_pool.push_back(ev);
+          else rd[w++] = ev;
+        }
+        rd.resize(w);
+      }
+      cudaEvent_t ev = nullptr;
+      if (!idx->reader_pool.empty()) {
+        ev = idx->reader_pool.back();
+        idx->reader_pool.pop_back();
+      } else {
+        CK(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
+      }
+      CK(cudaEventRecord(ev, s));
+      rd.push_back(ev);
+    }
   }
   if (idx->profiling) {
     CK(cudaStreamSynchronize(s));
@@ -652,7 +739,7 @@ int grand_search_host(grand_index* idx, const void* queries, uint64_t nq, uint32
 int grand_export_graph(const grand_index* idx, uint32_t* adj, uint32_t* deg, uint32_t* live, uint32_t* entry_out, grand_stream stream) {
   if (!idx) return GRAND_ERR_INVALID_ARG;
   cudaStream_t s = (cudaStream_t)stream;
-  if (adj) CK(cudaMemcpyAsync(adj, idx->adj, (size_t)idx->cap * idx->R * 4, cudaMemcpyDeviceToDevice, s));
+  if (adj) CK(cudaMemcpyAsync(adj, adj_of(idx, false), (size_t)idx->cap * idx->R * 4, cudaMemcpyDeviceToDevice, s));
   if (deg) CK(cudaMemcpyAsync(deg, idx->deg, idx->cap * 4, cudaMemcpyDeviceToDevice, s));
   if (live) CK(cudaMemcpyAsync(live, idx->live, (idx->cap + 31) / 32 * 4, cudaMemcpyDeviceToDevice, s));
   if (entry_out) *entry_out = idx->entry;
@@ -663,6 +750,7 @@ int grand_import_graph(grand_index* idx, const uint32_t* adj, const uint32_t* de
   if (!idx || !adj || !deg || !live || !vecs) return fail(idx, GRAND_ERR_INVALID_ARG, "null argument");
   cudaStream_t s = (cudaStream_t)stream;
   CK(cudaMemcpyAsync(idx->adj, adj, (size_t)idx->cap * idx->R * 4, cudaMemcpyDeviceToDevice, s));
+  idx->sync_n = idx->sync_ndirty = 0;  // both buffers are rewritten below
   CK(cudaMemcpyAsync(idx->deg, deg, idx->cap * 4, cudaMemcpyDeviceToDevice, s));
   CK(cudaMemcpyAsync(idx->live, live, (idx->cap + 31) / 32 * 4, cudaMemcpyDeviceToDevice, s));
   CK(launch_pad_rows(idx->lay, idx->store, vecs, idx->cap, s));
@@ -674,6 +762,7 @@ int grand_import_graph(grand_index* idx, const uint32_t* adj, const uint32_t* de
   }
   if (idx->rowd) CK(cudaMemsetAsync(idx->rowd, 0xFF, (size_t)idx->cap * idx->R * 4, s));
   CK(launch_pad_adjacency(idx->adj, idx->deg, idx->cap, idx->R, s));
+  if (idx->snap) CK(cudaMemcpyAsync(idx->adj_alt, idx->adj, (size_t)idx->cap * idx->R * 4, cudaMemcpyDeviceToDevice, s));
   idx->entry = entry;
   idx->nlive = 0;
   int rc;
@@ -687,7 +776,7 @@ int grand_reverse_graph(grand_index* idx, uint32_t* off, uint32_t* src, uint64_t
   if (!idx) return GRAND_ERR_INVALID_ARG;
   cudaStream_t s = (cudaStream_t)stream;
   int rc;
-  if ((rc = build_reverse(idx, true, nullptr, s))) return rc;
+  if ((rc = build_reverse(idx, true, nullptr, false, s))) return rc;
   uint32_t E = 0;
   CK(cudaMemcpyAsync(&E, (uint32_t*)idx->t_off.p + idx->cap, 4, cudaMemcpyDeviceToHost, s));
   CK(cudaStreamSynchronize(s));

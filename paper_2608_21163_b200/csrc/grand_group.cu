@@ -420,6 +420,25 @@ __global__ void pad_adjacency_kernel(uint32_t* adj, const uint32_t* deg, uint64_
     if ((uint32_t)(i - v * R) >= deg[v]) adj[i] = kInvalid;
   }
 }
+__global__ void copy_rows_kernel(const uint32_t* __restrict__ src, uint32_t* __restrict__ dst, const uint32_t* __restrict__ ids,
+                                 const uint64_t n, const uint32_t R, const uint64_t cap) {
+  const int lane = threadIdx.x & 31;
+  const uint64_t wglobal = (blockIdx.x * (uint64_t)blockDim.x + threadIdx.x) >> 5;
+  const uint64_t wtotal = ((uint64_t)gridDim.x * blockDim.x) >> 5;
+  for (uint64_t i = wglobal; i < n; i += wtotal) {
+    const uint32_t v = ids[i];
+    if (v >= cap) continue;
+    for (uint32_t s = lane; s < R; s += 32) dst[(size_t)v * R + s] = src[(size_t)v * R + s];
+  }
+}
+cudaError_t launch_copy_rows(const uint32_t* src, uint32_t* dst, const uint32_t* ids, uint64_t n, uint32_t R, uint64_t cap, cudaStream_t s) {
+  if (n == 0) return cudaSuccess;
+  uint64_t blocks = (n + 7) / 8;
+  if (blocks > 148u * 32u) blocks = 148u * 32u;
+  copy_rows_kernel<<<(unsigned)blocks, 256, 0, s>>>(src, dst, ids, n, R, cap);
+  count_launches(1);
+  return cudaGetLastError();
+}
 cudaError_t launch_pad_adjacency(uint32_t* adj, const uint32_t* deg, uint64_t cap, uint32_t R, cudaStream_t s) {
   pad_adjacency_kernel<<<grid_for(cap * R), kThreads, 0, s>>>(adj, deg, cap, R);
   count_launches(1);

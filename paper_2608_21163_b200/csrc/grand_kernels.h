@@ -213,6 +213,8 @@ cudaError_t launch_pad_rows(const Layout& lay, uint8_t* store, const void* vecs,
 // MIPS -> L2 reduction: norm check of a batch (status -1 above the bound) and the extra coordinate of stored rows
 cudaError_t launch_check_norms(const Layout& lay, const void* vecs, uint64_t n, double M2, DevState* st, cudaStream_t s);
 cudaError_t launch_augment_rows(const Layout& lay, uint8_t* store, const uint32_t* ids, uint64_t n, double M2, cudaStream_t s);
+// dst[v][:] = src[v][:] for the listed rows v (ids >= cap are skipped)
+cudaError_t launch_copy_rows(const uint32_t* src, uint32_t* dst, const uint32_t* ids, uint64_t n, uint32_t R, uint64_t cap, cudaStream_t s);
 cudaError_t launch_pad_adjacency(uint32_t* adj, const uint32_t* deg, uint64_t cap, uint32_t R, cudaStream_t s);
 cudaError_t launch_fill_u32(uint32_t* p, uint32_t v, uint64_t n, cudaStream_t s);
 

@@ -13,6 +13,7 @@ def oracle_opts(opts):
     o = dict(opts)
     if "visited_set_delete" in o:
         o["approx_delete"] = o.pop("visited_set_delete")
+    o.pop("snapshot_search", None)     # a property of the library's memory management, not of the method
     return o
 
 
