@@ -62,8 +62,16 @@ __device__ __forceinline__ bool visit_fresh(uint32_t* hash, uint32_t hash_bits, 
   return true;
 }
 
+// Resident blocks per SM that the register allocation must leave room for.  Only the 6-chunks-per-lane layout
+// needs a bound (without it the allocation costs a sixth block per SM); the widest rows keep so many loads in
+// flight per lane that any bound means spills, and short rows fit anyway.
+template <int G, int CPL>
+constexpr int search_min_blocks() {
+  return (G < 32 && CPL >= 6) ? 6 : 1;
+}
+
 template <typename T, int METRIC, int G, int CPL>
-__global__ void __launch_bounds__(kSearchWarps * 32) beam_search_kernel(const SearchArgs a, const uint32_t per_warp_bytes) {
+__global__ void __launch_bounds__(kSearchWarps * 32, search_min_blocks<G, CPL>()) beam_search_kernel(const SearchArgs a, const uint32_t per_warp_bytes) {
   using Dist = typename Elem<T>::Dist;
   constexpr int NT = 32 / G;                                   // teams per warp
   constexpr int U = CPL == 1 ? 4 : ((CPL == 2 || G == 32) ? 2 : 1);  // vectors in flight per team
@@ -139,7 +147,8 @@ __global__ void __launch_bounds__(kSearchWarps * 32) beam_search_kernel(const Se
         for (int u = 0; u < U; ++u) {
           const uint32_t idx = b0 + u * NT + team;
           idv[u] = kInvalid;
-          if (u > 0 && b0 + u * NT >= n) continue;  // warp-uniform: this slice of the pass is empty
+          // warp-uniform: this slice of the pass is empty (whole-warp teams keep both rows' loads back to back)
+          if (G < 32 && u > 0 && b0 + u * NT >= n) continue;
           if (idx < n) idv[u] = cid[idx];            // (no per-team early exit here: it would serialise the loads)
           if (idv[u] != kInvalid) {
             load_row<G, CPL>(store + (size_t)idv[u] * row_bytes, nchunk, t, v[u]);
@@ -150,7 +159,7 @@ __global__ void __launch_bounds__(kSearchWarps * 32) beam_search_kernel(const Se
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-          if (u > 0 && b0 + u * NT >= n) continue;
+          if (G < 32 && u > 0 && b0 + u * NT >= n) continue;
           const Dist d = team_dist_regs<T, METRIC, G, CPL>(q, v[u]);
           if (t == 0 && idv[u] != kInvalid) ckey[b0 + u * NT + team] = make_key(d, idv[u]);
         }
