@@ -62,12 +62,12 @@ __device__ __forceinline__ bool visit_fresh(uint32_t* hash, uint32_t hash_bits, 
   return true;
 }
 
-// Resident blocks per SM that the register allocation must leave room for.  Only the 6-chunks-per-lane layout
-// needs a bound (without it the allocation costs a sixth block per SM); the widest rows keep so many loads in
-// flight per lane that any bound means spills, and short rows fit anyway.
+// Resident blocks per SM that the register allocation must leave room for, per layout (measured: the 6-chunk
+// layout gains a sixth block from its bound; the widest rows keep so many loads in flight per lane that a tighter
+// bound than 3 blocks means spills; short rows run best at 7 blocks of the 8 their shared memory allows).
 template <int G, int CPL>
 constexpr int search_min_blocks() {
-  return (G < 32 && CPL >= 6) ? 6 : 1;
+  return G == 32 ? (CPL >= 8 ? 3 : CPL >= 4 ? 5 : 8) : (CPL >= 6 ? 6 : 7);
 }
 
 template <typename T, int METRIC, int G, int CPL>
