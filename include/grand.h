@@ -79,7 +79,9 @@ typedef struct {
                               publishes it when it returns, so a search sees exactly the graph of the last batch
                               that had returned when the search was issued.  Costs capacity*R*4 bytes and one
                               copy of the changed rows per batch.  Default 0: one copy, and a search must not
-                              overlap an update.  Not combinable with visited_set_delete. */
+                              overlap an update.  Only grand_search (device pointers) may overlap; the *_host
+                              variants share one staging area with the update calls, and profiling
+                              (grand_set_profiling) assumes one caller.  Not combinable with visited_set_delete. */
   /* device allocator hooks (default cudaMalloc / cudaFree); lets a host runtime pool the memory */
   void* (*dev_alloc)(size_t bytes, void* user);
   void (*dev_free)(void* ptr, void* user);

@@ -139,7 +139,9 @@ __global__ void __launch_bounds__(kSearchWarps * 32, search_min_blocks<G, CPL>()
 
     // Evaluate cid[0..n) against the query and merge the survivors into the worklist.
     auto process = [&](uint32_t n) {
-      // 1. distances: NT teams, U vectors in flight per team
+      // 1. distances: NT teams, U vectors in flight per team; only keys below the worst entry are kept
+      const unsigned long long worst = beam_n == L ? key_clean(beam[L - 1]) : kKeyMax;
+      uint32_t nkept = 0;
       for (uint32_t b0 = 0; b0 < n; b0 += NT * U) {
         uint4 v[U][CPL];
         uint32_t idv[U];
@@ -161,28 +163,29 @@ __global__ void __launch_bounds__(kSearchWarps * 32, search_min_blocks<G, CPL>()
         for (int u = 0; u < U; ++u) {
           if (G < 32 && u > 0 && b0 + u * NT >= n) continue;
           const Dist d = team_dist_regs<T, METRIC, G, CPL>(q, v[u]);
-          if (t == 0 && idv[u] != kInvalid) ckey[b0 + u * NT + team] = make_key(d, idv[u]);
+          const unsigned long long key = make_key(d, idv[u]);
+          const bool below = t == 0 && idv[u] != kInvalid && key < worst;
+          const unsigned bal = __ballot_sync(FULL, below);
+          if (below) ckey[nkept + __popc(bal & lt_mask)] = key;
+          nkept += __popc(bal);
         }
       }
       n_dist += n;
+      if (nkept == 0) return;  // the common case late in a search: nothing enters the worklist
       __syncwarp();
-      // 2. keep keys below the worst entry that are not already in the worklist; compact them in
-      //    place (a write never passes the reader of its own chunk) and remember their ranks
-      const unsigned long long worst = beam_n == L ? key_clean(beam[L - 1]) : kKeyMax;
+      // 2. drop keys that are already in the worklist; compact the rest in place (a write never passes the
+      //    reader of its own chunk) and remember their ranks
       uint32_t m = 0;
       unsigned long long best = kKeyMax;
-      for (uint32_t jb = 0; jb < n; jb += 32) {
+      for (uint32_t jb = 0; jb < nkept; jb += 32) {
         const uint32_t j = jb + lane;
         bool pass = false;
         unsigned long long key = 0;
         uint32_t b = 0;
-        if (j < n) {
+        if (j < nkept) {
           key = ckey[j];
-          pass = key < worst;
-          if (pass) {
-            b = lower_bound_clean(beam, beam_n, key);
-            if (b < beam_n && key_clean(beam[b]) == key) pass = false;
-          }
+          b = lower_bound_clean(beam, beam_n, key);
+          pass = !(b < beam_n && key_clean(beam[b]) == key);
         }
         const unsigned bal = __ballot_sync(FULL, pass);
         if (pass) {
