@@ -249,6 +249,8 @@ __global__ void __launch_bounds__(kPickWarps * 32) delete_picks_staged_kernel(co
   unsigned long long* ckeys = reinterpret_cast<unsigned long long*>(smem_raw + (size_t)kr * rs);  // their keys
   unsigned long long* keys = ckeys + kr + (size_t)warp * kMaxKRepair;          // per-warp pick scratch
   uint4* xb = reinterpret_cast<uint4*>(ckeys + ((kr + 1u) & ~1u) + (size_t)kPickWarps * kMaxKRepair) + (size_t)warp * nchunk;  // x's row
+  int* cnorm = reinterpret_cast<int*>(reinterpret_cast<uint4*>(ckeys + ((kr + 1u) & ~1u) + (size_t)kPickWarps * kMaxKRepair) +
+                                      (size_t)kPickWarps * nchunk);  // |y|^2 of the staged rows (integer rows only)
   const uint32_t nunits = a.unit_off[a.n];
   unsigned long long npair = 0;
   for (uint32_t unit = blockIdx.x; unit < nunits; unit += gridDim.x) {
@@ -269,6 +271,16 @@ __global__ void __launch_bounds__(kPickWarps * 32) delete_picks_staged_kernel(co
       reinterpret_cast<uint4*>(crow + (size_t)j * rs)[ch] = __ldg(reinterpret_cast<const uint4*>(a.g.store + (size_t)y * row_bytes) + ch);
     }
     __syncthreads();
+    if constexpr (sizeof(T) == 1) {
+      // |x - y|^2 = |x|^2 + |y|^2 - 2 x.y in exact integers: the pair loop then needs one dp4a per word, not two
+      for (uint32_t j = threadIdx.x; j < nc; j += blockDim.x) {
+        const uint4* cr = reinterpret_cast<const uint4*>(crow + (size_t)j * rs);
+        int acc = 0;
+        for (uint32_t ch = 0; ch < nchunk; ++ch) acc_chunk<T, kMetricIP>(cr[ch], cr[ch], acc);
+        cnorm[j] = acc;
+      }
+      __syncthreads();
+    }
     for (uint32_t q = q0 + warp; q < q1; q += kPickWarps) {
       const bool is_in = q < nin;
       uint32_t x = kInvalid;
@@ -288,7 +300,13 @@ __global__ void __launch_bounds__(kPickWarps * 32) delete_picks_staged_kernel(co
       if constexpr (sizeof(T) == 1) {
         // integer rows: any summation order gives the same distance, so one lane takes one candidate and walks
         // its staged row against x's row (a broadcast read); the keys stay in registers
-        for (uint32_t ch = lane; ch < nchunk; ch += 32) xb[ch] = __ldg(reinterpret_cast<const uint4*>(a.g.store + (size_t)x * row_bytes) + ch);
+        int xn = 0;
+        for (uint32_t ch = lane; ch < nchunk; ch += 32) {
+          const uint4 xv = __ldg(reinterpret_cast<const uint4*>(a.g.store + (size_t)x * row_bytes) + ch);
+          xb[ch] = xv;
+          acc_chunk<T, kMetricIP>(xv, xv, xn);
+        }
+        xn = __reduce_add_sync(FULL, xn);
         __syncwarp();
         unsigned long long k[kMaxKRepair / 32];
 #pragma unroll
@@ -297,13 +315,13 @@ __global__ void __launch_bounds__(kPickWarps * 32) delete_picks_staged_kernel(co
           if ((uint32_t)ps * 32u < nc) {
             const uint32_t j = (uint32_t)ps * 32u + lane;
             const uint4* cr = reinterpret_cast<const uint4*>(crow + (size_t)min(j, nc - 1u) * rs);
-            int acc = 0;
+            int dot = 0;
 #pragma unroll 2
-            for (uint32_t ch = 0; ch < nchunk; ++ch) acc_chunk<T, kMetricL2>(xb[ch], cr[ch], acc);
+            for (uint32_t ch = 0; ch < nchunk; ++ch) acc_chunk<T, kMetricIP>(xb[ch], cr[ch], dot);
             if (j < nc) {
               const uint32_t y = key_id(ckeys[j]);
               if (y != x) {
-                k[ps] = make_key(acc, y);
+                k[ps] = make_key(xn + cnorm[j] - 2 * dot, y);
                 ++npair;
               }
             }
@@ -396,7 +414,8 @@ static cudaError_t launch_delete_picks_t(const DeleteArgs& a, uint64_t total_in,
   const size_t stage = (size_t)a.k_repair * ((a.lay.nchunk | 1u) * 16u);
   if (stage <= 64 * 1024) {
     // candidate rows fit shared memory: one staged copy per work unit
-    const size_t smem = stage + ((size_t)((a.k_repair + 1u) & ~1u) + (size_t)kPickWarps * kMaxKRepair) * 8 + (size_t)kPickWarps * a.lay.row_bytes;
+    const size_t smem = stage + ((size_t)((a.k_repair + 1u) & ~1u) + (size_t)kPickWarps * kMaxKRepair) * 8 +
+                        (size_t)kPickWarps * a.lay.row_bytes + (size_t)a.k_repair * 4;
     auto kern = delete_picks_staged_kernel<T, METRIC, G, CPL>;
     static size_t smem_set = 0;
     if (smem > smem_set) {
