@@ -110,7 +110,6 @@ cudaError_t launch_delete_ci(const DeleteArgs& a, cudaStream_t s) {
 template <typename T, int METRIC, int G, int CPL>
 __global__ void __launch_bounds__(kPickWarps * 32) delete_picks_kernel(const DeleteArgs a, const uint64_t total_in) {
   using Dist = typename Elem<T>::Dist;
-  constexpr unsigned FULL = 0xFFFFFFFFu;
   constexpr int NT = 32 / G;
   __shared__ unsigned long long keys_s[kPickWarps][kMaxKRepair];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;

@@ -151,7 +151,7 @@ __global__ void __launch_bounds__(kRebuildWarps * 32) rebuild_kernel(const Rebui
     for (int c = 0; c < 4; ++c) {
       const uint32_t sb = (uint32_t)c * 32u;
       if (sb < du) {
-        const uint32_t s = sb + lane, v = vrow[c];
+        const uint32_t v = vrow[c];
         const bool ok = (okbits >> c) & 1u;
         // an old edge to an id that has come back since this row was written: a legal edge to the new node, but
         // nothing cached about it holds, and the pruned run ends in front of it
@@ -354,15 +354,25 @@ __global__ void __launch_bounds__(kRebuildWarps * 32) rebuild_kernel(const Rebui
         bitonic_sort_clean(cand, nC, (uint32_t)lane, 32u, wsync);
         cs = cand;
       }
-      for (uint32_t w = lane; w < nC * W; w += 32) prune[w] = 0u;
       if ((uint32_t)lane < W) hasp[lane] = 0u;
-      // ---- prune tests in parallel: pairs with an uncertain member, or the whole upper triangle
+      // lane w holds word w of the set of candidates that are still valid
+      uint32_t valid = 0;
+      if ((uint32_t)lane < W) {
+        const uint32_t lo = lane * 32;
+        valid = nC >= lo + 32 ? 0xFFFFFFFFu : (nC > lo ? (1u << (nC - lo)) - 1u : 0u);
+      }
       const uint32_t nu = nC - kpe;
       uint32_t jprev = kInvalid;
       uint4 rj[CPL];
 #pragma unroll
       for (int c = 0; c < CPL; ++c) rj[c] = make_uint4(0, 0, 0, 0);
-      if (nu <= 2 * P && 2 * nu + 1 < nC) {
+      if (nu <= 2 * P) {  // (the list of uncertain positions holds 2P entries)
+        // ---- few uncertain members among a pruned run.  Members of the run never prune each other, so the
+        //      sequential prune only ever changes at an uncertain member f, and those are taken in key order:
+        //      (a) does a valid member of the run in front of f prune it (earlier uncertain survivors have
+        //      already had their say in their own step b)?  then f is gone;  (b) otherwise f is selected and
+        //      prunes among the valid candidates behind it.  Only tests the sequential algorithm needs are
+        //      evaluated, and (a) stops at the first hit.
         uint32_t nfound = 0;
         for (uint32_t jb = 0; jb < nC; jb += 32) {
           const uint32_t j = jb + lane;
@@ -372,17 +382,25 @@ __global__ void __launch_bounds__(kRebuildWarps * 32) rebuild_kernel(const Rebui
           nfound += __popc(bal);
         }
         __syncwarp();
-        // each uncertain member f against every other candidate x; its row stays in registers
         for (uint32_t fi = 0; fi < nu; ++fi) {
           const uint32_t f = upos[fi];
+          const uint32_t fw = __shfl_sync(FULL, valid, f >> 5);
+          if (!((fw >> (f & 31)) & 1u)) continue;  // pruned by an earlier uncertain survivor
+          // once R valid candidates stand in front of f, neither f nor anything behind it reaches the row
+          uint32_t before = 0;
+          if ((uint32_t)lane < (f >> 5)) before = __popc(valid);
+          else if ((uint32_t)lane == (f >> 5)) before = __popc(valid & ((1u << (f & 31)) - 1u));
+          if (__reduce_add_sync(FULL, before) >= R) break;
           const unsigned long long kf = cs[f];
+          const Dist Df = key_dist<Dist>(kf);
           uint4 rf[CPL];
           load_row<G, CPL>(store + (size_t)key_id(kf) * row_bytes, nchunk, t, rf);
-          for (uint32_t xb = 0; xb < nC; xb += NT) {
+          bool pruned = false;
+          for (uint32_t xb = 0; xb < f && !pruned; xb += NT) {
             const uint32_t x = xb + team;
-            // skip self; a pair of two uncertain members is taken once, from its larger member
-            const unsigned long long kx = x < nC ? cs[x] : 0ull;
-            const bool act = x < nC && x != f && !(x > f && (kx & kExpandedBit));
+            const unsigned long long kx = x < f ? cs[x] : 0ull;
+            const uint32_t xw = __shfl_sync(FULL, valid, min(x, nC - 1u) >> 5);
+            const bool act = x < f && !(kx & kExpandedBit) && ((xw >> (x & 31)) & 1u);
             uint4 rx[CPL];
             if (act) {
               load_row<G, CPL>(store + (size_t)key_id(kx) * row_bytes, nchunk, t, rx);
@@ -391,17 +409,40 @@ __global__ void __launch_bounds__(kRebuildWarps * 32) rebuild_kernel(const Rebui
               for (int c = 0; c < CPL; ++c) rx[c] = make_uint4(0, 0, 0, 0);
             }
             const Dist d = team_dist_regs<T, kMetricL2, G, CPL>(rf, rx);  // bitwise symmetric in its operands
+            if (act && t == 0) ++npair;
+            if (__any_sync(FULL, act && alpha_test(ap, d, Df))) pruned = true;
+          }
+          if (pruned) {
+            if ((uint32_t)lane == (f >> 5)) valid &= ~(1u << (f & 31));
+            continue;
+          }
+          for (uint32_t xb = f + 1; xb < nC; xb += NT) {
+            const uint32_t x = xb + team;
+            const unsigned long long kx = x < nC ? cs[x] : 0ull;
+            const uint32_t xw = __shfl_sync(FULL, valid, min(x, nC - 1u) >> 5);
+            const bool act = x < nC && ((xw >> (x & 31)) & 1u);
+            uint4 rx[CPL];
+            if (act) {
+              load_row<G, CPL>(store + (size_t)key_id(kx) * row_bytes, nchunk, t, rx);
+            } else {
+#pragma unroll
+              for (int c = 0; c < CPL; ++c) rx[c] = make_uint4(0, 0, 0, 0);
+            }
+            const Dist d = team_dist_regs<T, kMetricL2, G, CPL>(rf, rx);
             if (act && t == 0) {
               ++npair;
-              const uint32_t i = min(f, x), j = max(f, x);
-              if (alpha_test(ap, d, key_dist<Dist>(x < f ? kf : kx))) {
-                atomicOr(&prune[i * W + (j >> 5)], 1u << (j & 31));
-                atomicOr(&hasp[i >> 5], 1u << (i & 31));
-              }
+              if (alpha_test(ap, d, key_dist<Dist>(kx))) atomicOr(&hasp[x >> 5], 1u << (x & 31));
             }
           }
+          __syncwarp();
+          if ((uint32_t)lane < W) {
+            valid &= ~hasp[lane];
+            hasp[lane] = 0u;
+          }
+          __syncwarp();
         }
       } else {
+        for (uint32_t w = lane; w < nC * W; w += 32) prune[w] = 0u;
         __syncwarp();
         const uint32_t npairs = nC * (nC - 1) / 2;
         for (uint32_t pb = 0; pb < npairs; pb += NT) {
@@ -416,25 +457,21 @@ __global__ void __launch_bounds__(kRebuildWarps * 32) rebuild_kernel(const Rebui
           }
           pair_test(act, i, j, jprev, rj);
         }
-      }
-      __syncwarp();
-      // ---- sequential selection replayed on bit masks (lane w holds word w of the valid set)
-      uint32_t valid = 0;
-      if ((uint32_t)lane < W) {
-        const uint32_t lo = lane * 32;
-        valid = nC >= lo + 32 ? 0xFFFFFFFFu : (nC > lo ? (1u << (nC - lo)) - 1u : 0u);
-      }
-      // The valid set only changes when a still-valid candidate with a non-zero matrix row is reached, so
-      // only those candidates are visited, in ascending order; everything valid in between is selected.
-      for (uint32_t w = 0; w < W; ++w) {
-        uint32_t hw = hasp[w];
-        while (hw) {
-          const uint32_t b = __ffs(hw) - 1;
-          hw &= hw - 1;
-          const uint32_t vw = __shfl_sync(FULL, valid, w);
-          if (((vw >> b) & 1u) && (uint32_t)lane < W) valid &= ~prune[(w * 32 + b) * W + lane];
+        __syncwarp();
+        // ---- sequential selection replayed on bit masks.  The valid set only changes when a still-valid
+        //      candidate with a non-zero matrix row is reached, so only those candidates are visited, in
+        //      ascending order; everything valid in between is selected.
+        for (uint32_t w = 0; w < W; ++w) {
+          uint32_t hw = hasp[w];
+          while (hw) {
+            const uint32_t b = __ffs(hw) - 1;
+            hw &= hw - 1;
+            const uint32_t vw = __shfl_sync(FULL, valid, w);
+            if (((vw >> b) & 1u) && (uint32_t)lane < W) valid &= ~prune[(w * 32 + b) * W + lane];
+          }
         }
       }
+      __syncwarp();
       // the first R members of the final valid set, in key order, are the new row
       uint32_t base_rank = 0;
       for (uint32_t sb = 0; sb < nC; sb += 32) {
