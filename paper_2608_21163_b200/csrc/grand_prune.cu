@@ -12,68 +12,54 @@ constexpr uint32_t kSegCap = 1024;   // request segment sorted in shared memory 
 constexpr uint32_t kMaxR = 128;
 
 // GrANDRobustPrune (Alg. 4) over candidate keys sorted ascending in shared memory.  The whole
-// block takes part.  Each iteration compacts the still-valid candidates into an index list, takes
-// its head as p*, and tests only the listed candidates against it (a team of G lanes per pair
-// distance).  Selected candidate indices go to out_idx; returns how many were selected.
+// block takes part.  The candidates are taken in key order and each is asked the one question the
+// sequential algorithm ever asks about it: does a member selected so far prune it
+// (alpha * dist(s, c) <= D_p[c])?  If none does, it is selected.  That is the same result as "select
+// the closest valid candidate, invalidate what it prunes", but a candidate costs at most as many
+// tests as there are selected members, the first hit ends it, and nothing behind the R-th selected
+// member is ever looked at.  A team of G lanes takes one selected member per pass.
+// Selected candidate indices go to out_idx; returns how many were selected.
 template <typename T, int G, int CPL>
 __device__ uint32_t block_prune(const uint8_t* __restrict__ store, uint32_t row_bytes, uint32_t nchunk, const AlphaParam ap,
-                                const unsigned long long* cand, uint32_t n, uint32_t R, uint32_t* validw, uint32_t* vlist,
-                                uint32_t* out_idx, volatile uint32_t* sh_sel, unsigned long long& npair) {
+                                const unsigned long long* cand, uint32_t n, uint32_t R, uint32_t* out_idx,
+                                unsigned long long& npair) {
   using Dist = typename Elem<T>::Dist;
   const uint32_t tid = threadIdx.x, nthreads = blockDim.x;
   const int lane = tid & 31, warp = tid >> 5;
   const int t = lane % G;
-  const uint32_t team_global = tid / G, nteams = nthreads / G;
-  const uint32_t nwords = (n + 31) >> 5;
-  for (uint32_t w = tid; w < nwords; w += nthreads)
-    validw[w] = (w * 32 + 32 <= n) ? 0xFFFFFFFFu : ((1u << (n - w * 32)) - 1u);
-  __syncthreads();
+  const uint32_t team_global = tid / G, nteams = nthreads / G, teams_per_warp = 32u / G;
   uint32_t cnt = 0;
-  for (;;) {
-    if (warp == 0) {  // compact the valid set (ascending); p* = its head
-      uint32_t nv = 0;
-      for (uint32_t wd = 0; wd < nwords; ++wd) {
-        const uint32_t bits = validw[wd];
-        if ((bits >> lane) & 1u) vlist[nv + __popc(bits & ((1u << lane) - 1u))] = wd * 32 + lane;
-        nv += __popc(bits);
-      }
-      __syncwarp();
-      if (lane == 0) {
-        const uint32_t s = nv ? vlist[0] : kInvalid;
-        sh_sel[0] = s;
-        sh_sel[1] = nv;
-        if (s != kInvalid) {
-          out_idx[cnt] = s;
-          validw[s >> 5] &= ~(1u << (s & 31));
-        }
-      }
-    }
-    __syncthreads();
-    const uint32_t s = sh_sel[0], nv = sh_sel[1];
-    if (s == kInvalid) break;
-    ++cnt;
-    if (cnt == R) break;
-    // invalidate every remaining p' with alpha * dist(p*, p') <= D_p[p']: only live candidates are visited
-    uint4 pstar[CPL];
-    load_row<G, CPL>(store + (size_t)key_id(cand[s]) * row_bytes, nchunk, t, pstar);
-    for (uint32_t jb = 1; jb < nv; jb += nteams) {
-      const uint32_t kk = jb + team_global;
-      const bool act = kk < nv;
-      const uint32_t j = act ? vlist[kk] : 0u;
-      uint4 v[CPL];
-      if (act) {
-        load_row<G, CPL>(store + (size_t)key_id(cand[j]) * row_bytes, nchunk, t, v);
-      } else {
+  for (uint32_t c = 0; c < n && cnt < R; ++c) {
+    const unsigned long long kc = cand[c];
+    const Dist Dc = key_dist<Dist>(kc);
+    bool pruned = false;
+    if (cnt) {
+      uint4 rc[CPL];
+      load_row<G, CPL>(store + (size_t)key_id(kc) * row_bytes, nchunk, t, rc);
+      for (uint32_t sb = 0; sb < cnt && !pruned; sb += nteams) {
+        bool hit = false;
+        if (sb + (uint32_t)warp * teams_per_warp < cnt) {  // (a warp without a member to test only joins the vote)
+          const uint32_t sidx = sb + team_global;
+          const bool act = sidx < cnt;
+          uint4 rs[CPL];
+          if (act) {
+            load_row<G, CPL>(store + (size_t)key_id(cand[out_idx[sidx]]) * row_bytes, nchunk, t, rs);
+          } else {
 #pragma unroll
-        for (int c = 0; c < CPL; ++c) v[c] = make_uint4(0, 0, 0, 0);
-      }
-      const Dist d = team_dist_regs<T, kMetricL2, G, CPL>(pstar, v);
-      if (act && t == 0) {
-        ++npair;
-        if (alpha_test(ap, d, key_dist<Dist>(cand[j]))) atomicAnd(&validw[j >> 5], ~(1u << (j & 31)));
+            for (int cc = 0; cc < CPL; ++cc) rs[cc] = make_uint4(0, 0, 0, 0);
+          }
+          const Dist d = team_dist_regs<T, kMetricL2, G, CPL>(rs, rc);
+          if (act && t == 0) ++npair;
+          hit = act && alpha_test(ap, d, Dc);
+        }
+        pruned = __syncthreads_or(hit) != 0;
       }
     }
-    __syncthreads();
+    if (!pruned) {
+      if (tid == 0) out_idx[cnt] = c;
+      ++cnt;
+      __syncthreads();  // the new member is visible before the next candidate's tests read the list
+    }
   }
   __syncthreads();
   return cnt;
@@ -82,10 +68,7 @@ __device__ uint32_t block_prune(const uint8_t* __restrict__ store, uint32_t row_
 template <typename T, int METRIC, int G, int CPL>
 __global__ void __launch_bounds__(kPruneThreads) forward_prune_kernel(const PruneArgs a) {
   __shared__ unsigned long long cand[kMaxCand];
-  __shared__ uint32_t validw[kMaxCand / 32];
-  __shared__ uint32_t vlist[kMaxCand];
   __shared__ uint32_t out_idx[kMaxR];
-  __shared__ uint32_t sh_sel[2];
   const uint32_t tid = threadIdx.x, nthreads = blockDim.x;
   const uint32_t R = a.g.R;
   const AlphaParam ap{a.A_fix, a.alpha};
@@ -109,7 +92,7 @@ __global__ void __launch_bounds__(kPruneThreads) forward_prune_kernel(const Prun
       for (uint32_t j = tid; j < cnt; j += nthreads) out_idx[j] = j;
       __syncthreads();
     } else {
-      cnt = block_prune<T, G, CPL>(a.g.store, a.lay.row_bytes, a.lay.nchunk, ap, cand, n, R, validw, vlist, out_idx, sh_sel, npair);
+      cnt = block_prune<T, G, CPL>(a.g.store, a.lay.row_bytes, a.lay.nchunk, ap, cand, n, R, out_idx, npair);
       ++nprune;
     }
     for (uint32_t s = tid; s < R; s += nthreads) {
@@ -139,9 +122,111 @@ __global__ void __launch_bounds__(kPruneThreads) forward_prune_kernel(const Prun
   if (tid == 0 && nprune) atomicAdd(&a.state->counters[CTR_PRUNE], (unsigned long long)nprune);
 }
 
+// The same candidate-ordered prune with one WARP per node, for short rows: a row of a few chunks keeps only a
+// few lanes busy per test, the tests of one candidate are few, and a block would spend its time in barriers.
+constexpr uint32_t kWarpPruneCand = 256;  // candidates per node this kernel accepts (shared memory per warp)
+constexpr int kWarpPruneWarps = 4;
+
+template <typename T, int G, int CPL>
+__global__ void __launch_bounds__(kWarpPruneWarps * 32) forward_prune_warp_kernel(const PruneArgs a) {
+  using Dist = typename Elem<T>::Dist;
+  constexpr unsigned FULL = 0xFFFFFFFFu;
+  constexpr int NT = 32 / G;
+  __shared__ unsigned long long cand_s[kWarpPruneWarps][kWarpPruneCand];
+  __shared__ uint32_t out_s[kWarpPruneWarps][kMaxR];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int t = lane % G, team = lane / G;
+  unsigned long long* cand = cand_s[warp];
+  uint32_t* out_idx = out_s[warp];
+  const uint32_t R = a.g.R, row_bytes = a.lay.row_bytes, nchunk = a.lay.nchunk;
+  const uint8_t* __restrict__ store = a.g.store;
+  const AlphaParam ap{a.A_fix, a.alpha};
+  unsigned long long npair = 0;
+  uint32_t nprune = 0;
+  auto wsync = [] { __syncwarp(); };
+  // (handing the nodes out through a counter was measured and is slower than this fixed assignment)
+  const uint64_t wglobal = (uint64_t)blockIdx.x * kWarpPruneWarps + warp, wtotal = (uint64_t)gridDim.x * kWarpPruneWarps;
+  for (uint64_t i = wglobal; i < a.n; i += wtotal) {
+    const uint32_t p = a.ids[i];
+    const uint32_t nc = min(min(a.cand_n[i], a.cand_stride), kWarpPruneCand);
+    for (uint32_t j = lane; j < nc; j += 32) {
+      const unsigned long long k = a.cand[i * a.cand_stride + j];
+      cand[j] = key_id(k) == p ? kKeyMax : k;
+    }
+    __syncwarp();
+    bitonic_sort_any(cand, nc, (uint32_t)lane, 32u, wsync);
+    uint32_t n = nc;
+    while (n > 0 && cand[n - 1] == kKeyMax) --n;
+    uint32_t cnt = 0;
+    for (uint32_t c = 0; c < n && cnt < R; ++c) {
+      const unsigned long long kc = cand[c];
+      const Dist Dc = key_dist<Dist>(kc);
+      bool pruned = false;
+      if (cnt) {
+        uint4 rc[CPL];
+        load_row<G, CPL>(store + (size_t)key_id(kc) * row_bytes, nchunk, t, rc);
+        for (uint32_t sb = 0; sb < cnt && !pruned; sb += NT) {
+          const uint32_t sidx = sb + team;
+          const bool act = sidx < cnt;
+          uint4 rs[CPL];
+          if (act) {
+            load_row<G, CPL>(store + (size_t)key_id(cand[out_idx[sidx]]) * row_bytes, nchunk, t, rs);
+          } else {
+#pragma unroll
+            for (int cc = 0; cc < CPL; ++cc) rs[cc] = make_uint4(0, 0, 0, 0);
+          }
+          const Dist d = team_dist_regs<T, kMetricL2, G, CPL>(rs, rc);
+          if (act && t == 0) ++npair;
+          if (__any_sync(FULL, act && alpha_test(ap, d, Dc))) pruned = true;
+        }
+      }
+      if (!pruned) {
+        if (lane == 0) out_idx[cnt] = c;
+        ++cnt;
+        __syncwarp();
+      }
+    }
+    ++nprune;
+    for (uint32_t sl = lane; sl < R; sl += 32) {
+      uint32_t id = kInvalid, db = kInvalid;
+      unsigned long long rk = 0;
+      if (sl < cnt) {
+        const unsigned long long k = cand[out_idx[sl]];
+        id = key_id(k);
+        rk = (k & 0xFFFFFFFF00000000ull) | p;  // dist(p, id) is symmetric: the request carries it
+        db = (uint32_t)(k >> 32);
+      }
+      a.g.adj[(size_t)p * R + sl] = id;
+      if (a.g.rowd) a.g.rowd[(size_t)p * R + sl] = db;
+      a.req_tgt[i * R + sl] = id;
+      a.req_key[i * R + sl] = rk;
+    }
+    if (lane == 0) {
+      a.g.deg[p] = cnt;
+      a.g.rowpfx[p] = (uint8_t)cnt;
+      if (a.g.birth) {
+        a.g.birth[p] = a.g.epoch;
+        a.g.rowepoch[p] = a.g.epoch;
+      }
+    }
+    __syncwarp();
+  }
+  if (npair) atomicAdd(&a.state->counters[CTR_PAIR], npair);
+  if (lane == 0 && nprune) atomicAdd(&a.state->counters[CTR_PRUNE], (unsigned long long)nprune);
+}
+
 template <typename T, int METRIC, int G, int CPL>
 static cudaError_t launch_forward_prune_t(const PruneArgs& a, cudaStream_t s) {
   if (a.n == 0) return cudaSuccess;
+  if constexpr (G * CPL <= 16) {
+    if (!a.fixed_mode && a.cand_stride <= kWarpPruneCand) {
+      const uint64_t want = (a.n + kWarpPruneWarps - 1) / kWarpPruneWarps;
+      const unsigned blocks = (unsigned)(want < 148u * 16u ? want : 148u * 16u);
+      forward_prune_warp_kernel<T, G, CPL><<<blocks, kWarpPruneWarps * 32, 0, s>>>(a);
+      count_launches(1);
+      return cudaGetLastError();
+    }
+  }
   const unsigned blocks = (unsigned)(a.n < 148u * 16u ? a.n : 148u * 16u);
   forward_prune_kernel<T, METRIC, G, CPL><<<blocks, kPruneThreads, 0, s>>>(a);
   count_launches(1);
