@@ -154,22 +154,29 @@ cudaError_t launch_exclusive_scan(const uint32_t* in, uint32_t* out, uint64_t n,
 // ---- reverse graph
 // `heads` (optional bitmap): only edges whose head is marked are counted / scattered, i.e. only the
 // in-neighbour rows of the marked nodes are materialised (the delete path reads no other row).
+// One warp per adjacency row (a coalesced read of the row, its degree fetched once, no index arithmetic per edge).
 __global__ void transpose_hist_kernel(const GraphView g, uint32_t* indeg, const uint32_t* heads) {
-  const uint64_t total = g.cap * g.R;
-  for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < total; i += (uint64_t)gridDim.x * blockDim.x) {
-    const uint64_t v = i / g.R;
-    if ((uint32_t)(i - v * g.R) >= g.deg[v]) continue;
-    const uint32_t z = g.adj[i];
-    if (!heads || bit_test(heads, z)) atomicAdd(&indeg[z], 1u);
+  const int lane = threadIdx.x & 31;
+  const uint64_t wglobal = (blockIdx.x * (uint64_t)blockDim.x + threadIdx.x) >> 5;
+  const uint64_t wtotal = ((uint64_t)gridDim.x * blockDim.x) >> 5;
+  for (uint64_t v = wglobal; v < g.cap; v += wtotal) {
+    const uint32_t dv = min(g.deg[v], g.R);
+    for (uint32_t sl = lane; sl < dv; sl += 32) {
+      const uint32_t z = g.adj[v * g.R + sl];
+      if (!heads || bit_test(heads, z)) atomicAdd(&indeg[z], 1u);
+    }
   }
 }
 __global__ void transpose_scatter_kernel(const GraphView g, const uint32_t* off, uint32_t* fillc, uint32_t* src, const uint32_t* heads) {
-  const uint64_t total = g.cap * g.R;
-  for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < total; i += (uint64_t)gridDim.x * blockDim.x) {
-    const uint64_t v = i / g.R;
-    if ((uint32_t)(i - v * g.R) >= g.deg[v]) continue;
-    const uint32_t z = g.adj[i];
-    if (!heads || bit_test(heads, z)) src[off[z] + atomicAdd(&fillc[z], 1u)] = (uint32_t)v;
+  const int lane = threadIdx.x & 31;
+  const uint64_t wglobal = (blockIdx.x * (uint64_t)blockDim.x + threadIdx.x) >> 5;
+  const uint64_t wtotal = ((uint64_t)gridDim.x * blockDim.x) >> 5;
+  for (uint64_t v = wglobal; v < g.cap; v += wtotal) {
+    const uint32_t dv = min(g.deg[v], g.R);
+    for (uint32_t sl = lane; sl < dv; sl += 32) {
+      const uint32_t z = g.adj[v * g.R + sl];
+      if (!heads || bit_test(heads, z)) src[off[z] + atomicAdd(&fillc[z], 1u)] = (uint32_t)v;
+    }
   }
 }
 // ascending rows: shared-memory sort for short rows, in place in global memory for long ones
@@ -194,13 +201,13 @@ __global__ void __launch_bounds__(128) transpose_sort_rows_kernel(uint64_t cap, 
 cudaError_t launch_transpose(const TransposeArgs& a, cudaStream_t s) {
   const uint64_t cap = a.g.cap;
   cudaMemsetAsync(a.indeg, 0, (cap + 1) * 4, s);
-  transpose_hist_kernel<<<grid_for(cap * a.g.R), kThreads, 0, s>>>(a.g, a.indeg, a.heads);
+  transpose_hist_kernel<<<grid_for(cap * 32), kThreads, 0, s>>>(a.g, a.indeg, a.heads);
   count_launches(1);
   cudaError_t e = launch_exclusive_scan(a.indeg, a.off, cap + 1, a.scan_tmp, s);
   if (e != cudaSuccess) return e;
   if (a.src) {
     cudaMemsetAsync(a.fillc, 0, cap * 4, s);
-    transpose_scatter_kernel<<<grid_for(cap * a.g.R), kThreads, 0, s>>>(a.g, a.off, a.fillc, a.src, a.heads);
+    transpose_scatter_kernel<<<grid_for(cap * 32), kThreads, 0, s>>>(a.g, a.off, a.fillc, a.src, a.heads);
     count_launches(a.sort_rows ? 2 : 1);
     if (a.sort_rows) transpose_sort_rows_kernel<<<(unsigned)(cap < 148u * 16u ? cap : 148u * 16u), 128, 0, s>>>(cap, a.off, a.src);
   }
