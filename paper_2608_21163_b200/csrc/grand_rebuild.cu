@@ -366,7 +366,7 @@ __global__ void __launch_bounds__(kRebuildWarps * 32) rebuild_kernel(const Rebui
       uint4 rj[CPL];
 #pragma unroll
       for (int c = 0; c < CPL; ++c) rj[c] = make_uint4(0, 0, 0, 0);
-      if (nu <= 2 * P) {  // (the list of uncertain positions holds 2P entries)
+      if (nu <= 2 * P && kpe == kp) {  // (the list of uncertain positions holds 2P entries; the tags must be trusted)
         // ---- few uncertain members among a pruned run.  Members of the run never prune each other, so the
         //      sequential prune only ever changes at an uncertain member f, and those are taken in key order:
         //      (a) does a valid member of the run in front of f prune it (earlier uncertain survivors have
@@ -382,7 +382,7 @@ __global__ void __launch_bounds__(kRebuildWarps * 32) rebuild_kernel(const Rebui
           nfound += __popc(bal);
         }
         __syncwarp();
-        for (uint32_t fi = 0; fi < nu; ++fi) {
+        for (uint32_t fi = 0; fi < nfound; ++fi) {
           const uint32_t f = upos[fi];
           const uint32_t fw = __shfl_sync(FULL, valid, f >> 5);
           if (!((fw >> (f & 31)) & 1u)) continue;  // pruned by an earlier uncertain survivor

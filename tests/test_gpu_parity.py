@@ -65,6 +65,31 @@ def test_search_bit_exact_on_oracle_graph(dim, dtype):
         assert (od == gd.astype(np.float64)).all()
 
 
+def test_updates_continue_bit_exact_on_an_imported_graph():
+    """An imported graph carries no cached distances and no pruned-run lengths: every row entry is of unknown
+    standing when its node is next rebuilt.  Inserts, deletes and re-inserts then have to match the oracle, which
+    kept the same graph all along."""
+    torch = torch_()
+    n, dim, R, L = 6000, 32, 16, 32
+    base = synth.uniform_u8(7, "base", 0, n, dim)
+    cfg = dict(dim=dim, dtype=go.U8, metric=go.L2, R=R, L=L, alpha=1.2, mode=go.VAMANA, max_build_batch=500, ins=500, dele=500)
+    o, g = make_pair(cfg, n)
+    for lo in range(0, 4000, 500):
+        o.insert_batch(np.arange(lo, lo + 500, dtype=np.uint32), base[lo:lo + 500])
+    import_from_oracle(o, g, base)
+    assert_same_graph(o, g, "import")
+    alive = np.zeros(n, bool); alive[:4000] = True
+    for r in range(4):
+        ids = np.arange(4000 + 500 * r, 4500 + 500 * r, dtype=np.uint32)
+        o.insert_batch(ids, base[ids]); g.insert_batch(torch.from_numpy(ids), torch.from_numpy(base[ids]))
+        alive[ids] = True
+        assert_same_graph(o, g, f"insert {r} after import")
+        dele = synth.choose_ids(7, f"del/{r}", np.flatnonzero(alive).astype(np.uint32), 500)
+        o.delete_batch(dele); g.delete_batch(torch.from_numpy(dele))
+        alive[dele] = False
+        assert_same_graph(o, g, f"delete {r} after import")
+
+
 def test_search_fp32_tolerance_and_ip():
     n, dim, R, L = 4000, 96, 24, 64
     base = synth.gaussian_unit_f32(2, "base", 0, n, dim)
