@@ -250,6 +250,7 @@ __global__ void __launch_bounds__(kPickWarps * 32) delete_picks_staged_kernel(co
   uint4* xb = reinterpret_cast<uint4*>(ckeys + ((kr + 1u) & ~1u) + (size_t)kPickWarps * kMaxKRepair) + (size_t)warp * nchunk;  // x's row
   int* cnorm = reinterpret_cast<int*>(reinterpret_cast<uint4*>(ckeys + ((kr + 1u) & ~1u) + (size_t)kPickWarps * kMaxKRepair) +
                                       (size_t)kPickWarps * nchunk);  // |y|^2 of the staged rows (integer rows only)
+  uint32_t* xid = reinterpret_cast<uint32_t*>(cnorm + kr);  // the unit's x ids (invalid id = nothing to do for the pair)
   const uint32_t nunits = a.unit_off[a.n];
   unsigned long long npair = 0;
   for (uint32_t unit = blockIdx.x; unit < nunits; unit += gridDim.x) {
@@ -269,6 +270,21 @@ __global__ void __launch_bounds__(kPickWarps * 32) delete_picks_staged_kernel(co
       const uint32_t y = key_id(a.Ci[(size_t)i * kr + j]);
       reinterpret_cast<uint4*>(crow + (size_t)j * rs)[ch] = __ldg(reinterpret_cast<const uint4*>(a.g.store + (size_t)y * row_bytes) + ch);
     }
+    // the unit's x ids, resolved by the whole block at once (id, batch and liveness bits are dependent loads that a
+    // warp would otherwise wait for pair by pair), and their vectors requested towards L2
+    for (uint32_t j = threadIdx.x; j < q1 - q0; j += blockDim.x) {
+      const uint32_t q = q0 + j;
+      uint32_t x = kInvalid;
+      if (q < nin) {
+        x = a.src[in_base(a, i) + q];
+      } else if (q - nin < a.g.deg[p]) {
+        x = a.g.adj[(size_t)p * R + (q - nin)];
+      }
+      if (x != kInvalid && (bit_test(a.delmap, x) || (a.livemap && !bit_test(a.livemap, x)))) x = kInvalid;
+      xid[j] = x;
+      if (x != kInvalid)
+        for (uint32_t b = 0; b < row_bytes; b += 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(a.g.store + (size_t)x * row_bytes + b));
+    }
     __syncthreads();
     if constexpr (sizeof(T) == 1) {
       // |x - y|^2 = |x|^2 + |y|^2 - 2 x.y in exact integers: the pair loop then needs one dp4a per word, not two
@@ -282,17 +298,9 @@ __global__ void __launch_bounds__(kPickWarps * 32) delete_picks_staged_kernel(co
     }
     for (uint32_t q = q0 + warp; q < q1; q += kPickWarps) {
       const bool is_in = q < nin;
-      uint32_t x = kInvalid;
-      uint64_t rbase;
-      if (is_in) {
-        x = a.src[in_base(a, i) + q];
-        rbase = ((uint64_t)a.pair_off[i] + q) * c;
-      } else {
-        const uint32_t sl = q - nin;
-        if (sl < a.g.deg[p]) x = a.g.adj[(size_t)p * R + sl];
-        rbase = (total_in + (uint64_t)i * R + sl) * c;
-      }
-      if (x == kInvalid || bit_test(a.delmap, x) || (a.livemap && !bit_test(a.livemap, x))) {
+      const uint32_t x = xid[q - q0];
+      const uint64_t rbase = is_in ? ((uint64_t)a.pair_off[i] + q) * c : (total_in + (uint64_t)i * R + (q - nin)) * c;
+      if (x == kInvalid) {
         if (lane < c) a.req_tgt[rbase + lane] = kInvalid;
         continue;
       }
@@ -414,7 +422,7 @@ static cudaError_t launch_delete_picks_t(const DeleteArgs& a, uint64_t total_in,
   if (stage <= 64 * 1024) {
     // candidate rows fit shared memory: one staged copy per work unit
     const size_t smem = stage + ((size_t)((a.k_repair + 1u) & ~1u) + (size_t)kPickWarps * kMaxKRepair) * 8 +
-                        (size_t)kPickWarps * a.lay.row_bytes + (size_t)a.k_repair * 4;
+                        (size_t)kPickWarps * a.lay.row_bytes + (size_t)a.k_repair * 4 + (size_t)kUnitPairs * 4;
     auto kern = delete_picks_staged_kernel<T, METRIC, G, CPL>;
     static size_t smem_set = 0;
     if (smem > smem_set) {
