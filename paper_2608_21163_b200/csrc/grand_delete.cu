@@ -223,10 +223,10 @@ __global__ void delete_touch_kernel(const DeleteArgs a, const uint64_t total_in)
 // shared memory once and its warps run the pairs of that node against the copy.  Work units are
 // chunks of kUnitPairs pairs of one node (hubs with long in-neighbour rows are split over blocks).
 constexpr uint32_t kUnitPairs = 256;
-__global__ void delete_units_kernel(const DeleteArgs a) {
+__global__ void delete_units_kernel(const DeleteArgs a, const uint32_t unit_pairs) {
   for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i <= a.n; i += (uint64_t)gridDim.x * blockDim.x) {
     uint32_t units = 0;
-    if (i < a.n) units = (a.pair_off[i + 1] - a.pair_off[i] + a.g.R + kUnitPairs - 1) / kUnitPairs;
+    if (i < a.n) units = (a.pair_off[i + 1] - a.pair_off[i] + a.g.R + unit_pairs - 1) / unit_pairs;
     a.in_cnt[i] = units;  // the in-degree counts are not needed once their prefix exists
   }
 }
@@ -408,6 +408,169 @@ __global__ void __launch_bounds__(kPickWarps * 32) delete_picks_staged_kernel(co
   if (npair) atomicAdd(&a.state->counters[CTR_PAIR], npair);
 }
 
+// ---- tensor-core variant for integer rows.  All pairs (x, y) of one deleted node, x among its surviving in- and
+// out-neighbours and y in C_i, need dist(x, y): a dense cross-distance block.  With
+// |x - y|^2 = |x|^2 + |y|^2 - 2 x.y the cross term is an integer matrix product X * C_i^T, exact in int32, which
+// the tensor cores take as 8-bit mma tiles (m16n8k32).  A work unit is up to kMmaUnitPairs rows of X for one node:
+// the block stages the unit's x rows and the candidate rows (zero-padded to 32-byte steps, on a stride that keeps
+// the fragment loads free of bank conflicts), each warp multiplies 16-row tiles against all candidate tiles and
+// then picks the c smallest (dist, id) per row out of the accumulators.
+constexpr uint32_t kMmaUnitPairs = 128;
+constexpr int kMmaNTiles = 7;  // candidate tiles of 8: k_repair <= 56
+constexpr int kMmaWarps = 4;
+
+template <typename T>
+__device__ __forceinline__ void mma_m16n8k32(int (&d)[4], const uint32_t (&x)[4], const uint32_t (&y)[2]) {
+  if constexpr (T(-1) < T(0)) {
+    asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+                 : "r"(x[0]), "r"(x[1]), "r"(x[2]), "r"(x[3]), "r"(y[0]), "r"(y[1]));
+  } else {
+    asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+                 : "r"(x[0]), "r"(x[1]), "r"(x[2]), "r"(x[3]), "r"(y[0]), "r"(y[1]));
+  }
+}
+
+static size_t delete_picks_mma_smem(uint32_t row_bytes) {
+  const size_t rs = ((row_bytes + 31u) & ~31u) + 16u;
+  return (size_t)(kMmaUnitPairs + kMmaNTiles * 8) * rs + (size_t)kMmaNTiles * 8 * 12 + (size_t)kMmaUnitPairs * 8;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kMmaWarps * 32) delete_picks_mma_kernel(const DeleteArgs a, const uint64_t total_in) {
+  constexpr unsigned FULL = 0xFFFFFFFFu;
+  constexpr uint32_t NC = kMmaNTiles * 8;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int gid = lane >> 2, tig = lane & 3;
+  const uint32_t R = a.g.R, c = a.c, kr = a.k_repair;
+  const uint32_t row_bytes = a.lay.row_bytes, nchunk = a.lay.nchunk;
+  const uint32_t kb = (row_bytes + 31u) & ~31u, rs = kb + 16u, kch = kb / 16u, ksteps = kb / 32u;
+  uint8_t* xrow = smem_raw;                                   // kMmaUnitPairs rows of X
+  uint8_t* crow = xrow + (size_t)kMmaUnitPairs * rs;          // NC candidate rows
+  unsigned long long* ckeys = reinterpret_cast<unsigned long long*>(crow + (size_t)NC * rs);
+  int* cnorm = reinterpret_cast<int*>(ckeys + NC);
+  int* xnorm = cnorm + NC;
+  uint32_t* xid = reinterpret_cast<uint32_t*>(xnorm + kMmaUnitPairs);
+  const uint32_t nunits = a.unit_off[a.n];
+  unsigned long long npair = 0;
+  for (uint32_t unit = blockIdx.x; unit < nunits; unit += gridDim.x) {
+    uint32_t lo = 0, hi = (uint32_t)a.n;  // largest i with unit_off[i] <= unit
+    while (hi - lo > 1) {
+      const uint32_t mid = (lo + hi) >> 1;
+      if (a.unit_off[mid] <= unit) lo = mid; else hi = mid;
+    }
+    const uint32_t i = lo, p = a.ids[i];
+    const uint32_t nin = a.pair_off[i + 1] - a.pair_off[i];
+    const uint32_t q0 = (unit - a.unit_off[i]) * kMmaUnitPairs, q1 = min(nin + R, q0 + kMmaUnitPairs);
+    const uint32_t M = q1 - q0, nc = min(a.Ci_n[i], NC);
+    __syncthreads();  // the previous unit's readers are done with the staged rows
+    for (uint32_t j = threadIdx.x; j < NC; j += blockDim.x) ckeys[j] = j < nc ? a.Ci[(size_t)i * kr + j] : kKeyMax;
+    for (uint32_t e = threadIdx.x; e < NC * kch; e += blockDim.x) {
+      const uint32_t j = e / kch, ch = e - j * kch;
+      uint4 v = make_uint4(0, 0, 0, 0);
+      if (j < nc && ch < nchunk)
+        v = __ldg(reinterpret_cast<const uint4*>(a.g.store + (size_t)key_id(a.Ci[(size_t)i * kr + j]) * row_bytes) + ch);
+      reinterpret_cast<uint4*>(crow + (size_t)j * rs)[ch] = v;
+    }
+    for (uint32_t j = threadIdx.x; j < kMmaUnitPairs; j += blockDim.x) {
+      const uint32_t q = q0 + j;
+      uint32_t x = kInvalid;
+      if (j < M) {
+        if (q < nin) {
+          x = a.src[in_base(a, i) + q];
+        } else if (q - nin < a.g.deg[p]) {
+          x = a.g.adj[(size_t)p * R + (q - nin)];
+        }
+        if (x != kInvalid && (bit_test(a.delmap, x) || (a.livemap && !bit_test(a.livemap, x)))) x = kInvalid;
+      }
+      xid[j] = x;
+    }
+    __syncthreads();
+    for (uint32_t e = threadIdx.x; e < kMmaUnitPairs * kch; e += blockDim.x) {
+      const uint32_t j = e / kch, ch = e - j * kch;
+      const uint32_t x = xid[j];
+      uint4 v = make_uint4(0, 0, 0, 0);
+      if (x != kInvalid && ch < nchunk) v = __ldg(reinterpret_cast<const uint4*>(a.g.store + (size_t)x * row_bytes) + ch);
+      reinterpret_cast<uint4*>(xrow + (size_t)j * rs)[ch] = v;
+    }
+    __syncthreads();
+    for (uint32_t j = threadIdx.x; j < kMmaUnitPairs + NC; j += blockDim.x) {  // squared norms of all staged rows
+      const uint4* rp = reinterpret_cast<const uint4*>(j < kMmaUnitPairs ? xrow + (size_t)j * rs : crow + (size_t)(j - kMmaUnitPairs) * rs);
+      int acc = 0;
+      for (uint32_t ch = 0; ch < nchunk; ++ch) acc_chunk<T, kMetricIP>(rp[ch], rp[ch], acc);
+      if (j < kMmaUnitPairs) xnorm[j] = acc; else cnorm[j - kMmaUnitPairs] = acc;
+    }
+    __syncthreads();
+    for (uint32_t mt = warp; mt * 16u < M; mt += kMmaWarps) {
+      int acc[kMmaNTiles][4];
+#pragma unroll
+      for (int nt = 0; nt < kMmaNTiles; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0;
+      const uint8_t* xr0 = xrow + (size_t)(mt * 16u + gid) * rs + tig * 4;
+      const uint8_t* xr1 = xr0 + 8 * (size_t)rs;
+      const uint8_t* cr = crow + (size_t)gid * rs + tig * 4;
+      for (uint32_t ks = 0; ks < ksteps; ++ks) {
+        uint32_t xa[4];
+        xa[0] = *reinterpret_cast<const uint32_t*>(xr0 + ks * 32);
+        xa[1] = *reinterpret_cast<const uint32_t*>(xr1 + ks * 32);
+        xa[2] = *reinterpret_cast<const uint32_t*>(xr0 + ks * 32 + 16);
+        xa[3] = *reinterpret_cast<const uint32_t*>(xr1 + ks * 32 + 16);
+#pragma unroll
+        for (int nt = 0; nt < kMmaNTiles; ++nt) {
+          uint32_t yb[2];
+          yb[0] = *reinterpret_cast<const uint32_t*>(cr + (size_t)nt * 8 * rs + ks * 32);
+          yb[1] = *reinterpret_cast<const uint32_t*>(cr + (size_t)nt * 8 * rs + ks * 32 + 16);
+          mma_m16n8k32<T>(acc[nt], xa, yb);
+        }
+      }
+      // accumulator element (nt, h * 2 + jj) of this lane: row mt * 16 + gid + 8 h, candidate nt * 8 + tig * 2 + jj
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const uint32_t r = mt * 16u + gid + 8u * h;
+        const uint32_t x = xid[r];
+        const int xn = xnorm[r];
+        const uint32_t q = q0 + r;
+        const bool is_in = q < nin;
+        const uint64_t rbase = is_in ? ((uint64_t)a.pair_off[i] + q) * c : (total_in + (uint64_t)i * R + (q - nin)) * c;
+        unsigned long long prev = 0;  // every key is larger (order-preserving distance bits are non-zero)
+        for (uint32_t round = 0; round < c; ++round) {
+          unsigned long long best = kKeyMax;  // smallest key above the previous round's pick
+#pragma unroll
+          for (int nt = 0; nt < kMmaNTiles; ++nt) {
+#pragma unroll
+            for (int jj = 0; jj < 2; ++jj) {
+              const uint32_t n = nt * 8 + tig * 2 + jj;
+              const unsigned long long kc = ckeys[n];
+              const uint32_t y = key_id(kc);
+              if (kc != kKeyMax && y != x) {
+                const unsigned long long key = make_key(xn + cnorm[n] - 2 * acc[nt][h * 2 + jj], y);
+                if (key > prev && key < best) best = key;
+              }
+            }
+          }
+          best = min(best, __shfl_xor_sync(FULL, best, 1));
+          best = min(best, __shfl_xor_sync(FULL, best, 2));
+          if (tig == 0 && r < M) {
+            if (x == kInvalid || best == kKeyMax) {
+              a.req_tgt[rbase + round] = kInvalid;
+            } else if (is_in) {
+              a.req_tgt[rbase + round] = x;
+              a.req_key[rbase + round] = best;
+            } else {
+              a.req_tgt[rbase + round] = key_id(best);
+              a.req_key[rbase + round] = (best & 0xFFFFFFFF00000000ull) | x;
+            }
+          }
+          prev = best;
+        }
+        if (tig == 0 && r < M && x != kInvalid) npair += nc;
+      }
+    }
+  }
+  if (npair) atomicAdd(&a.state->counters[CTR_PAIR], npair);
+}
+
 template <typename T, int METRIC, int G, int CPL>
 static cudaError_t launch_delete_picks_t(const DeleteArgs& a, uint64_t total_in, cudaStream_t s) {
   const uint64_t total = total_in + a.n * a.g.R;
@@ -417,6 +580,28 @@ static cudaError_t launch_delete_picks_t(const DeleteArgs& a, uint64_t total_in,
     if (tb > 148u * 32u) tb = 148u * 32u;
     delete_touch_kernel<<<(unsigned)tb, 256, 0, s>>>(a, total_in);
     count_launches(1);
+  }
+  if constexpr (sizeof(T) == 1) {
+    if (a.k_repair <= (uint32_t)kMmaNTiles * 8u && a.lay.row_bytes <= 256u) {
+      const size_t smem = delete_picks_mma_smem(a.lay.row_bytes);
+      auto kern = delete_picks_mma_kernel<T>;
+      // (one kernel serves every row layout of this element type, so the limit is raised once, to the largest case)
+      static bool smem_set = false;
+      if (!smem_set) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)delete_picks_mma_smem(256u));
+        if (e != cudaSuccess) return e;
+        smem_set = true;
+      }
+      const unsigned ub = (unsigned)((a.n + 256) / 256 > 148u * 16u ? 148u * 16u : (a.n + 256) / 256);
+      delete_units_kernel<<<ub, 256, 0, s>>>(a, kMmaUnitPairs);
+      cudaError_t e = launch_exclusive_scan(a.in_cnt, a.unit_off, a.n + 1, a.scan_tmp, s);
+      if (e != cudaSuccess) return e;
+      uint64_t blocks = (total + kMmaUnitPairs - 1) / kMmaUnitPairs + a.n;  // upper bound on the number of units
+      if (blocks > 148u * 8u) blocks = 148u * 8u;
+      kern<<<(unsigned)blocks, kMmaWarps * 32, smem, s>>>(a, total_in);
+      count_launches(2);
+      return cudaGetLastError();
+    }
   }
   const size_t stage = (size_t)a.k_repair * ((a.lay.nchunk | 1u) * 16u);
   if (stage <= 64 * 1024) {
@@ -431,7 +616,7 @@ static cudaError_t launch_delete_picks_t(const DeleteArgs& a, uint64_t total_in,
       smem_set = smem;
     }
     const unsigned ub = (unsigned)((a.n + 256) / 256 > 148u * 16u ? 148u * 16u : (a.n + 256) / 256);
-    delete_units_kernel<<<ub, 256, 0, s>>>(a);
+    delete_units_kernel<<<ub, 256, 0, s>>>(a, kUnitPairs);
     cudaError_t e = launch_exclusive_scan(a.in_cnt, a.unit_off, a.n + 1, a.scan_tmp, s);
     if (e != cudaSuccess) return e;
     uint64_t blocks = (total + kUnitPairs - 1) / kUnitPairs + a.n;  // upper bound on the number of units
