@@ -190,6 +190,37 @@ def test_ragged_dim_int8_and_small_params_bit_exact():
     assert_same_graph(o, g, "reinsert")
 
 
+@pytest.mark.parametrize("dim,dtype", [(16, go.U8), (100, go.U8), (200, go.U8), (250, go.U8), (33, go.I8), (256, go.I8)])
+def test_delete_repair_bit_exact_across_row_sizes(dim, dtype):
+    """The delete repair's neighbour-by-candidate distance block on integer rows of every padding class (row
+    bytes a multiple of 32 or not, one to eight 32-byte steps), extreme values included."""
+    torch = torch_()
+    n = 3000
+    rng = np.random.default_rng(100 + dim)
+    if dtype == go.U8:
+        base = synth.uniform_u8(11, f"base{dim}", 0, n, dim)
+        base[:5] = 255; base[5:10] = 0
+    else:
+        base = rng.integers(-128, 128, (n, dim)).astype(np.int8)
+        base[:5] = -128; base[5:10] = 127
+    base[:10, 0] = np.arange(10).astype(base.dtype)         # keep the extreme rows distinct
+    cfg = dict(dim=dim, dtype=dtype, metric=go.L2, R=20, L=40, alpha=1.2, mode=go.VAMANA, max_build_batch=600, ins=1, dele=600)
+    o, g = make_pair(cfg, n)
+    for lo in range(0, n, 600):
+        ids = np.arange(lo, lo + 600, dtype=np.uint32)
+        o.insert_batch(ids, base[ids]); g.insert_batch(torch.from_numpy(ids), torch.from_numpy(base[ids]))
+    assert_same_graph(o, g, "build")
+    alive = np.ones(n, bool)
+    for r in range(3):
+        dele = synth.choose_ids(dim, f"del/{r}", np.flatnonzero(alive).astype(np.uint32), 600)
+        if r == 0:
+            dele[:10] = np.arange(10)                        # the extreme rows go first (ids 0..9 are still live)
+            dele = np.unique(dele).astype(np.uint32)
+        o.delete_batch(dele); g.delete_batch(torch.from_numpy(dele))
+        alive[dele] = False
+        assert_same_graph(o, g, f"delete {r}")
+
+
 def test_hub_segment_longer_than_shared_memory_cap():
     """Every point of a large batch links to the same few hubs: request segments far above the
     in-kernel shared-memory cap take the in-place global-memory sort."""
