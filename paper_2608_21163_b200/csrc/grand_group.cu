@@ -154,30 +154,40 @@ cudaError_t launch_exclusive_scan(const uint32_t* in, uint32_t* out, uint64_t n,
 // ---- reverse graph
 // `heads` (optional bitmap): only edges whose head is marked are counted / scattered, i.e. only the
 // in-neighbour rows of the marked nodes are materialised (the delete path reads no other row).
-// One warp per adjacency row (a coalesced read of the row, its degree fetched once, no index arithmetic per edge).
-__global__ void transpose_hist_kernel(const GraphView g, uint32_t* indeg, const uint32_t* heads) {
+// One warp per adjacency row (a coalesced read of the row, its degree fetched once, no index arithmetic per edge),
+// four rows in flight per warp: degree -> row -> bitmap word is a chain of dependent loads, and one row at a time
+// left the kernels waiting on it at a fifth of the memory bandwidth.
+constexpr int kTransposeRows = 4;
+template <typename F>
+__device__ __forceinline__ void for_each_marked_edge(const GraphView& g, const uint32_t* heads, F&& f) {
   const int lane = threadIdx.x & 31;
   const uint64_t wglobal = (blockIdx.x * (uint64_t)blockDim.x + threadIdx.x) >> 5;
   const uint64_t wtotal = ((uint64_t)gridDim.x * blockDim.x) >> 5;
-  for (uint64_t v = wglobal; v < g.cap; v += wtotal) {
-    const uint32_t dv = min(g.deg[v], g.R);
-    for (uint32_t sl = lane; sl < dv; sl += 32) {
-      const uint32_t z = g.adj[v * g.R + sl];
-      if (!heads || bit_test(heads, z)) atomicAdd(&indeg[z], 1u);
+  for (uint64_t v0 = wglobal; v0 < g.cap; v0 += kTransposeRows * wtotal) {
+    uint32_t dv[kTransposeRows];
+#pragma unroll
+    for (int k = 0; k < kTransposeRows; ++k) {
+      const uint64_t v = v0 + k * wtotal;
+      dv[k] = v < g.cap ? min(g.deg[v], g.R) : 0u;
+    }
+    for (uint32_t sb = 0; sb < g.R; sb += 32) {
+      uint32_t z[kTransposeRows];
+#pragma unroll
+      for (int k = 0; k < kTransposeRows; ++k) z[k] = sb + lane < dv[k] ? g.adj[(v0 + k * wtotal) * g.R + sb + lane] : 0xFFFFFFFFu;
+      bool hit[kTransposeRows];
+#pragma unroll
+      for (int k = 0; k < kTransposeRows; ++k) hit[k] = z[k] != 0xFFFFFFFFu && (!heads || bit_test(heads, z[k]));
+#pragma unroll
+      for (int k = 0; k < kTransposeRows; ++k)
+        if (hit[k]) f(z[k], (uint32_t)(v0 + k * wtotal));
     }
   }
 }
+__global__ void transpose_hist_kernel(const GraphView g, uint32_t* indeg, const uint32_t* heads) {
+  for_each_marked_edge(g, heads, [&](uint32_t z, uint32_t) { atomicAdd(&indeg[z], 1u); });
+}
 __global__ void transpose_scatter_kernel(const GraphView g, const uint32_t* off, uint32_t* fillc, uint32_t* src, const uint32_t* heads) {
-  const int lane = threadIdx.x & 31;
-  const uint64_t wglobal = (blockIdx.x * (uint64_t)blockDim.x + threadIdx.x) >> 5;
-  const uint64_t wtotal = ((uint64_t)gridDim.x * blockDim.x) >> 5;
-  for (uint64_t v = wglobal; v < g.cap; v += wtotal) {
-    const uint32_t dv = min(g.deg[v], g.R);
-    for (uint32_t sl = lane; sl < dv; sl += 32) {
-      const uint32_t z = g.adj[v * g.R + sl];
-      if (!heads || bit_test(heads, z)) src[off[z] + atomicAdd(&fillc[z], 1u)] = (uint32_t)v;
-    }
-  }
+  for_each_marked_edge(g, heads, [&](uint32_t z, uint32_t v) { src[off[z] + atomicAdd(&fillc[z], 1u)] = v; });
 }
 // ascending rows: shared-memory sort for short rows, in place in global memory for long ones
 __global__ void __launch_bounds__(128) transpose_sort_rows_kernel(uint64_t cap, const uint32_t* off, uint32_t* src) {
