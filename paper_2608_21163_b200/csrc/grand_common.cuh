@@ -104,6 +104,23 @@ __device__ __forceinline__ typename Elem<T>::Dist team_dist_regs(const uint4 (&a
   return finish_dist<T, METRIC>(acc);
 }
 
+// ---- tensor-core tile for integer rows: D (16 x 8, int32) += X (16 x 32 bytes, row-major) * Y^T (8 rows of 32 bytes).
+// Lane l (g = l / 4, t = l % 4) holds x[0] = X[g][4t..], x[1] = X[g + 8][4t..], x[2] = X[g][16 + 4t..],
+// x[3] = X[g + 8][16 + 4t..]; y[0] = Y[g][4t..], y[1] = Y[g][16 + 4t..]; d[0..1] = D[g][2t, 2t + 1],
+// d[2..3] = D[g + 8][2t, 2t + 1].
+template <typename T>
+__device__ __forceinline__ void mma_m16n8k32(int (&d)[4], const uint32_t (&x)[4], const uint32_t (&y)[2]) {
+  if constexpr (T(-1) < T(0)) {
+    asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+                 : "r"(x[0]), "r"(x[1]), "r"(x[2]), "r"(x[3]), "r"(y[0]), "r"(y[1]));
+  } else {
+    asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+                 : "r"(x[0]), "r"(x[1]), "r"(x[2]), "r"(x[3]), "r"(y[0]), "r"(y[1]));
+  }
+}
+
 // ---- sorting: bitonic network with min-to-lower-index comparators only, so any length works
 // (indices >= n behave as +inf and are never touched).  `sync` separates the stages.
 template <typename K, typename SyncFn>

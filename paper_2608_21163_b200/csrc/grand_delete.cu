@@ -419,19 +419,6 @@ constexpr uint32_t kMmaUnitPairs = 128;
 constexpr int kMmaNTiles = 7;  // candidate tiles of 8: k_repair <= 56
 constexpr int kMmaWarps = 4;
 
-template <typename T>
-__device__ __forceinline__ void mma_m16n8k32(int (&d)[4], const uint32_t (&x)[4], const uint32_t (&y)[2]) {
-  if constexpr (T(-1) < T(0)) {
-    asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                 : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
-                 : "r"(x[0]), "r"(x[1]), "r"(x[2]), "r"(x[3]), "r"(y[0]), "r"(y[1]));
-  } else {
-    asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                 : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
-                 : "r"(x[0]), "r"(x[1]), "r"(x[2]), "r"(x[3]), "r"(y[0]), "r"(y[1]));
-  }
-}
-
 static size_t delete_picks_mma_smem(uint32_t row_bytes) {
   const size_t rs = ((row_bytes + 31u) & ~31u) + 16u;
   return (size_t)(kMmaUnitPairs + kMmaNTiles * 8) * rs + (size_t)kMmaNTiles * 8 * 12 + (size_t)kMmaUnitPairs * 8;

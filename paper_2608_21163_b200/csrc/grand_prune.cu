@@ -215,9 +215,231 @@ __global__ void __launch_bounds__(kWarpPruneWarps * 32) forward_prune_warp_kerne
   if (lane == 0 && nprune) atomicAdd(&a.state->counters[CTR_PRUNE], (unsigned long long)nprune);
 }
 
+// The candidate-ordered prune on tensor cores, for integer rows of at most 128 bytes and R <= 64: one warp per
+// node takes the sorted candidates 16 at a time.  With |s - c|^2 = |s|^2 + |c|^2 - 2 s.c and the threshold
+// T_c = floor(D_p[c] * 65536 / A) (so that A * d <= D_p[c] * 65536 <=> d <= T_c, exact for integers), "member s
+// prunes candidate c" is  |s|^2 - 2 s.c <= T_c - |c|^2: one integer product per pair, taken as 8-bit mma tiles of
+// the block's 16 rows against the rows of the members selected so far and against the block itself.  The 16
+// candidates are then resolved in order on bit masks (a candidate falls to a member selected before the block or
+// to an earlier candidate of the block that was itself selected) and the selected ones join the member rows.
+constexpr uint32_t kMmaPruneR = 64, kMmaPruneCand = 256;
+constexpr int kMmaPruneWarps = 4;
+
+static size_t forward_prune_mma_smem_per_warp(uint32_t row_bytes) {
+  const size_t rs = ((row_bytes + 31u) & ~31u) + 16u;
+  return (size_t)kMmaPruneCand * 8 + (size_t)(kMmaPruneR + 16) * rs + (size_t)(kMmaPruneR + 16 + 16) * 4 + (size_t)kMmaPruneR * 4;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kMmaPruneWarps * 32) forward_prune_mma_kernel(const PruneArgs a, const uint32_t per_warp_bytes) {
+  constexpr unsigned FULL = 0xFFFFFFFFu;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int gid = lane >> 2, tig = lane & 3;
+  const uint32_t R = a.g.R, row_bytes = a.lay.row_bytes, nchunk = a.lay.nchunk;
+  const uint32_t kb = (row_bytes + 31u) & ~31u, rs = kb + 16u, kch = kb / 16u, ksteps = kb / 32u;
+  unsigned char* base = smem_raw + (size_t)warp * per_warp_bytes;
+  unsigned long long* cand = reinterpret_cast<unsigned long long*>(base);
+  uint8_t* srow = base + (size_t)kMmaPruneCand * 8;            // rows of the selected members
+  uint8_t* brow = srow + (size_t)kMmaPruneR * rs;              // rows of the block's 16 candidates
+  int* sV = reinterpret_cast<int*>(brow + 16 * (size_t)rs);    // |s|^2 per selected member
+  int* bU = sV + kMmaPruneR;                                   // T_c - |c|^2 per block candidate
+  int* bN = bU + 16;                                           // |c|^2 per block candidate
+  uint32_t* out_idx = reinterpret_cast<uint32_t*>(bN + 16);
+  const uint8_t* __restrict__ store = a.g.store;
+  unsigned long long npair = 0;
+  uint32_t nprune = 0;
+  auto wsync = [] { __syncwarp(); };
+  const uint64_t wglobal = (uint64_t)blockIdx.x * kMmaPruneWarps + warp, wtotal = (uint64_t)gridDim.x * kMmaPruneWarps;
+  for (uint64_t i = wglobal; i < a.n; i += wtotal) {
+    const uint32_t p = a.ids[i];
+    const uint32_t nc = min(min(a.cand_n[i], a.cand_stride), kMmaPruneCand);
+    for (uint32_t j = lane; j < nc; j += 32) {
+      const unsigned long long k = a.cand[i * a.cand_stride + j];
+      cand[j] = key_id(k) == p ? kKeyMax : k;
+    }
+    __syncwarp();
+    bitonic_sort_any(cand, nc, (uint32_t)lane, 32u, wsync);
+    uint32_t n = nc;
+    while (n > 0 && cand[n - 1] == kKeyMax) --n;
+    uint32_t cnt = 0;
+    for (uint32_t c0 = 0; c0 < n && cnt < R; c0 += 16) {
+      const uint32_t nb = min(16u, n - c0);
+      // ---- the block's rows (zero beyond the row and beyond the block), their norms and thresholds
+      for (uint32_t e = lane; e < 16 * kch; e += 32) {
+        const uint32_t j = e / kch, ch = e - j * kch;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (j < nb && ch < nchunk) v = __ldg(reinterpret_cast<const uint4*>(store + (size_t)key_id(cand[c0 + j]) * row_bytes) + ch);
+        reinterpret_cast<uint4*>(brow + (size_t)j * rs)[ch] = v;
+      }
+      __syncwarp();
+      if (lane < 16) {
+        const uint4* rp = reinterpret_cast<const uint4*>(brow + (size_t)lane * rs);
+        int nrm = 0;
+        for (uint32_t ch = 0; ch < nchunk; ++ch) acc_chunk<T, kMetricIP>(rp[ch], rp[ch], nrm);
+        long long thr = 0;
+        if ((uint32_t)lane < nb) thr = ((long long)key_dist<int>(cand[c0 + lane]) * 65536ll) / a.A_fix;
+        if (thr > 0x7FFFFFFFll) thr = 0x7FFFFFFFll;  // no distance is larger: the clamp changes no test
+        bN[lane] = nrm;
+        bU[lane] = (int)(thr - (long long)nrm > -0x80000000ll ? thr - (long long)nrm : -0x80000000ll);
+      }
+      __syncwarp();
+      // ---- tiles: the block against the selected members, and against itself
+      uint32_t xa[4][4];  // the block's fragments for up to 4 steps of 32 bytes
+      {
+        const uint8_t* x0 = brow + (size_t)gid * rs + tig * 4;
+        const uint8_t* x1 = x0 + 8 * (size_t)rs;
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks) {
+          if ((uint32_t)ks < ksteps) {
+            xa[ks][0] = *reinterpret_cast<const uint32_t*>(x0 + ks * 32);
+            xa[ks][1] = *reinterpret_cast<const uint32_t*>(x1 + ks * 32);
+            xa[ks][2] = *reinterpret_cast<const uint32_t*>(x0 + ks * 32 + 16);
+            xa[ks][3] = *reinterpret_cast<const uint32_t*>(x1 + ks * 32 + 16);
+          } else {
+            xa[ks][0] = xa[ks][1] = xa[ks][2] = xa[ks][3] = 0u;
+          }
+        }
+      }
+      const int u0 = bU[gid], u1 = bU[gid + 8];
+      bool old0 = false, old1 = false;  // rows gid / gid + 8 fall to a member selected before this block
+      for (uint32_t nt = 0; nt * 8 < cnt; ++nt) {
+        int acc[4] = {0, 0, 0, 0};
+        const uint8_t* yr = srow + (size_t)(nt * 8 + gid) * rs + tig * 4;
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks) {
+          if ((uint32_t)ks < ksteps) {
+            uint32_t yb[2];
+            yb[0] = *reinterpret_cast<const uint32_t*>(yr + ks * 32);
+            yb[1] = *reinterpret_cast<const uint32_t*>(yr + ks * 32 + 16);
+            mma_m16n8k32<T>(acc, xa[ks], yb);
+          }
+        }
+#pragma unroll
+        for (int jj = 0; jj < 2; ++jj) {
+          const uint32_t sidx = nt * 8 + tig * 2 + jj;
+          if (sidx < cnt) {
+            const int vs = sV[sidx];
+            old0 |= vs - 2 * acc[jj] <= u0;
+            old1 |= vs - 2 * acc[2 + jj] <= u1;
+          }
+        }
+      }
+      uint32_t rm0 = 0, rm1 = 0;  // bit j: candidate j of the block prunes candidate gid / gid + 8 of the block
+#pragma unroll
+      for (int nt = 0; nt < 2; ++nt) {
+        int acc[4] = {0, 0, 0, 0};
+        const uint8_t* yr = brow + (size_t)(nt * 8 + gid) * rs + tig * 4;
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks) {
+          if ((uint32_t)ks < ksteps) {
+            uint32_t yb[2];
+            yb[0] = *reinterpret_cast<const uint32_t*>(yr + ks * 32);
+            yb[1] = *reinterpret_cast<const uint32_t*>(yr + ks * 32 + 16);
+            mma_m16n8k32<T>(acc, xa[ks], yb);
+          }
+        }
+#pragma unroll
+        for (int jj = 0; jj < 2; ++jj) {
+          const uint32_t j = nt * 8 + tig * 2 + jj;
+          const int vj = bN[j];
+          if (vj - 2 * acc[jj] <= u0) rm0 |= 1u << j;
+          if (vj - 2 * acc[2 + jj] <= u1) rm1 |= 1u << j;
+        }
+      }
+      // a row's results are spread over the 4 lanes of its group
+      {
+        uint32_t o = (old0 ? 1u : 0u) | (old1 ? 2u : 0u);
+        o |= __shfl_xor_sync(FULL, o, 1);
+        o |= __shfl_xor_sync(FULL, o, 2);
+        old0 = o & 1u;
+        old1 = o & 2u;
+        rm0 |= __shfl_xor_sync(FULL, rm0, 1);
+        rm0 |= __shfl_xor_sync(FULL, rm0, 2);
+        rm1 |= __shfl_xor_sync(FULL, rm1, 1);
+        rm1 |= __shfl_xor_sync(FULL, rm1, 2);
+      }
+      const unsigned oldlo = __ballot_sync(FULL, old0), oldhi = __ballot_sync(FULL, old1);  // row r: bit 4 * (r & 7)
+      // ---- the 16 candidates in order
+      uint32_t sel = 0;
+      uint32_t room = R - cnt;
+      for (uint32_t r = 0; r < nb && room; ++r) {
+        const uint32_t rm = __shfl_sync(FULL, r < 8 ? rm0 : rm1, 4 * (r & 7));
+        const bool old = ((r < 8 ? oldlo : oldhi) >> (4 * (r & 7))) & 1u;
+        if (!old && !(rm & sel)) {  // (sel holds only earlier candidates)
+          sel |= 1u << r;
+          --room;
+        }
+      }
+      if (lane == 0) npair += (unsigned long long)nb * cnt + (unsigned long long)nb * (nb - 1) / 2;
+      // ---- the selected candidates join the members: index, norm, row
+      const uint32_t nsel = __popc(sel);
+      if (lane < 16 && ((sel >> lane) & 1u)) {
+        const uint32_t dst = cnt + __popc(sel & ((1u << lane) - 1u));
+        out_idx[dst] = c0 + lane;
+        sV[dst] = bN[lane];
+      }
+      for (uint32_t e = lane; e < 16 * kch; e += 32) {
+        const uint32_t j = e / kch, ch = e - j * kch;
+        if ((sel >> j) & 1u) {
+          const uint32_t dst = cnt + __popc(sel & ((1u << j) - 1u));
+          reinterpret_cast<uint4*>(srow + (size_t)dst * rs)[ch] = reinterpret_cast<const uint4*>(brow + (size_t)j * rs)[ch];
+        }
+      }
+      cnt += nsel;
+      __syncwarp();
+    }
+    ++nprune;
+    for (uint32_t sl = lane; sl < R; sl += 32) {
+      uint32_t id = kInvalid, db = kInvalid;
+      unsigned long long rk = 0;
+      if (sl < cnt) {
+        const unsigned long long k = cand[out_idx[sl]];
+        id = key_id(k);
+        rk = (k & 0xFFFFFFFF00000000ull) | p;  // dist(p, id) is symmetric: the request carries it
+        db = (uint32_t)(k >> 32);
+      }
+      a.g.adj[(size_t)p * R + sl] = id;
+      if (a.g.rowd) a.g.rowd[(size_t)p * R + sl] = db;
+      a.req_tgt[i * R + sl] = id;
+      a.req_key[i * R + sl] = rk;
+    }
+    if (lane == 0) {
+      a.g.deg[p] = cnt;
+      a.g.rowpfx[p] = (uint8_t)cnt;
+      if (a.g.birth) {
+        a.g.birth[p] = a.g.epoch;
+        a.g.rowepoch[p] = a.g.epoch;
+      }
+    }
+    __syncwarp();
+  }
+  if (npair) atomicAdd(&a.state->counters[CTR_PAIR], npair);
+  if (lane == 0 && nprune) atomicAdd(&a.state->counters[CTR_PRUNE], (unsigned long long)nprune);
+}
+
 template <typename T, int METRIC, int G, int CPL>
 static cudaError_t launch_forward_prune_t(const PruneArgs& a, cudaStream_t s) {
   if (a.n == 0) return cudaSuccess;
+  if constexpr (sizeof(T) == 1) {
+    if (!a.fixed_mode && a.lay.row_bytes <= 128u && a.g.R <= kMmaPruneR && a.cand_stride <= kMmaPruneCand && a.A_fix > 0) {
+      const size_t per_warp = (forward_prune_mma_smem_per_warp(a.lay.row_bytes) + 15) / 16 * 16;
+      const size_t smem = per_warp * kMmaPruneWarps;
+      auto kern = forward_prune_mma_kernel<T>;
+      static bool smem_set = false;  // (one kernel serves every row layout of this element type)
+      if (!smem_set) {
+        const size_t most = (forward_prune_mma_smem_per_warp(128u) + 15) / 16 * 16 * kMmaPruneWarps;
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)most);
+        if (e != cudaSuccess) return e;
+        smem_set = true;
+      }
+      const uint64_t want = (a.n + kMmaPruneWarps - 1) / kMmaPruneWarps;
+      const unsigned blocks = (unsigned)(want < 148u * 8u ? want : 148u * 8u);
+      kern<<<blocks, kMmaPruneWarps * 32, smem, s>>>(a, (uint32_t)per_warp);
+      count_launches(1);
+      return cudaGetLastError();
+    }
+  }
   if constexpr (G * CPL <= 16) {
     if (!a.fixed_mode && a.cand_stride <= kWarpPruneCand) {
       const uint64_t want = (a.n + kWarpPruneWarps - 1) / kWarpPruneWarps;
