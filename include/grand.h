@@ -61,7 +61,8 @@ typedef struct {
   uint32_t c;         /* replacement edges per repaired neighbour; default 2; <= 8 */
   uint32_t k_repair;  /* repair candidates per deleted node; default min(50, L); <= 128 */
   uint32_t vmax;      /* expansion cap of update searches; default 2*L; <= 1024 */
-  uint32_t mode;      /* grand_mode; default GRAND_MODE_VAMANA */
+  uint32_t mode;      /* grand_mode; default GRAND_MODE_VAMANA.  GRAND_MODE_FIXED_DEGREE needs R <= L (Alg. 7 keeps
+                         the R closest entries of a search result of L entries); else GRAND_ERR_INVALID_ARG */
   uint32_t hash_bits; /* log2 of the per-query visited cache in 4-byte words; default 10; 8..13, and 4 << hash_bits >= padded row bytes */
   uint32_t full_transpose; /* 1: every delete batch builds the whole reverse graph; default 0: only the rows of the
                               batch's nodes (the only rows the repair reads; identical result) */

@@ -653,6 +653,7 @@ int grand_oracle_create(uint32_t dim, uint32_t dtype, uint32_t metric, uint32_t 
   if (!out || dim == 0 || R == 0 || L == 0 || dtype > 2 || metric > 1 || mode > 1 || capacity == 0) return ERR_INVALID_ARG;
   const bool augment = mode == MODE_VAMANA && metric == M_IP && max_norm > 0.0f && dtype == DT_F32;
   if (mode == MODE_VAMANA && metric == M_IP && !augment) return ERR_UNSUPPORTED;
+  if (mode == MODE_FIXED && R > L) return ERR_INVALID_ARG;  // Alg. 7: the forward row is the R closest of a search result of L entries
   Index* ix = new Index();
   ix->udim = dim;
   ix->approx_delete = approx_delete != 0 && mode == MODE_VAMANA;

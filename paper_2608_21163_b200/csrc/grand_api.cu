@@ -318,6 +318,7 @@ int grand_create_ex(uint32_t dim, uint32_t dtype, uint32_t metric, uint32_t R, u
   const bool mips = o->mode == GRAND_MODE_VAMANA && metric == GRAND_IP && o->mips_max_norm > 0.0f && dtype == GRAND_F32;
   if (o->mode == GRAND_MODE_VAMANA && metric == GRAND_IP && !mips) return GRAND_ERR_UNSUPPORTED;
   if (o->snapshot_search && o->visited_set_delete) return GRAND_ERR_UNSUPPORTED;  // those searches read the live bitmap, which has one copy
+  if (o->mode == GRAND_MODE_FIXED_DEGREE && R > L) return GRAND_ERR_INVALID_ARG;  // Alg. 7 keeps the R closest of a search result of L entries
   // MIPS -> L2 reduction: rows carry one extra coordinate and the index works on squared L2
   Layout lay = mips ? make_layout(dim + 1, dtype, GRAND_L2) : make_layout(dim, dtype, metric);
   lay.udim = dim;

@@ -351,6 +351,13 @@ def test_errors_leave_index_unchanged():
     assert_same_graph(o, g, "after recovery")
 
 
+def test_fixed_degree_mode_rejects_a_row_longer_than_the_search_list():
+    from paper_2608_21163_b200 import binding as gb
+    with pytest.raises(gb.GrandError):
+        gb.GrandIndex(8, gb.U8, gb.L2, 33, 32, 1.2, capacity=100, max_batch=10, mode=gb.FIXED_DEGREE)
+    gb.GrandIndex(8, gb.U8, gb.L2, 32, 32, 1.2, capacity=100, max_batch=10, mode=gb.FIXED_DEGREE)
+
+
 def test_host_entry_points_match_device_entry_points():
     torch = torch_()
     cfg = small_cfg("tiny_u8_d32", 0.1, rounds=0)

@@ -631,3 +631,11 @@ def test_visited_set_delete_stream_invariants():
         t, _ = brute_knn(base, live_ids, q[i], 10)
         ra += len(set(t.tolist()) & set(ia[i].tolist())); rb += len(set(t.tolist()) & set(ib[i].tolist()))
     assert ra / 2000 > 0.85 and abs(ra - rb) / 2000 < 0.05
+
+
+def test_fixed_degree_mode_needs_the_search_list_to_hold_a_row():
+    """Alg. 7 takes the R closest entries of the search result, which holds L entries: R > L has no meaning there."""
+    with pytest.raises(go.OracleError):
+        go.Oracle(8, go.U8, go.L2, 33, 32, 1.2, 100, mode=go.FIXED_DEGREE)
+    go.Oracle(8, go.U8, go.L2, 32, 32, 1.2, 100, mode=go.FIXED_DEGREE)
+    go.Oracle(8, go.U8, go.L2, 33, 32, 1.2, 100)            # Vamana mode prunes the visited list: any R
