@@ -11,11 +11,13 @@ from tests.helpers import INV, assert_same_graph
 pytestmark = pytest.mark.gpu
 
 
-def run_config(seed):
+def run_config(seed, wide=False):
     from paper_2608_21163_b200 import binding as gb
     rng = np.random.default_rng(seed)
     dtype = int(rng.choice([go.U8, go.U8, go.I8]))
     dim = int(rng.choice([3, 8, 16, 17, 31, 32, 48, 64, 96, 100, 127, 128, 129, 160, 200, 256, 300]))
+    if wide:                                           # rows of 257..4000 bytes: the whole-warp distance layouts
+        dim = int(rng.choice([257, 384, 512, 513, 700, 1024, 1500, 2048, 3000, 4000]))
     R = int(rng.choice([4, 7, 8, 13, 16, 24, 32, 33, 48, 64, 65, 96]))
     L = max(int(rng.choice([R, R + 3, 2 * R, 40, 64, 100, 128])), 4)
     alpha = float(rng.choice([1.0, 1.1, 1.2, 1.5, 2.0]))
@@ -33,6 +35,8 @@ def run_config(seed):
     kr = min(kr, L)
     n = int(rng.choice([600, 1500, 3000]))
     nb = int(rng.choice([100, 250, 500]))
+    if wide:
+        n, nb = int(rng.choice([400, 800])), int(rng.choice([50, 100, 200]))
     if dtype == go.U8:
         if rng.random() < 0.5:
             cen = rng.integers(0, 256, (8, dim))
@@ -77,3 +81,8 @@ def run_config(seed):
 def test_random_configurations_bit_exact(block):
     for seed in range(5000 + 25 * block, 5000 + 25 * (block + 1)):
         run_config(seed)
+
+
+def test_random_configurations_wide_rows_bit_exact():
+    for seed in range(6000, 6030):
+        run_config(seed, wide=True)
