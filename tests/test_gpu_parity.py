@@ -475,3 +475,32 @@ def test_mips_reduction_vamana_ip_matches_oracle():
     g.insert_batch(torch.from_numpy(dele[:2]), torch.from_numpy(base[dele[:2]]))   # the index is still usable
     with pytest.raises(gb.GrandError):
         gb.GrandIndex(d, gb.U8, gb.IP, R, L, 1.2, capacity=n, mips_max_norm=1.0)  # fp32 only
+
+
+# ------------------------------------------------------------------ hand-worked cases, straight from tests/golden/
+from tests import golden_cases as gc
+
+
+@pytest.mark.parametrize("fname,case", gc.all_cases(), ids=lambda x: x["name"] if isinstance(x, dict) else x.split(".")[0])
+def test_hand_worked_graph_cases_on_the_gpu(fname, case):
+    """The CUDA library against the hand-worked expected rows and medoids themselves (no oracle in between):
+    Alg. 7 slot choice and forward row, Alg. 8 rewire and medoid replacement, the scratch bound of Alg. 6,
+    the rounding of the initial medoid."""
+    torch = torch_()
+    from paper_2608_21163_b200 import binding as gb
+    g = gb.GrandIndex(case["dim"], case["dtype"], case["metric"], case["R"], case["L"], case["alpha"], capacity=case["cap"],
+                      max_batch=8, mode=case["mode"], **case["opts"])
+    s = case["start"]
+    if s is not None:
+        g.import_graph(torch.from_numpy(s["adj"]), torch.from_numpy(s["deg"]), torch.from_numpy(go.pack_bitmap(s["live"])),
+                       s["entry"], torch.from_numpy(s["vecs"]))
+    for kind, ids, v in case["ops"]:
+        if kind == "insert":
+            g.insert_batch(torch.from_numpy(ids), torch.from_numpy(v))
+        else:
+            g.delete_batch(torch.from_numpy(ids))
+    adj, deg, live, entry = gpu_graph(g)
+    for v, want in case["expect_rows"].items():
+        assert adj[v, :deg[v]].tolist() == want, (case["name"], v, adj[v, :deg[v]].tolist(), want)
+    if case["expect_entry"] is not None:
+        assert entry == case["expect_entry"]

@@ -639,3 +639,33 @@ def test_fixed_degree_mode_needs_the_search_list_to_hold_a_row():
         go.Oracle(8, go.U8, go.L2, 33, 32, 1.2, 100, mode=go.FIXED_DEGREE)
     go.Oracle(8, go.U8, go.L2, 32, 32, 1.2, 100, mode=go.FIXED_DEGREE)
     go.Oracle(8, go.U8, go.L2, 33, 32, 1.2, 100)            # Vamana mode prunes the visited list: any R
+
+
+# ------------------------------------------------------------------ hand-worked graph cases (tests/golden/*_cases.txt)
+# Alg. 7 backward-edge slot rule and forward-row source, Alg. 8 medoid replacement, Alg. 6 scratch bound, initial
+# medoid rounding: each expected row / medoid below was worked by hand in the fixture's comments.
+from tests import golden_cases as gc
+
+
+def replay_on_oracle(case):
+    o = go.Oracle(case["dim"], case["dtype"], case["metric"], case["R"], case["L"], case["alpha"], case["cap"],
+                  mode=case["mode"], nthreads=2, **case["opts"])
+    s = case["start"]
+    if s is not None:
+        o.import_graph(s["adj"], s["deg"], go.pack_bitmap(s["live"]), s["entry"], s["vecs"])
+    for kind, ids, v in case["ops"]:
+        if kind == "insert":
+            o.insert_batch(ids, v)
+        else:
+            o.delete_batch(ids)
+    return o
+
+
+@pytest.mark.parametrize("fname,case", gc.all_cases(), ids=lambda x: x["name"] if isinstance(x, dict) else x.split(".")[0])
+def test_hand_worked_graph_cases(fname, case):
+    o = replay_on_oracle(case)
+    adj, deg, live, entry = o.export_graph()
+    for v, want in case["expect_rows"].items():
+        assert adj[v, :deg[v]].tolist() == want, (case["name"], v, adj[v, :deg[v]].tolist(), want)
+    if case["expect_entry"] is not None:
+        assert entry == case["expect_entry"], (case["name"], entry)
