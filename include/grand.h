@@ -4,7 +4,10 @@
  *
  * One handle = one index on one GPU = one mutator at a time.  The library owns the device-resident
  * vector store (row stride padded to 16 B), the fixed-stride adjacency array uint32[capacity x R]
- * with a degree counter per node, the live bitmap and a grow-only workspace pool; the caller owns
+ * with a degree counter per node, the live bitmap and a workspace pool that is allocated when the
+ * index is created (the pre-allocated resource pool of Sec. 3.1): grand_insert_batch, grand_delete_batch,
+ * grand_search and the host variants of the two update calls allocate nothing.  (grand_reverse_graph and
+ * grand_search_host keep buffers of their own that grow with the largest request.)  The caller owns
  * every buffer it passes in, and the library keeps no caller pointer past a call.  Unless a
  * function says "host", pointer arguments are DEVICE pointers, row-major and densely packed.
  *
@@ -37,14 +40,14 @@ typedef enum { GRAND_MODE_VAMANA = 0, GRAND_MODE_FIXED_DEGREE = 1 } grand_mode;
 typedef enum {
   GRAND_OK = 0,
   GRAND_ERR_INVALID_ARG = -1,  /* null pointer, k > L, parameter beyond a compile-time bound */
-  GRAND_ERR_CAPACITY = -2,     /* id >= capacity, or batch larger than max_batch */
+  GRAND_ERR_CAPACITY = -2,     /* id >= capacity, batch larger than max_batch, or a delete batch that touches more
+                                  in-neighbour entries than max_delete_edges */
   GRAND_ERR_DUPLICATE_ID = -3, /* the same id twice in one batch */
   GRAND_ERR_ALREADY_LIVE = -4, /* insert of a live id */
   GRAND_ERR_NOT_LIVE = -5,     /* delete of an id that is not live */
   GRAND_ERR_UNSUPPORTED = -6,  /* Vamana mode with the IP metric and no mips_max_norm (alpha-pruning needs a metric) */
   GRAND_ERR_CUDA = -7,         /* a CUDA call failed; text in grand_last_error */
-  GRAND_ERR_LIMIT = -8,        /* a bounded device loop hit its bound */
-  GRAND_ERR_NOMEM = -9         /* device allocation failed */
+  GRAND_ERR_NOMEM = -9         /* device allocation failed (index creation, or growth of an introspection buffer) */
 } grand_status;
 
 #define GRAND_INVALID_ID 0xFFFFFFFFu
@@ -75,6 +78,10 @@ typedef struct {
                               the search did not visit stay behind; searches and rebuilds skip neighbours that
                               are not live.  Default 0: exact in-neighbours, no edge to a deleted node survives.
                               Vamana mode only. */
+  uint64_t max_delete_edges;   /* most in-neighbour entries (sum of the in-degrees of its nodes) one delete batch may
+                              touch; default min(3 * max_batch * R, capacity * R).  The workspace of the update
+                              calls is sized from max_batch and this bound when the index is created; a delete
+                              batch beyond it fails with GRAND_ERR_CAPACITY and leaves the index unchanged. */
   uint32_t snapshot_search;    /* 1: searches may run on other streams (and from other host threads) WHILE an update
                               batch runs.  The adjacency is kept twice; a batch works on the unpublished copy and
                               publishes it when it returns, so a search sees exactly the graph of the last batch
@@ -98,16 +105,25 @@ typedef struct {
   uint64_t dirty_nodes;    /* adjacency rows rebuilt */
   uint64_t prunes;         /* RobustPrune invocations (forward + rebuild) */
   uint64_t requests;       /* reverse-edge / repair requests grouped */
-  uint64_t kernel_launches;
-  uint64_t reserved;
+  uint64_t kernel_launches; /* kernels launched through this handle */
+  uint64_t rebuild_bytes;  /* bytes the dirty-node rebuild has to move: per rebuilt row its read and write (2 * R * 4),
+                              its request tuples (12 each) and, when a prune runs, one vector per candidate */
+  uint64_t picks_bytes;    /* bytes the delete repair has to move: one vector per (deleted node, surviving in- or
+                              out-neighbour) pair plus the repair candidates' vectors once per deleted node */
+  uint64_t prune_bytes;    /* forward RobustPrune: one vector per candidate looked at */
+  uint64_t rebuild_prunes; /* rebuilt rows that went through a prune (the rest were appends / compactions) */
   double ms_search;        /* beam-search kernels (search, insert and delete searches) */
   double ms_prune;         /* forward RobustPrune */
-  double ms_group;         /* request emission, grouping */
+  double ms_group;         /* request grouping, and the set-up kernels of the repair picks */
   double ms_rebuild;       /* dirty-node rebuild */
   double ms_transpose;     /* reverse-graph construction */
-  double ms_picks;         /* delete repair picks */
+  double ms_picks;         /* delete repair picks (the pick kernel alone) */
   double ms_other;         /* validation, store write, publish / retire */
-  uint64_t n_search_launches;
+  uint64_t n_search_launches;  /* launches behind ms_search, ms_prune, ms_rebuild, ms_picks, ms_transpose: */
+  uint64_t n_prune_launches;
+  uint64_t n_rebuild_launches;
+  uint64_t n_picks_launches;
+  uint64_t n_transpose_launches;
 } grand_stats;
 
 /* Index life cycle (problem statement of Sec. 3-4: capacity fixed at initialisation, ids in
@@ -150,7 +166,8 @@ int grand_search_host(grand_index* idx, const void* queries_host, uint64_t nq, u
  * ceil(capacity/32) words, bit v%32 of word v/32; entry_out_host: HOST pointer to the medoid id. */
 int grand_export_graph(const grand_index* idx, uint32_t* adj_dev, uint32_t* deg_dev, uint32_t* live_bitmap_dev,
                        uint32_t* entry_out_host, grand_stream stream);
-/* Replaces the whole state (tests only).  vecs_dev: capacity x dim packed elements. */
+/* Replaces the whole state (tests, and loading a saved index).  vecs_dev: capacity x dim packed elements.  Every
+ * degree must be <= R and every listed neighbour id < capacity, else GRAND_ERR_INVALID_ARG and nothing is replaced. */
 int grand_import_graph(grand_index* idx, const uint32_t* adj_dev, const uint32_t* deg_dev,
                        const uint32_t* live_bitmap_dev, uint32_t entry, const void* vecs_dev, grand_stream stream);
 /* Exact reverse graph in CSR (Alg. 8): off_dev has capacity+1 entries, row z of src_dev lists every live
@@ -163,8 +180,9 @@ int grand_reverse_graph(grand_index* idx, uint32_t* off_dev, uint32_t* src_dev, 
  * frozen at start-up (a serving process that has handed all of HBM to its own pool, a sandboxed plug-in
  * barred from the driver's allocator, a real-time loop that cannot take cudaMalloc's implicit
  * synchronisation or its failure mid-request).  The paper has no counterpart for this call.  It needs no
- * index handle: adj_dev (n_nodes x R, unused slots ignored through deg_dev) and deg_dev (n_nodes) are the
- * caller's inputs, off_dev (n_nodes + 1) and src_dev (src_capacity entries; NULL = offsets only) the caller's
+ * index handle: adj_dev (n_nodes x R, unused slots ignored through deg_dev; every listed neighbour id must be
+ * < n_nodes, otherwise the call returns GRAND_ERR_INVALID_ARG - such an edge is never followed, so nothing is
+ * written outside the caller's buffers) and deg_dev (n_nodes) are the caller's inputs, off_dev (n_nodes + 1) and src_dev (src_capacity entries; NULL = offsets only) the caller's
  * outputs, E_out_host a HOST pointer to the edge count.  The result equals grand_reverse_graph on the same
  * graph.  Its working memory is one fixed device array inside the library, GRAND_NOALLOC_SCRATCH_BYTES per GPU
  * for the life of the process: n_nodes > GRAND_NOALLOC_MAX_NODES returns GRAND_ERR_CAPACITY, and so does a

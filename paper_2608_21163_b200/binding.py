@@ -30,20 +30,22 @@ class GrandOptions(C.Structure):
     _fields_ = [("capacity", C.c_uint64), ("max_batch", C.c_uint64), ("P", C.c_uint32), ("c", C.c_uint32),
                 ("k_repair", C.c_uint32), ("vmax", C.c_uint32), ("mode", C.c_uint32), ("hash_bits", C.c_uint32),
                 ("full_transpose", C.c_uint32), ("mips_max_norm", C.c_float),
-                ("visited_set_delete", C.c_uint32), ("snapshot_search", C.c_uint32),
+                ("visited_set_delete", C.c_uint32), ("max_delete_edges", C.c_uint64), ("snapshot_search", C.c_uint32),
                 ("dev_alloc", C.c_void_p), ("dev_free", C.c_void_p), ("user", C.c_void_p)]
 
 
 class GrandStats(C.Structure):
     _fields_ = [("expansions", C.c_uint64), ("dist_evals", C.c_uint64), ("pair_dists", C.c_uint64),
                 ("dirty_nodes", C.c_uint64), ("prunes", C.c_uint64), ("requests", C.c_uint64),
-                ("kernel_launches", C.c_uint64), ("reserved", C.c_uint64),
+                ("kernel_launches", C.c_uint64), ("rebuild_bytes", C.c_uint64), ("picks_bytes", C.c_uint64),
+                ("prune_bytes", C.c_uint64), ("rebuild_prunes", C.c_uint64),
                 ("ms_search", C.c_double), ("ms_prune", C.c_double), ("ms_group", C.c_double),
                 ("ms_rebuild", C.c_double), ("ms_transpose", C.c_double), ("ms_picks", C.c_double),
-                ("ms_other", C.c_double), ("n_search_launches", C.c_uint64)]
+                ("ms_other", C.c_double), ("n_search_launches", C.c_uint64), ("n_prune_launches", C.c_uint64),
+                ("n_rebuild_launches", C.c_uint64), ("n_picks_launches", C.c_uint64), ("n_transpose_launches", C.c_uint64)]
 
     def as_dict(self):
-        return {k: getattr(self, k) for k, _ in self._fields_ if k != "reserved"}
+        return {k: getattr(self, k) for k, _ in self._fields_}
 
 
 _lib = None
@@ -106,7 +108,7 @@ class GrandIndex:
 
     def __init__(self, dim, dtype, metric, R, L, alpha, capacity=0, max_batch=0, P=0, c=0, k_repair=0, vmax=0,
                  mode=VAMANA, hash_bits=0, full_transpose=0, mips_max_norm=0.0, visited_set_delete=0,
-                 snapshot_search=0):
+                 snapshot_search=0, max_delete_edges=0, dev_alloc=None, dev_free=None):
         if not torch.cuda.is_available():
             raise RuntimeError("a CUDA device is required (no CPU fallback)")
         self.lib = load()
@@ -115,7 +117,13 @@ class GrandIndex:
         self.dist_dtype = torch.float32 if dtype == F32 else torch.int32
         o = GrandOptions(capacity=capacity, max_batch=max_batch, P=P, c=c, k_repair=k_repair, vmax=vmax, mode=mode,
                          hash_bits=hash_bits, full_transpose=full_transpose, mips_max_norm=mips_max_norm,
-                         visited_set_delete=visited_set_delete, snapshot_search=snapshot_search)
+                         visited_set_delete=visited_set_delete, snapshot_search=snapshot_search,
+                         max_delete_edges=max_delete_edges)
+        # optional allocator hooks: ctypes callbacks (void* (size_t, void*) / void (void*, void*)); kept alive here
+        self._hooks = (dev_alloc, dev_free)
+        if dev_alloc is not None:
+            o.dev_alloc = C.cast(dev_alloc, C.c_void_p)
+            o.dev_free = C.cast(dev_free, C.c_void_p)
         h = C.c_void_p()
         rc = self.lib.grand_create_ex(C.c_uint32(dim), C.c_uint32(dtype), C.c_uint32(metric), C.c_uint32(R),
                                       C.c_uint32(L), C.c_float(alpha), C.byref(o), C.byref(h))

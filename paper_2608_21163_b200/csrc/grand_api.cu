@@ -15,9 +15,46 @@
 
 namespace grand {
 
-static std::atomic<unsigned long long> g_launches{0};
-void count_launches(unsigned n) { g_launches += n; }
-unsigned long long launches_so_far() { return g_launches.load(); }
+// Launch counting: the entry point that runs on this thread names its handle's counter.
+static thread_local unsigned long long* tl_launches = nullptr;
+void count_launches(unsigned n) {
+  if (tl_launches) *tl_launches += n;
+}
+LaunchScope::LaunchScope(unsigned long long* counter) : prev(tl_launches) { tl_launches = counter; }
+LaunchScope::~LaunchScope() { tl_launches = prev; }
+
+// Per-device facts, looked up on first use on that device.
+static std::atomic<int> g_sm_count[kMaxDevices];
+static std::atomic<int> g_smem_optin[kMaxDevices];
+static int current_device() {
+  int dev = 0;
+  cudaGetDevice(&dev);
+  return dev >= 0 && dev < kMaxDevices ? dev : 0;
+}
+int sm_count() {
+  const int dev = current_device();
+  int n = g_sm_count[dev].load(std::memory_order_relaxed);
+  if (n == 0) {
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    if (n <= 0) n = 1;
+    g_sm_count[dev].store(n, std::memory_order_relaxed);
+  }
+  return n;
+}
+cudaError_t allow_full_dynamic_smem(const void* kernel, SmemOptIn* done) {
+  const int dev = current_device();
+  // (two threads may both find the slot empty; they then set the same value twice)
+  if (__atomic_load_n(&done->done[dev], __ATOMIC_ACQUIRE)) return cudaSuccess;
+  int most = g_smem_optin[dev].load(std::memory_order_relaxed);
+  if (most == 0) {
+    cudaDeviceGetAttribute(&most, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    g_smem_optin[dev].store(most, std::memory_order_relaxed);
+  }
+  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
+  if (e != cudaSuccess) return e;
+  __atomic_store_n(&done->done[dev], 1, __ATOMIC_RELEASE);
+  return cudaSuccess;
+}
 
 Layout make_layout(uint32_t dim, uint32_t dtype, uint32_t metric) {
   Layout l{};
@@ -90,13 +127,24 @@ struct grand_index {
   unsigned long long* Ci = nullptr;
   uint32_t *Ci_n = nullptr, *in_cnt = nullptr, *pair_off = nullptr, *unit_off = nullptr, *scan_tmp = nullptr;
   uint8_t* mean_row = nullptr;
-  uint32_t* search_ctrs = nullptr;  // ring of work counters, one per in-flight search launch
-  std::atomic<uint32_t> ctr_next{0};
-  Buf req_tgt, req_key, seg_keys, dirty;              // grow-only, sized by the number of requests
-  Buf t_indeg, t_off, t_fill, t_src;                  // reverse graph, allocated at the first delete
-  Buf st_ids, st_vecs, st_out_ids, st_out_d;          // staging of the *_host entry points
+  // Work counters of the search launches.  Slot 0 serves the searches inside update calls (each such call ends
+  // with a stream synchronisation, so its launch is over before the next one starts).  grand_search is
+  // asynchronous: it takes a ring slot whose previous launch has completed (an event per slot tells), and runs
+  // with static query striding when none is free.
+  static constexpr int kCtrSlots = 64;
+  uint32_t* search_ctrs = nullptr;  // 1 + kCtrSlots counters
+  cudaEvent_t ctr_done[kCtrSlots] = {};
+  bool ctr_used[kCtrSlots] = {};
+  uint32_t ctr_next = 0;             // (ring state is touched only under pub_mu)
+  uint64_t max_requests = 0;       // request tuples a batch may emit (buffers below are sized for it at creation)
+  uint64_t max_delete_edges = 0;   // in-neighbour entries a delete batch may touch
+  Buf req_tgt, req_key, seg_keys, dirty;              // sized at creation for max_requests
+  Buf t_indeg, t_off, t_fill, t_src;                  // reverse graph of a delete batch, sized at creation
+  Buf x_indeg, x_off, x_fill, x_src;                  // full reverse graph for grand_reverse_graph (introspection; grown on demand)
+  Buf st_ids, st_vecs, st_out_ids, st_out_d;          // staging of the *_host entry points (updates: sized at creation)
   std::vector<void*> owned;
   // stats
+  unsigned long long launches = 0;
   grand_stats stats{};
   bool profiling = false;
   std::vector<cudaEvent_t> ev_pool;
@@ -139,16 +187,18 @@ int alloc_dev(grand_index* idx, T** out, size_t count, bool zero) {
   return GRAND_OK;
 }
 int ensure(grand_index* idx, Buf& b, size_t bytes, cudaStream_t s) {
-  if (b.bytes >= bytes) return GRAND_OK;
+  if (b.bytes >= bytes && b.p) return GRAND_OK;
+  const bool regrow = b.p != nullptr;
   if (b.p) {
     CK(cudaStreamSynchronize(s));
     idx->dev_free(b.p, idx->user);
     b.p = nullptr;
     b.bytes = 0;
   }
-  size_t want = bytes + bytes / 4;
+  size_t want = regrow ? bytes + bytes / 4 : bytes;  // first allocation: exact; regrowth: with headroom
+  if (want == 0) want = 16;
   void* p = idx->dev_alloc(want, idx->user);
-  if (!p) return fail(idx, GRAND_ERR_NOMEM, "workspace growth to " + std::to_string(want) + " bytes failed");
+  if (!p) return fail(idx, GRAND_ERR_NOMEM, "workspace allocation of " + std::to_string(want) + " bytes failed");
   b.p = p;
   b.bytes = want;
   return GRAND_OK;
@@ -220,10 +270,11 @@ int write_state_head(grand_index* idx, cudaStream_t s) {
   return GRAND_OK;
 }
 
-SearchArgs search_args(grand_index* idx, cudaStream_t s, bool work) {
+// slot < 0: the counter of the update calls; otherwise a ring slot taken by take_ctr_slot (or -2: none free)
+SearchArgs search_args(grand_index* idx, cudaStream_t s, bool work, int slot = -1) {
   SearchArgs a{};
-  a.work_ctr = idx->search_ctrs + (idx->ctr_next.fetch_add(1u) & 63u);
-  cudaMemsetAsync(a.work_ctr, 0, 4, s);
+  a.work_ctr = slot == -2 ? nullptr : idx->search_ctrs + (slot < 0 ? 0 : 1 + slot);
+  if (a.work_ctr) cudaMemsetAsync(a.work_ctr, 0, 4, s);
   a.lay = idx->lay;
   a.g = view(idx, work);
   a.entry = idx->entry;
@@ -233,6 +284,19 @@ SearchArgs search_args(grand_index* idx, cudaStream_t s, bool work) {
   a.mips_M2 = (float)idx->mips_M2;
   a.state = idx->d_state;
   return a;
+}
+
+// A ring slot whose last launch is over, or -2.  Caller holds pub_mu until the launch's end event is recorded.
+int take_ctr_slot(grand_index* idx) {
+  for (int tries = 0; tries < grand_index::kCtrSlots; ++tries) {
+    const int slot = (int)(idx->ctr_next++ % grand_index::kCtrSlots);
+    if (!idx->ctr_used[slot] || cudaEventQuery(idx->ctr_done[slot]) == cudaSuccess) {
+      idx->ctr_used[slot] = true;
+      return slot;
+    }
+    if (tries >= 3) break;  // a few probes, then static striding: the ring is full of running launches
+  }
+  return -2;
 }
 
 int ensure_requests(grand_index* idx, uint64_t nreq, cudaStream_t s) {
@@ -295,7 +359,6 @@ const char* grand_strerror(int st) {
     case GRAND_ERR_NOT_LIVE: return "id is not live";
     case GRAND_ERR_UNSUPPORTED: return "unsupported configuration";
     case GRAND_ERR_CUDA: return "CUDA error";
-    case GRAND_ERR_LIMIT: return "device loop limit reached";
     case GRAND_ERR_NOMEM: return "device memory allocation failed";
     default: return "unknown status";
   }
@@ -329,6 +392,7 @@ int grand_create_ex(uint32_t dim, uint32_t dtype, uint32_t metric, uint32_t R, u
   idx->A_fix = (long long)llround((double)alpha * 65536.0);
   idx->cap = o->capacity ? o->capacity : (1ull << 20);
   idx->max_batch = o->max_batch ? o->max_batch : (1ull << 17);
+  if (idx->max_batch > idx->cap) idx->max_batch = idx->cap;  // a batch names distinct ids
   idx->P = o->P ? o->P : 64;
   idx->c = o->c ? o->c : 2;
   idx->k_repair = o->k_repair ? o->k_repair : (L < 50 ? L : 50);
@@ -352,6 +416,17 @@ int grand_create_ex(uint32_t dim, uint32_t dtype, uint32_t metric, uint32_t R, u
   }
   cudaGetDevice(&idx->device);
   const uint64_t cap = idx->cap, mb = idx->max_batch;
+  // Request tuples of one batch: an insert emits n*R; a Vamana delete c per (deleted node, surviving in- or
+  // out-neighbour) pair; a fixed-degree delete one per in-neighbour entry.  The in-neighbour entries of a delete
+  // batch are bounded by max_delete_edges (default: three times the out-edges of a full batch, or every edge of
+  // the graph if that is less).
+  idx->max_delete_edges = o->max_delete_edges ? o->max_delete_edges : std::min<uint64_t>(3 * mb * R, cap * R);
+  idx->max_requests = std::max<uint64_t>(mb * R, idx->mode == GRAND_MODE_FIXED_DEGREE ? idx->max_delete_edges + 1
+                                                                                          : (idx->max_delete_edges + mb * R) * idx->c);
+  if (idx->max_requests >= (1ull << 32) || idx->max_delete_edges >= (1ull << 32)) {
+    delete idx;
+    return GRAND_ERR_INVALID_ARG;
+  }
   const size_t words = (cap + 31) / 32;
   int rc = GRAND_OK;
   auto A = [&](int r) { if (rc == GRAND_OK) rc = r; };
@@ -389,7 +464,7 @@ int grand_create_ex(uint32_t dim, uint32_t dtype, uint32_t metric, uint32_t R, u
     A(alloc_dev(idx, &idx->birth, cap, true));
     A(alloc_dev(idx, &idx->rowepoch, cap, true));
   }
-  A(alloc_dev(idx, &idx->search_ctrs, 64, true));
+  A(alloc_dev(idx, &idx->search_ctrs, 1 + grand_index::kCtrSlots, true));
   if (rc == GRAND_OK && cudaMemset(idx->adj, 0xFF, (size_t)cap * R * 4) != cudaSuccess) rc = GRAND_ERR_CUDA;
   if (rc == GRAND_OK && idx->snap && cudaMemset(idx->adj_alt, 0xFF, (size_t)cap * R * 4) != cudaSuccess) rc = GRAND_ERR_CUDA;
   if (rc == GRAND_OK && idx->rowd && cudaMemset(idx->rowd, 0xFF, (size_t)cap * R * 4) != cudaSuccess) rc = GRAND_ERR_CUDA;
@@ -399,7 +474,17 @@ int grand_create_ex(uint32_t dim, uint32_t dtype, uint32_t metric, uint32_t R, u
     idx->h_state->entry = GRAND_INVALID_ID;
     if (cudaMemcpy(idx->d_state, idx->h_state, sizeof(DevState), cudaMemcpyHostToDevice) != cudaSuccess) rc = GRAND_ERR_CUDA;
   }
-  if (rc == GRAND_OK) rc = ensure_requests(idx, mb * R, 0);
+  // everything an update batch can need is allocated here: no allocation happens on the update path
+  if (rc == GRAND_OK) rc = ensure_requests(idx, idx->max_requests, 0);
+  if (rc == GRAND_OK && idx->snap) rc = ensure(idx, idx->sync_dirty, idx->max_requests * 4, 0);  // trades places with `dirty`
+  if (rc == GRAND_OK) rc = ensure(idx, idx->t_indeg, (cap + 1) * 4, 0);
+  if (rc == GRAND_OK) rc = ensure(idx, idx->t_off, (cap + 1) * 4, 0);
+  if (rc == GRAND_OK) rc = ensure(idx, idx->t_fill, cap * 4, 0);
+  if (rc == GRAND_OK) rc = ensure(idx, idx->t_src, (idx->full_transpose ? cap * R : idx->max_delete_edges) * 4, 0);
+  if (rc == GRAND_OK) rc = ensure(idx, idx->st_ids, mb * 4, 0);
+  if (rc == GRAND_OK) rc = ensure(idx, idx->st_vecs, mb * (size_t)lay.udim * lay.esize, 0);
+  for (int i = 0; rc == GRAND_OK && i < grand_index::kCtrSlots; ++i)
+    if (cudaEventCreateWithFlags(&idx->ctr_done[i], cudaEventDisableTiming) != cudaSuccess) rc = GRAND_ERR_CUDA;
   if (rc != GRAND_OK) {
     grand_destroy(idx);
     return rc;
@@ -413,8 +498,10 @@ int grand_destroy(grand_index* idx) {
   cudaDeviceSynchronize();
   for (void* p : idx->owned) idx->dev_free(p, idx->user);
   for (Buf* b : {&idx->req_tgt, &idx->req_key, &idx->seg_keys, &idx->dirty, &idx->sync_dirty, &idx->t_indeg, &idx->t_off, &idx->t_fill, &idx->t_src,
-                 &idx->st_ids, &idx->st_vecs, &idx->st_out_ids, &idx->st_out_d})
+                 &idx->x_indeg, &idx->x_off, &idx->x_fill, &idx->x_src, &idx->st_ids, &idx->st_vecs, &idx->st_out_ids, &idx->st_out_d})
     if (b->p) idx->dev_free(b->p, idx->user);
+  for (auto e : idx->ctr_done)
+    if (e) cudaEventDestroy(e);
   if (idx->h_state) cudaFreeHost(idx->h_state);
   for (auto e : idx->ev_pool) cudaEventDestroy(e);
   for (auto e : idx->reader_pool) cudaEventDestroy(e);
@@ -423,35 +510,45 @@ int grand_destroy(grand_index* idx) {
   return GRAND_OK;
 }
 
+// An update call that gives up after validation has marked its ids: clear the marks, drain the stream, report.
+// Nothing of the index has been changed at the points where this is used, or the failure is a CUDA error.
+static int abandon_batch(grand_index* idx, const uint32_t* ids, uint64_t n, cudaStream_t s, int code, const std::string& msg) {
+  launch_clear_marks(ids, n, idx->cap, idx->mark, s);
+  cudaStreamSynchronize(s);
+  collect_spans(idx);
+  return fail(idx, code, msg);
+}
+#define CKB(call)                                                                                           \
+  do {                                                                                                      \
+    cudaError_t e__ = (call);                                                                               \
+    if (e__ != cudaSuccess)                                                                                 \
+      return abandon_batch(idx, ids, n, s, GRAND_ERR_CUDA, std::string(#call) + ": " + cudaGetErrorString(e__)); \
+  } while (0)
+
 int grand_insert_batch(grand_index* idx, const uint32_t* ids, const void* vecs, uint64_t n, grand_stream stream) {
   if (!idx || (n && (!ids || !vecs))) return fail(idx, GRAND_ERR_INVALID_ARG, "null argument");
   if (n == 0) return GRAND_OK;
   if (n > idx->max_batch) return fail(idx, GRAND_ERR_CAPACITY, "batch larger than max_batch");
+  LaunchScope scope(&idx->launches);
   cudaStream_t s = (cudaStream_t)stream;
   const bool fixed = idx->mode == GRAND_MODE_FIXED_DEGREE;
   const uint32_t R = idx->R;
   int rc;
   if ((rc = write_state_head(idx, s))) return rc;
-  if ((rc = begin_update(idx, ids, n, s))) return rc;
   {
     PhaseTimer pt(idx, s, PH_OTHER);
-    CK(launch_validate(ids, n, idx->cap, idx->live, idx->mark, 0, idx->d_state, s));
-    if (idx->mips) CK(launch_check_norms(idx->lay, vecs, n, idx->mips_M2, idx->d_state, s));
+    CKB(launch_validate(ids, n, idx->cap, idx->live, idx->mark, 0, idx->d_state, s));
+    if (idx->mips) CKB(launch_check_norms(idx->lay, vecs, n, idx->mips_M2, idx->d_state, s));
   }
-  if ((rc = read_state(idx, s))) return rc;
-  if (idx->h_state->status != 0) {
-    CK(launch_clear_marks(ids, n, idx->cap, idx->mark, s));
-    CK(cudaStreamSynchronize(s));
-    collect_spans(idx);
-    return fail(idx, idx->h_state->status, grand_strerror(idx->h_state->status));
-  }
-  if ((rc = ensure_requests(idx, n * R, s))) return rc;
+  if ((rc = read_state(idx, s))) return abandon_batch(idx, ids, n, s, rc, idx->last_error);
+  if (idx->h_state->status != 0) return abandon_batch(idx, ids, n, s, idx->h_state->status, grand_strerror(idx->h_state->status));
+  if ((rc = begin_update(idx, ids, n, s))) return abandon_batch(idx, ids, n, s, rc, idx->last_error);
   ++idx->epoch;
   GraphView g = view(idx, true);
   {
     PhaseTimer pt(idx, s, PH_OTHER);
-    CK(launch_store_write(idx->lay, idx->store, idx->deg, idx->slot_of, ids, vecs, n, s));
-    if (idx->mips) CK(launch_augment_rows(idx->lay, idx->store, ids, n, idx->mips_M2, s));
+    CKB(launch_store_write(idx->lay, idx->store, idx->deg, idx->slot_of, ids, vecs, n, s));
+    if (idx->mips) CKB(launch_augment_rows(idx->lay, idx->store, ids, n, idx->mips_M2, s));
   }
   const bool bootstrap = idx->nlive == 0;
   {
@@ -471,7 +568,7 @@ int grand_insert_batch(grand_index* idx, const uint32_t* ids, const void* vecs, 
     } else {
       a.out_vis = idx->wk_keys; a.out_vis_n = idx->wk_n; a.vis_stride = idx->wk_stride;
     }
-    CK(launch_beam_search(a, s));
+    CKB(launch_beam_search(a, s));
     idx->stats.n_search_launches++;
   }
   {
@@ -483,7 +580,8 @@ int grand_insert_batch(grand_index* idx, const uint32_t* ids, const void* vecs, 
     a.fixed_mode = fixed;
     a.req_tgt = (uint32_t*)idx->req_tgt.p; a.req_key = (unsigned long long*)idx->req_key.p;
     a.state = idx->d_state;
-    CK(launch_forward_prune(a, s));
+    CKB(launch_forward_prune(a, s));
+    idx->stats.n_prune_launches++;
   }
   {
     PhaseTimer pt(idx, s, PH_GROUP);
@@ -491,18 +589,19 @@ int grand_insert_batch(grand_index* idx, const uint32_t* ids, const void* vecs, 
     a.req_tgt = (uint32_t*)idx->req_tgt.p; a.req_key = (unsigned long long*)idx->req_key.p; a.nreq = n * R;
     a.cnt = idx->cnt; a.fill = idx->fill; a.start = idx->start; a.flag = idx->flag;
     a.dirty = (uint32_t*)idx->dirty.p; a.seg_keys = (unsigned long long*)idx->seg_keys.p; a.state = idx->d_state;
-    CK(launch_group_requests(a, s));
+    CKB(launch_group_requests(a, s));
   }
   {
     PhaseTimer pt(idx, s, PH_REBUILD);
-    const uint64_t mbk = n * R < 148u * 16u ? n * R : 148u * 16u;
+    const uint64_t most = (uint64_t)sm_count() * 16u;
+    const uint64_t mbk = n * R < most ? n * R : most;
     if (fixed) {
       FixedReverseArgs a{};
       a.g = g; a.slot_of = idx->slot_of; a.fwd_rows = (uint32_t*)idx->req_tgt.p;
       a.cnt = idx->cnt; a.fill = idx->fill; a.start = idx->start; a.flag = idx->flag;
       a.dirty = (uint32_t*)idx->dirty.p; a.seg_keys = (unsigned long long*)idx->seg_keys.p;
       a.max_blocks = (uint32_t)mbk; a.state = idx->d_state;
-      CK(launch_fixed_reverse(a, s));
+      CKB(launch_fixed_reverse(a, s));
     } else {
       RebuildArgs a{};
       a.lay = idx->lay; a.g = g; a.A_fix = idx->A_fix; a.alpha = idx->alpha; a.P = idx->P; a.delmap = nullptr;
@@ -510,13 +609,14 @@ int grand_insert_batch(grand_index* idx, const uint32_t* ids, const void* vecs, 
       a.cnt = idx->cnt; a.fill = idx->fill; a.start = idx->start; a.flag = idx->flag;
       a.dirty = (uint32_t*)idx->dirty.p; a.seg_keys = (unsigned long long*)idx->seg_keys.p;
       a.max_blocks = (uint32_t)mbk; a.state = idx->d_state;
-      CK(launch_rebuild(a, s));
+      CKB(launch_rebuild(a, s));
+      idx->stats.n_rebuild_launches++;
     }
   }
   {
     PhaseTimer pt(idx, s, PH_OTHER);
-    CK(launch_publish(ids, n, idx->live, idx->mark, idx->d_state, s));
-    if (idx->entry == GRAND_INVALID_ID) CK(launch_pick_medoid(idx->lay, g, ids, n, idx->mean_row, idx->d_state, s));
+    CKB(launch_publish(ids, n, idx->live, idx->mark, idx->d_state, s));
+    if (idx->entry == GRAND_INVALID_ID) CKB(launch_pick_medoid(idx->lay, g, ids, n, idx->mean_row, idx->d_state, s));
   }
   if ((rc = read_state(idx, s))) return rc;
   collect_spans(idx);
@@ -525,17 +625,25 @@ int grand_insert_batch(grand_index* idx, const uint32_t* ids, const void* vecs, 
   return GRAND_OK;
 }
 
-static int build_reverse(grand_index* idx, bool sort_rows, const uint32_t* heads, bool work, cudaStream_t s) {
+// Reverse graph of the current adjacency (Alg. 8, first loops).  heads != nullptr: only the rows of the marked nodes,
+// into the buffers sized at creation (an update batch); heads == nullptr and !work: the whole graph for
+// grand_reverse_graph, into buffers that grow on demand (introspection is the only caller that may allocate).
+static int build_reverse(grand_index* idx, bool sort_rows, const uint32_t* heads, bool work, bool introspection, cudaStream_t s) {
   int rc;
   const uint64_t cap = idx->cap;
-  if ((rc = ensure(idx, idx->t_indeg, (cap + 1) * 4, s))) return rc;
-  if ((rc = ensure(idx, idx->t_off, (cap + 1) * 4, s))) return rc;
-  if ((rc = ensure(idx, idx->t_fill, cap * 4, s))) return rc;
-  if ((rc = ensure(idx, idx->t_src, cap * idx->R * 4, s))) return rc;
+  Buf *indeg = &idx->t_indeg, *off = &idx->t_off, *fillc = &idx->t_fill, *src = &idx->t_src;
+  if (introspection) {
+    indeg = &idx->x_indeg; off = &idx->x_off; fillc = &idx->x_fill; src = &idx->x_src;
+    if ((rc = ensure(idx, *indeg, (cap + 1) * 4, s))) return rc;
+    if ((rc = ensure(idx, *off, (cap + 1) * 4, s))) return rc;
+    if ((rc = ensure(idx, *fillc, cap * 4, s))) return rc;
+    if ((rc = ensure(idx, *src, cap * idx->R * 4, s))) return rc;
+  }
   TransposeArgs t{};
   t.g = view(idx, work);
-  t.indeg = (uint32_t*)idx->t_indeg.p; t.off = (uint32_t*)idx->t_off.p; t.fillc = (uint32_t*)idx->t_fill.p;
-  t.src = (uint32_t*)idx->t_src.p; t.scan_tmp = idx->scan_tmp; t.sort_rows = sort_rows; t.heads = heads;
+  t.indeg = (uint32_t*)indeg->p; t.off = (uint32_t*)off->p; t.fillc = (uint32_t*)fillc->p;
+  t.src = (uint32_t*)src->p; t.scan_tmp = idx->scan_tmp; t.sort_rows = sort_rows; t.heads = heads;
+  t.src_capacity = src->bytes / 4;
   CK(launch_transpose(t, s));
   return GRAND_OK;
 }
@@ -544,16 +652,19 @@ int grand_delete_batch(grand_index* idx, const uint32_t* ids, uint64_t n, grand_
   if (!idx || (n && !ids)) return fail(idx, GRAND_ERR_INVALID_ARG, "null argument");
   if (n == 0) return GRAND_OK;
   if (n > idx->max_batch) return fail(idx, GRAND_ERR_CAPACITY, "batch larger than max_batch");
+  LaunchScope scope(&idx->launches);
   cudaStream_t s = (cudaStream_t)stream;
   const bool fixed = idx->mode == GRAND_MODE_FIXED_DEGREE;
   const uint32_t R = idx->R;
   int rc;
   if ((rc = write_state_head(idx, s))) return rc;
-  if ((rc = begin_update(idx, ids, n, s))) return rc;
   {
     PhaseTimer pt(idx, s, PH_OTHER);
-    CK(launch_validate(ids, n, idx->cap, idx->live, idx->mark, 1, idx->d_state, s));
+    CKB(launch_validate(ids, n, idx->cap, idx->live, idx->mark, 1, idx->d_state, s));
   }
+  // (the status of the validation is read back together with the in-degree total below: what runs in between
+  // only reads the graph and writes scratch, and skips ids beyond the capacity)
+  if ((rc = begin_update(idx, ids, n, s))) return abandon_batch(idx, ids, n, s, rc, idx->last_error);
   ++idx->epoch;
   GraphView g = view(idx, true);
   DeleteArgs d{};
@@ -567,17 +678,14 @@ int grand_delete_batch(grand_index* idx, const uint32_t* ids, uint64_t n, grand_
     // reverse graph of the snapshot: exact in-neighbours, rebuilt per batch and not kept
     PhaseTimer pt(idx, s, PH_TRANSPOSE);
     // only the in-neighbour rows of the batch are read below, so only those are materialised
-    if ((rc = build_reverse(idx, false, idx->full_transpose ? nullptr : idx->mark, true, s))) return rc;
+    if ((rc = build_reverse(idx, false, idx->full_transpose ? nullptr : idx->mark, true, false, s)))
+      return abandon_batch(idx, ids, n, s, rc, idx->last_error);
+    idx->stats.n_transpose_launches++;
     d.off = (uint32_t*)idx->t_off.p; d.src = (uint32_t*)idx->t_src.p;
-    CK(launch_delete_prepare(d, s));
+    CKB(launch_delete_prepare(d, s));
   }
-  if ((rc = read_state(idx, s))) return rc;
-  if (idx->h_state->status != 0) {
-    CK(launch_clear_marks(ids, n, idx->cap, idx->mark, s));
-    CK(cudaStreamSynchronize(s));
-    collect_spans(idx);
-    return fail(idx, idx->h_state->status, grand_strerror(idx->h_state->status));
-  }
+  if ((rc = read_state(idx, s))) return abandon_batch(idx, ids, n, s, rc, idx->last_error);
+  if (idx->h_state->status != 0) return abandon_batch(idx, ids, n, s, idx->h_state->status, grand_strerror(idx->h_state->status));
   if (approx) {
     // Alg. 6 as printed: the searches come first, their visited sets are the only place where
     // in-neighbours are looked for
@@ -587,39 +695,50 @@ int grand_delete_batch(grand_index* idx, const uint32_t* ids, uint64_t n, grand_
       a.qids = ids; a.nq = n; a.L = idx->L; a.vmax = idx->vmax;
       a.out_beam = idx->wk_keys; a.out_beam_n = idx->wk_n; a.beam_stride = idx->wk_stride;
       a.out_vis = idx->vis_keys; a.out_vis_n = idx->vis_n; a.vis_stride = idx->vmax;
-      CK(launch_beam_search(a, s));
+      CKB(launch_beam_search(a, s));
       idx->stats.n_search_launches++;
     }
-    PhaseTimer pt(idx, s, PH_TRANSPOSE);
-    d.vis = idx->vis_keys; d.vis_n = idx->vis_n; d.vis_stride = idx->vmax;
-    d.src = idx->vis_in; d.src_stride = idx->vmax; d.livemap = idx->live;
-    CK(launch_delete_visited_in(d, idx->vis_in, s));
+    {
+      PhaseTimer pt(idx, s, PH_TRANSPOSE);
+      d.vis = idx->vis_keys; d.vis_n = idx->vis_n; d.vis_stride = idx->vmax;
+      d.src = idx->vis_in; d.src_stride = idx->vmax; d.livemap = idx->live;
+      CKB(launch_delete_visited_in(d, idx->vis_in, s));
+    }
+    if ((rc = read_state(idx, s))) return abandon_batch(idx, ids, n, s, rc, idx->last_error);
   }
-  if (approx && (rc = read_state(idx, s))) return rc;
   const uint64_t total_in = idx->h_state->total_in;
   const uint64_t nreq = fixed ? total_in + 1 : (total_in + n * R) * idx->c;
-  if (nreq >= (1ull << 32)) return fail(idx, GRAND_ERR_CAPACITY, "delete batch touches too many edges");
-  if ((rc = ensure_requests(idx, nreq, s))) return rc;
+  // nothing of the index has been written so far: a batch that touches more edges than the workspace was sized
+  // for is refused as a whole
+  if (total_in > idx->max_delete_edges || nreq > idx->max_requests)
+    return abandon_batch(idx, ids, n, s, GRAND_ERR_CAPACITY,
+                         "delete batch touches " + std::to_string(total_in) + " in-neighbour entries; the workspace holds " +
+                             std::to_string(idx->max_delete_edges) + " (option max_delete_edges)");
   d.req_tgt = (uint32_t*)idx->req_tgt.p; d.req_key = (unsigned long long*)idx->req_key.p; d.dirty = (uint32_t*)idx->dirty.p;
   if (fixed) {
     PhaseTimer pt(idx, s, PH_REBUILD);
     FixedDeleteArgs f{};
     f.g = g; f.ids = ids; f.n = n; f.delmap = idx->mark; f.off = d.off; f.src = d.src; f.pair_off = idx->pair_off;
     f.flag = idx->flag; f.dirty = (uint32_t*)idx->dirty.p; f.state = idx->d_state;
-    CK(launch_fixed_delete(f, total_in, s));
+    CKB(launch_fixed_delete(f, total_in, s));
   } else {
     if (!approx) {
       PhaseTimer pt(idx, s, PH_SEARCH);
       SearchArgs a = search_args(idx, s, true);
       a.qids = ids; a.nq = n; a.L = idx->L; a.vmax = idx->vmax;
       a.out_beam = idx->wk_keys; a.out_beam_n = idx->wk_n; a.beam_stride = idx->wk_stride;
-      CK(launch_beam_search(a, s));
+      CKB(launch_beam_search(a, s));
       idx->stats.n_search_launches++;
     }
     {
+      PhaseTimer pt(idx, s, PH_GROUP);  // set-up of the picks: C_i, dirty marks of the in-neighbours, work units
+      CKB(launch_delete_ci(d, s));
+      CKB(launch_delete_picks_prepare(d, total_in, s));
+    }
+    {
       PhaseTimer pt(idx, s, PH_PICKS);
-      CK(launch_delete_ci(d, s));
-      CK(launch_delete_picks(d, total_in, s));
+      CKB(launch_delete_picks(d, total_in, s));
+      idx->stats.n_picks_launches++;
     }
     {
       PhaseTimer pt(idx, s, PH_GROUP);
@@ -627,7 +746,7 @@ int grand_delete_batch(grand_index* idx, const uint32_t* ids, uint64_t n, grand_
       a.req_tgt = d.req_tgt; a.req_key = d.req_key; a.nreq = nreq;
       a.cnt = idx->cnt; a.fill = idx->fill; a.start = idx->start; a.flag = idx->flag;
       a.dirty = d.dirty; a.seg_keys = (unsigned long long*)idx->seg_keys.p; a.state = idx->d_state;
-      CK(launch_group_requests(a, s));
+      CKB(launch_group_requests(a, s));
     }
     {
       PhaseTimer pt(idx, s, PH_REBUILD);
@@ -636,13 +755,15 @@ int grand_delete_batch(grand_index* idx, const uint32_t* ids, uint64_t n, grand_
       if (approx) a.livemap = idx->live;
       a.cnt = idx->cnt; a.fill = idx->fill; a.start = idx->start; a.flag = idx->flag;
       a.dirty = d.dirty; a.seg_keys = (unsigned long long*)idx->seg_keys.p;
-      a.max_blocks = (uint32_t)(nreq < 148u * 16u ? nreq : 148u * 16u); a.state = idx->d_state;
-      CK(launch_rebuild(a, s));
+      const uint64_t most = (uint64_t)sm_count() * 16u;
+      a.max_blocks = (uint32_t)(nreq < most ? nreq : most); a.state = idx->d_state;
+      CKB(launch_rebuild(a, s));
+      idx->stats.n_rebuild_launches++;
     }
   }
   {
     PhaseTimer pt(idx, s, PH_OTHER);
-    CK(launch_retire(g, ids, n, idx->mark, idx->Ci, idx->Ci_n, idx->k_repair, fixed, idx->d_state, s));
+    CKB(launch_retire(g, ids, n, idx->mark, idx->Ci, idx->Ci_n, idx->k_repair, fixed, idx->d_state, s));
   }
   if ((rc = read_state(idx, s))) return rc;
   collect_spans(idx);
@@ -662,11 +783,14 @@ int grand_search(const grand_index* cidx, const void* queries, uint64_t nq, uint
     // the lock keeps the choice of the published buffer, the launch and the registration of the launch's end
     // as a reader of that buffer together (an update batch on another host thread may publish at any time)
     std::lock_guard<std::mutex> lk(idx->pub_mu);
+    LaunchScope scope(&idx->launches);
     PhaseTimer pt(idx, s, PH_SEARCH);
-    SearchArgs a = search_args(idx, s, false);
+    const int slot = take_ctr_slot(idx);
+    SearchArgs a = search_args(idx, s, false, slot);
     a.queries = queries; a.nq = nq; a.L = L; a.vmax = 2 * L; a.k = k;
     a.out_ids = out_ids; a.out_dists = out_dists;
     CK(launch_beam_search(a, s));
+    if (slot >= 0) CK(cudaEventRecord(idx->ctr_done[slot], s));
     idx->stats.n_search_launches++;
     if (idx->snap) {
       std::vector<cudaEvent_t>& rd = idx->readers[idx->pub];
@@ -700,10 +824,11 @@ int grand_search(const grand_index* cidx, const void* queries, uint64_t nq, uint
 int grand_insert_batch_host(grand_index* idx, const uint32_t* ids, const void* vecs, uint64_t n, grand_stream stream) {
   if (!idx || (n && (!ids || !vecs))) return fail(idx, GRAND_ERR_INVALID_ARG, "null argument");
   if (n == 0) return GRAND_OK;
+  if (n > idx->max_batch) return fail(idx, GRAND_ERR_CAPACITY, "batch larger than max_batch");
   cudaStream_t s = (cudaStream_t)stream;
   int rc;
   const size_t vb = (size_t)n * idx->lay.udim * idx->lay.esize;
-  if ((rc = ensure(idx, idx->st_ids, n * 4, s))) return rc;
+  if ((rc = ensure(idx, idx->st_ids, n * 4, s))) return rc;  // (sized for max_batch at creation: no allocation here)
   if ((rc = ensure(idx, idx->st_vecs, vb, s))) return rc;
   CK(cudaMemcpyAsync(idx->st_ids.p, ids, n * 4, cudaMemcpyHostToDevice, s));
   CK(cudaMemcpyAsync(idx->st_vecs.p, vecs, vb, cudaMemcpyHostToDevice, s));
@@ -712,6 +837,7 @@ int grand_insert_batch_host(grand_index* idx, const uint32_t* ids, const void* v
 int grand_delete_batch_host(grand_index* idx, const uint32_t* ids, uint64_t n, grand_stream stream) {
   if (!idx || (n && !ids)) return fail(idx, GRAND_ERR_INVALID_ARG, "null argument");
   if (n == 0) return GRAND_OK;
+  if (n > idx->max_batch) return fail(idx, GRAND_ERR_CAPACITY, "batch larger than max_batch");
   cudaStream_t s = (cudaStream_t)stream;
   int rc;
   if ((rc = ensure(idx, idx->st_ids, n * 4, s))) return rc;
@@ -750,6 +876,13 @@ int grand_import_graph(grand_index* idx, const uint32_t* adj, const uint32_t* de
                        const void* vecs, grand_stream stream) {
   if (!idx || !adj || !deg || !live || !vecs) return fail(idx, GRAND_ERR_INVALID_ARG, "null argument");
   cudaStream_t s = (cudaStream_t)stream;
+  LaunchScope scope(&idx->launches);
+  int rc;
+  // the caller's graph is checked before anything is replaced: degrees <= R, listed neighbour ids < capacity
+  if ((rc = write_state_head(idx, s))) return rc;
+  CK(launch_check_graph(adj, deg, idx->cap, idx->R, idx->d_state, s));
+  if ((rc = read_state(idx, s))) return rc;
+  if (idx->h_state->status != 0) return fail(idx, GRAND_ERR_INVALID_ARG, "imported graph: a degree above R or a neighbour id beyond the capacity");
   CK(cudaMemcpyAsync(idx->adj, adj, (size_t)idx->cap * idx->R * 4, cudaMemcpyDeviceToDevice, s));
   idx->sync_n = idx->sync_ndirty = 0;  // both buffers are rewritten below
   CK(cudaMemcpyAsync(idx->deg, deg, idx->cap * 4, cudaMemcpyDeviceToDevice, s));
@@ -766,7 +899,6 @@ int grand_import_graph(grand_index* idx, const uint32_t* adj, const uint32_t* de
   if (idx->snap) CK(cudaMemcpyAsync(idx->adj_alt, idx->adj, (size_t)idx->cap * idx->R * 4, cudaMemcpyDeviceToDevice, s));
   idx->entry = entry;
   idx->nlive = 0;
-  int rc;
   if ((rc = write_state_head(idx, s))) return rc;
   CK(launch_count_live(idx->live, idx->cap, idx->d_state, s));
   if ((rc = read_state(idx, s))) return rc;
@@ -776,13 +908,14 @@ int grand_import_graph(grand_index* idx, const uint32_t* adj, const uint32_t* de
 int grand_reverse_graph(grand_index* idx, uint32_t* off, uint32_t* src, uint64_t* E_out, grand_stream stream) {
   if (!idx) return GRAND_ERR_INVALID_ARG;
   cudaStream_t s = (cudaStream_t)stream;
+  LaunchScope scope(&idx->launches);
   int rc;
-  if ((rc = build_reverse(idx, true, nullptr, false, s))) return rc;
+  if ((rc = build_reverse(idx, true, nullptr, false, true, s))) return rc;
   uint32_t E = 0;
-  CK(cudaMemcpyAsync(&E, (uint32_t*)idx->t_off.p + idx->cap, 4, cudaMemcpyDeviceToHost, s));
+  CK(cudaMemcpyAsync(&E, (uint32_t*)idx->x_off.p + idx->cap, 4, cudaMemcpyDeviceToHost, s));
   CK(cudaStreamSynchronize(s));
-  if (off) CK(cudaMemcpyAsync(off, idx->t_off.p, (idx->cap + 1) * 4, cudaMemcpyDeviceToDevice, s));
-  if (src && E) CK(cudaMemcpyAsync(src, idx->t_src.p, (size_t)E * 4, cudaMemcpyDeviceToDevice, s));
+  if (off) CK(cudaMemcpyAsync(off, idx->x_off.p, (idx->cap + 1) * 4, cudaMemcpyDeviceToDevice, s));
+  if (src && E) CK(cudaMemcpyAsync(src, idx->x_src.p, (size_t)E * 4, cudaMemcpyDeviceToDevice, s));
   if (E_out) *E_out = E;
   CK(cudaStreamSynchronize(s));
   return GRAND_OK;
@@ -820,16 +953,18 @@ int grand_get_stats(const grand_index* cidx, grand_stats* out) {
   idx->stats.dirty_nodes = st.counters[CTR_DIRTY];
   idx->stats.prunes = st.counters[CTR_PRUNE];
   idx->stats.requests = st.counters[CTR_REQ];
-  idx->stats.kernel_launches = launches_so_far();
+  idx->stats.rebuild_bytes = st.counters[CTR_RB_BYTES];
+  idx->stats.picks_bytes = st.counters[CTR_PK_BYTES];
+  idx->stats.prune_bytes = st.counters[CTR_FP_BYTES];
+  idx->stats.rebuild_prunes = st.counters[CTR_RB_PRUNED];
+  idx->stats.kernel_launches = idx->launches;
   *out = idx->stats;
   return GRAND_OK;
 }
 int grand_reset_stats(grand_index* idx) {
   if (!idx) return GRAND_ERR_INVALID_ARG;
   CK(cudaMemset(idx->d_state->counters, 0, sizeof(idx->d_state->counters)));
-  const uint64_t keep = idx->stats.kernel_launches;
-  idx->stats = grand_stats{};
-  idx->stats.kernel_launches = keep;
+  idx->stats = grand_stats{};  // (kernel_launches is refilled from the handle's running count)
   return GRAND_OK;
 }
 int grand_set_profiling(grand_index* idx, int on) {

@@ -30,7 +30,8 @@ __global__ void delete_incnt_kernel(const DeleteArgs a) {
 __global__ void delete_total_kernel(const uint32_t* pair_off, uint64_t n, DevState* st) { st->total_in = pair_off[n]; }
 
 cudaError_t launch_delete_prepare(const DeleteArgs& a, cudaStream_t s) {
-  const unsigned blocks = (unsigned)((a.n + 256) / 256 > 148u * 16u ? 148u * 16u : (a.n + 256) / 256);
+  const uint64_t cap16 = (uint64_t)sm_count() * 16u;
+  const unsigned blocks = (unsigned)((a.n + 256) / 256 > cap16 ? cap16 : (a.n + 256) / 256);
   delete_incnt_kernel<<<blocks, 256, 0, s>>>(a);
   cudaError_t e = launch_exclusive_scan(a.in_cnt, a.pair_off, a.n + 1, a.scan_tmp, s);
   if (e != cudaSuccess) return e;
@@ -64,7 +65,7 @@ __global__ void delete_visited_in_kernel(const DeleteArgs a, uint32_t* inlist) {
 cudaError_t launch_delete_visited_in(const DeleteArgs& a, uint32_t* inlist, cudaStream_t s) {
   cudaMemsetAsync(a.in_cnt, 0, (a.n + 1) * 4, s);
   uint64_t blocks = (a.n * a.vis_stride + 3) / 4;
-  if (blocks > 148u * 32u) blocks = 148u * 32u;
+  if (blocks > (uint64_t)sm_count() * 32u) blocks = (uint64_t)sm_count() * 32u;
   delete_visited_in_kernel<<<(unsigned)blocks, 128, 0, s>>>(a, inlist);
   cudaError_t e = launch_exclusive_scan(a.in_cnt, a.pair_off, a.n + 1, a.scan_tmp, s);
   if (e != cudaSuccess) return e;
@@ -79,6 +80,7 @@ __global__ void delete_ci_kernel(const DeleteArgs a) {
   const int lane = threadIdx.x & 31;
   const uint64_t wglobal = (blockIdx.x * (uint64_t)blockDim.x + threadIdx.x) >> 5;
   const uint64_t wtotal = ((uint64_t)gridDim.x * blockDim.x) >> 5;
+  unsigned long long ncand = 0;
   for (uint64_t i = wglobal; i < a.n; i += wtotal) {
     const uint32_t nb = min(a.beam_n[i], a.beam_stride);
     uint32_t nc = 0;
@@ -95,11 +97,17 @@ __global__ void delete_ci_kernel(const DeleteArgs a) {
       if (ok && pos < a.k_repair) a.Ci[i * a.k_repair + pos] = k;
       nc += __popc(bal);
     }
-    if (lane == 0) a.Ci_n[i] = min(nc, a.k_repair);
+    if (lane == 0) {
+      a.Ci_n[i] = min(nc, a.k_repair);
+      ncand += min(nc, a.k_repair);
+    }
   }
+  // the repair has to fetch every candidate row once per deleted node
+  if (lane == 0 && ncand) atomicAdd(&a.state->counters[CTR_PK_BYTES], ncand * a.lay.row_bytes);
 }
 cudaError_t launch_delete_ci(const DeleteArgs& a, cudaStream_t s) {
-  const unsigned blocks = (unsigned)((a.n + 3) / 4 > 148u * 16u ? 148u * 16u : (a.n + 3) / 4);
+  const uint64_t cap16 = (uint64_t)sm_count() * 16u;
+  const unsigned blocks = (unsigned)((a.n + 3) / 4 > cap16 ? cap16 : (a.n + 3) / 4);
   delete_ci_kernel<<<blocks ? blocks : 1, 128, 0, s>>>(a);
   count_launches(1);
   return cudaGetLastError();
@@ -119,7 +127,7 @@ __global__ void __launch_bounds__(kPickWarps * 32) delete_picks_kernel(const Del
   const uint32_t row_bytes = a.lay.row_bytes, nchunk = a.lay.nchunk;
   const uint64_t total = total_in + a.n * R;
   const uint64_t wglobal = (uint64_t)blockIdx.x * kPickWarps + warp, wtotal = (uint64_t)gridDim.x * kPickWarps;
-  unsigned long long npair = 0;
+  unsigned long long npair = 0, nrows = 0;
   for (uint64_t pair = wglobal; pair < total; pair += wtotal) {
     const bool is_in = pair < total_in;
     uint64_t i;
@@ -148,6 +156,7 @@ __global__ void __launch_bounds__(kPickWarps * 32) delete_picks_kernel(const Del
     uint4 xr[CPL];
     load_row<G, CPL>(a.g.store + (size_t)x * row_bytes, nchunk, t, xr);
     const uint32_t nc = a.Ci_n[i];
+    if (lane == 0) ++nrows;  // rows the method has to fetch here: x once per pair (C_i is charged where it is formed)
     constexpr int U = CPL == 1 ? 4 : (CPL == 2 ? 2 : 1);  // candidate rows in flight per team
     for (uint32_t jb = 0; jb < nc; jb += NT * U) {
       uint4 v[U][CPL];
@@ -198,6 +207,7 @@ __global__ void __launch_bounds__(kPickWarps * 32) delete_picks_kernel(const Del
     }
   }
   if (npair) atomicAdd(&a.state->counters[CTR_PAIR], npair);
+  if (nrows) atomicAdd(&a.state->counters[CTR_PK_BYTES], nrows * row_bytes);
 }
 // Every surviving in-neighbour of a deleted node is dirty even if it receives no candidate.
 __global__ void delete_touch_kernel(const DeleteArgs a, const uint64_t total_in) {
@@ -252,7 +262,7 @@ __global__ void __launch_bounds__(kPickWarps * 32) delete_picks_staged_kernel(co
                                       (size_t)kPickWarps * nchunk);  // |y|^2 of the staged rows (integer rows only)
   uint32_t* xid = reinterpret_cast<uint32_t*>(cnorm + kr);  // the unit's x ids (invalid id = nothing to do for the pair)
   const uint32_t nunits = a.unit_off[a.n];
-  unsigned long long npair = 0;
+  unsigned long long npair = 0, nrows = 0;
   for (uint32_t unit = blockIdx.x; unit < nunits; unit += gridDim.x) {
     uint32_t lo = 0, hi = (uint32_t)a.n;  // largest i with unit_off[i] <= unit
     while (hi - lo > 1) {
@@ -304,6 +314,7 @@ __global__ void __launch_bounds__(kPickWarps * 32) delete_picks_staged_kernel(co
         if (lane < c) a.req_tgt[rbase + lane] = kInvalid;
         continue;
       }
+      if (lane == 0) ++nrows;  // x's row, fetched once per pair
       if constexpr (sizeof(T) == 1) {
         // integer rows: any summation order gives the same distance, so one lane takes one candidate and walks
         // its staged row against x's row (a broadcast read); the keys stay in registers
@@ -406,6 +417,7 @@ __global__ void __launch_bounds__(kPickWarps * 32) delete_picks_staged_kernel(co
     }
   }
   if (npair) atomicAdd(&a.state->counters[CTR_PAIR], npair);
+  if (nrows) atomicAdd(&a.state->counters[CTR_PK_BYTES], nrows * row_bytes);
 }
 
 // ---- tensor-core variant for integer rows.  All pairs (x, y) of one deleted node, x among its surviving in- and
@@ -441,7 +453,7 @@ __global__ void __launch_bounds__(kMmaWarps * 32) delete_picks_mma_kernel(const 
   int* xnorm = cnorm + NC;
   uint32_t* xid = reinterpret_cast<uint32_t*>(xnorm + kMmaUnitPairs);
   const uint32_t nunits = a.unit_off[a.n];
-  unsigned long long npair = 0;
+  unsigned long long npair = 0, nrows = 0;
   for (uint32_t unit = blockIdx.x; unit < nunits; unit += gridDim.x) {
     uint32_t lo = 0, hi = (uint32_t)a.n;  // largest i with unit_off[i] <= unit
     while (hi - lo > 1) {
@@ -551,72 +563,89 @@ __global__ void __launch_bounds__(kMmaWarps * 32) delete_picks_mma_kernel(const 
           }
           prev = best;
         }
-        if (tig == 0 && r < M && x != kInvalid) npair += nc;
+        if (tig == 0 && r < M && x != kInvalid) {
+          npair += nc;
+          ++nrows;  // x's row, fetched once per pair
+        }
       }
     }
   }
   if (npair) atomicAdd(&a.state->counters[CTR_PAIR], npair);
+  if (nrows) atomicAdd(&a.state->counters[CTR_PK_BYTES], nrows * row_bytes);
+}
+
+// Which pick kernel serves this index: 2 = tensor-core tiles (integer rows up to 256 bytes, k_repair <= 56),
+// 1 = candidate rows staged in shared memory, 0 = rows straight from L2.
+template <typename T>
+static int picks_variant(const DeleteArgs& a) {
+  if (sizeof(T) == 1 && a.k_repair <= (uint32_t)kMmaNTiles * 8u && a.lay.row_bytes <= 256u) return 2;
+  const size_t stage = (size_t)a.k_repair * ((a.lay.nchunk | 1u) * 16u);
+  return stage <= 64 * 1024 ? 1 : 0;
+}
+
+template <typename T, int METRIC, int G, int CPL>
+static cudaError_t launch_delete_picks_prepare_t(const DeleteArgs& a, uint64_t total_in, cudaStream_t s) {
+  const uint64_t total = total_in + a.n * a.g.R;
+  if (total == 0) return cudaSuccess;
+  if (total_in) {
+    uint64_t tb = (total_in + 255) / 256;
+    if (tb > (uint64_t)sm_count() * 32u) tb = (uint64_t)sm_count() * 32u;
+    delete_touch_kernel<<<(unsigned)tb, 256, 0, s>>>(a, total_in);
+    count_launches(1);
+  }
+  const int variant = picks_variant<T>(a);
+  if (variant == 0) return cudaGetLastError();
+  const uint64_t cap16 = (uint64_t)sm_count() * 16u;
+  const unsigned ub = (unsigned)((a.n + 256) / 256 > cap16 ? cap16 : (a.n + 256) / 256);
+  delete_units_kernel<<<ub, 256, 0, s>>>(a, variant == 2 ? kMmaUnitPairs : kUnitPairs);
+  count_launches(1);
+  return launch_exclusive_scan(a.in_cnt, a.unit_off, a.n + 1, a.scan_tmp, s);
 }
 
 template <typename T, int METRIC, int G, int CPL>
 static cudaError_t launch_delete_picks_t(const DeleteArgs& a, uint64_t total_in, cudaStream_t s) {
   const uint64_t total = total_in + a.n * a.g.R;
   if (total == 0) return cudaSuccess;
-  if (total_in) {
-    uint64_t tb = (total_in + 255) / 256;
-    if (tb > 148u * 32u) tb = 148u * 32u;
-    delete_touch_kernel<<<(unsigned)tb, 256, 0, s>>>(a, total_in);
-    count_launches(1);
-  }
+  const int variant = picks_variant<T>(a);
+  const uint64_t sms = (uint64_t)sm_count();
   if constexpr (sizeof(T) == 1) {
-    if (a.k_repair <= (uint32_t)kMmaNTiles * 8u && a.lay.row_bytes <= 256u) {
+    if (variant == 2) {
       const size_t smem = delete_picks_mma_smem(a.lay.row_bytes);
       auto kern = delete_picks_mma_kernel<T>;
-      // (one kernel serves every row layout of this element type, so the limit is raised once, to the largest case)
-      static bool smem_set = false;
-      if (!smem_set) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)delete_picks_mma_smem(256u));
-        if (e != cudaSuccess) return e;
-        smem_set = true;
-      }
-      const unsigned ub = (unsigned)((a.n + 256) / 256 > 148u * 16u ? 148u * 16u : (a.n + 256) / 256);
-      delete_units_kernel<<<ub, 256, 0, s>>>(a, kMmaUnitPairs);
-      cudaError_t e = launch_exclusive_scan(a.in_cnt, a.unit_off, a.n + 1, a.scan_tmp, s);
+      static SmemOptIn optin{};
+      cudaError_t e = allow_full_dynamic_smem((const void*)kern, &optin);
       if (e != cudaSuccess) return e;
       uint64_t blocks = (total + kMmaUnitPairs - 1) / kMmaUnitPairs + a.n;  // upper bound on the number of units
-      if (blocks > 148u * 8u) blocks = 148u * 8u;
+      if (blocks > sms * 8u) blocks = sms * 8u;
       kern<<<(unsigned)blocks, kMmaWarps * 32, smem, s>>>(a, total_in);
-      count_launches(2);
+      count_launches(1);
       return cudaGetLastError();
     }
   }
-  const size_t stage = (size_t)a.k_repair * ((a.lay.nchunk | 1u) * 16u);
-  if (stage <= 64 * 1024) {
+  if (variant == 1) {
     // candidate rows fit shared memory: one staged copy per work unit
+    const size_t stage = (size_t)a.k_repair * ((a.lay.nchunk | 1u) * 16u);
     const size_t smem = stage + ((size_t)((a.k_repair + 1u) & ~1u) + (size_t)kPickWarps * kMaxKRepair) * 8 +
                         (size_t)kPickWarps * a.lay.row_bytes + (size_t)a.k_repair * 4 + (size_t)kUnitPairs * 4;
     auto kern = delete_picks_staged_kernel<T, METRIC, G, CPL>;
-    static size_t smem_set = 0;
-    if (smem > smem_set) {
-      cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-      if (e != cudaSuccess) return e;
-      smem_set = smem;
-    }
-    const unsigned ub = (unsigned)((a.n + 256) / 256 > 148u * 16u ? 148u * 16u : (a.n + 256) / 256);
-    delete_units_kernel<<<ub, 256, 0, s>>>(a, kUnitPairs);
-    cudaError_t e = launch_exclusive_scan(a.in_cnt, a.unit_off, a.n + 1, a.scan_tmp, s);
+    static SmemOptIn optin{};
+    cudaError_t e = allow_full_dynamic_smem((const void*)kern, &optin);
     if (e != cudaSuccess) return e;
     uint64_t blocks = (total + kUnitPairs - 1) / kUnitPairs + a.n;  // upper bound on the number of units
-    if (blocks > 148u * 16u) blocks = 148u * 16u;
+    if (blocks > sms * 16u) blocks = sms * 16u;
     kern<<<(unsigned)blocks, kPickWarps * 32, smem, s>>>(a, total_in);
-    count_launches(2);
+    count_launches(1);
     return cudaGetLastError();
   }
   uint64_t blocks = (total + kPickWarps - 1) / kPickWarps;
-  if (blocks > 148u * 16u) blocks = 148u * 16u;
+  if (blocks > sms * 16u) blocks = sms * 16u;
   delete_picks_kernel<T, METRIC, G, CPL><<<(unsigned)blocks, kPickWarps * 32, 0, s>>>(a, total_in);
   count_launches(1);
   return cudaGetLastError();
+}
+cudaError_t launch_delete_picks_prepare(const DeleteArgs& a, uint64_t total_in, cudaStream_t s) {
+  GRAND_DISPATCH_L2(a.lay, launch_delete_picks_prepare_t, a, total_in, s);
+  return cudaErrorInvalidValue;
 }
 cudaError_t launch_delete_picks(const DeleteArgs& a, uint64_t total_in, cudaStream_t s) {
   GRAND_DISPATCH_L2(a.lay, launch_delete_picks_t, a, total_in, s);
@@ -697,11 +726,11 @@ __global__ void __launch_bounds__(128) fixed_delete_rewire_kernel(const FixedDel
 cudaError_t launch_fixed_delete(const FixedDeleteArgs& a, uint64_t total_in, cudaStream_t s) {
   if (total_in) {
     uint64_t blocks = (total_in + 255) / 256;
-    if (blocks > 148u * 32u) blocks = 148u * 32u;
+    if (blocks > (uint64_t)sm_count() * 32u) blocks = (uint64_t)sm_count() * 32u;
     fixed_delete_mark_kernel<<<(unsigned)blocks, 256, 0, s>>>(a, total_in);
     count_launches(1);
   }
-  fixed_delete_rewire_kernel<<<148 * 8, 128, 0, s>>>(a);
+  fixed_delete_rewire_kernel<<<(unsigned)sm_count() * 8u, 128, 0, s>>>(a);
   count_launches(1);
   return cudaGetLastError();
 }
@@ -766,7 +795,7 @@ static cudaError_t launch_pick_medoid_t(const Layout& lay, const GraphView& g, c
   medoid_begin_kernel<<<1, 1, 0, s>>>(st);
   medoid_mean_kernel<T><<<(lay.row_bytes / sizeof(T) + 127) / 128, 128, 0, s>>>(g.store, ids, n, lay.dim, lay.row_bytes, mean_row);
   uint64_t blocks = (n + 3) / 4;
-  if (blocks > 148u * 8u) blocks = 148u * 8u;
+  if (blocks > (uint64_t)sm_count() * 8u) blocks = (uint64_t)sm_count() * 8u;
   if (blocks < 1) blocks = 1;
   medoid_argmin_kernel<T, METRIC, G, CPL><<<(unsigned)blocks, 128, 0, s>>>(g.store, ids, n, lay.row_bytes, lay.nchunk, mean_row, st);
   medoid_end_kernel<<<1, 1, 0, s>>>(st);

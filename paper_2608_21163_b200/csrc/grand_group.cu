@@ -7,7 +7,8 @@
 namespace grand {
 
 constexpr int kThreads = 256;
-static inline unsigned grid_for(uint64_t n, int threads = kThreads, unsigned maxb = 148u * 32u) {
+static inline unsigned grid_for(uint64_t n, int threads = kThreads) {
+  const uint64_t maxb = (uint64_t)sm_count() * 32u;
   uint64_t b = (n + threads - 1) / threads;
   if (b < 1) b = 1;
   return (unsigned)(b > maxb ? maxb : b);
@@ -158,8 +159,10 @@ cudaError_t launch_exclusive_scan(const uint32_t* in, uint32_t* out, uint64_t n,
 // four rows in flight per warp: degree -> row -> bitmap word is a chain of dependent loads, and one row at a time
 // left the kernels waiting on it at a fifth of the memory bandwidth.
 constexpr int kTransposeRows = 4;
+// A neighbour id at or beyond the node count is never followed (a caller-supplied graph may hold one); `bad`, when
+// given, records that one was met.
 template <typename F>
-__device__ __forceinline__ void for_each_marked_edge(const GraphView& g, const uint32_t* heads, F&& f) {
+__device__ __forceinline__ void for_each_marked_edge(const GraphView& g, const uint32_t* heads, uint32_t* bad, F&& f) {
   const int lane = threadIdx.x & 31;
   const uint64_t wglobal = (blockIdx.x * (uint64_t)blockDim.x + threadIdx.x) >> 5;
   const uint64_t wtotal = ((uint64_t)gridDim.x * blockDim.x) >> 5;
@@ -176,27 +179,34 @@ __device__ __forceinline__ void for_each_marked_edge(const GraphView& g, const u
       for (int k = 0; k < kTransposeRows; ++k) z[k] = sb + lane < dv[k] ? g.adj[(v0 + k * wtotal) * g.R + sb + lane] : 0xFFFFFFFFu;
       bool hit[kTransposeRows];
 #pragma unroll
-      for (int k = 0; k < kTransposeRows; ++k) hit[k] = z[k] != 0xFFFFFFFFu && (!heads || bit_test(heads, z[k]));
+      for (int k = 0; k < kTransposeRows; ++k) {
+        hit[k] = z[k] < g.cap && (!heads || bit_test(heads, z[k]));
+        if (bad && z[k] != 0xFFFFFFFFu && z[k] >= g.cap) *bad = 1u;
+      }
 #pragma unroll
       for (int k = 0; k < kTransposeRows; ++k)
         if (hit[k]) f(z[k], (uint32_t)(v0 + k * wtotal));
     }
   }
 }
-__global__ void transpose_hist_kernel(const GraphView g, uint32_t* indeg, const uint32_t* heads) {
-  for_each_marked_edge(g, heads, [&](uint32_t z, uint32_t) { atomicAdd(&indeg[z], 1u); });
+__global__ void transpose_hist_kernel(const GraphView g, uint32_t* indeg, const uint32_t* heads, uint32_t* bad) {
+  for_each_marked_edge(g, heads, bad, [&](uint32_t z, uint32_t) { atomicAdd(&indeg[z], 1u); });
 }
-__global__ void transpose_scatter_kernel(const GraphView g, const uint32_t* off, uint32_t* fillc, uint32_t* src, const uint32_t* heads) {
-  for_each_marked_edge(g, heads, [&](uint32_t z, uint32_t v) { src[off[z] + atomicAdd(&fillc[z], 1u)] = v; });
+__global__ void transpose_scatter_kernel(const GraphView g, const uint32_t* off, uint32_t* fillc, uint32_t* src, const uint32_t* heads,
+                                         const uint64_t src_capacity) {
+  for_each_marked_edge(g, heads, nullptr, [&](uint32_t z, uint32_t v) {
+    const uint64_t at = (uint64_t)off[z] + atomicAdd(&fillc[z], 1u);
+    if (at < src_capacity) src[at] = v;
+  });
 }
 // ascending rows: shared-memory sort for short rows, in place in global memory for long ones
-__global__ void __launch_bounds__(128) transpose_sort_rows_kernel(uint64_t cap, const uint32_t* off, uint32_t* src) {
+__global__ void __launch_bounds__(128) transpose_sort_rows_kernel(uint64_t cap, const uint32_t* off, uint32_t* src, const uint64_t src_capacity) {
   constexpr uint32_t kRowCap = 4096;
   __shared__ uint32_t sh[kRowCap];
   auto sync = [] { __syncthreads(); };
   for (uint64_t z = blockIdx.x; z < cap; z += gridDim.x) {
     const uint32_t b = off[z], n = off[z + 1] - b;
-    if (n < 2) continue;
+    if (n < 2 || (uint64_t)b + n > src_capacity) continue;
     if (n <= kRowCap) {
       for (uint32_t j = threadIdx.x; j < n; j += blockDim.x) sh[j] = src[b + j];
       __syncthreads();
@@ -211,15 +221,16 @@ __global__ void __launch_bounds__(128) transpose_sort_rows_kernel(uint64_t cap, 
 cudaError_t launch_transpose(const TransposeArgs& a, cudaStream_t s) {
   const uint64_t cap = a.g.cap;
   cudaMemsetAsync(a.indeg, 0, (cap + 1) * 4, s);
-  transpose_hist_kernel<<<grid_for(cap * 32), kThreads, 0, s>>>(a.g, a.indeg, a.heads);
+  transpose_hist_kernel<<<grid_for(cap * 32), kThreads, 0, s>>>(a.g, a.indeg, a.heads, a.bad);
   count_launches(1);
   cudaError_t e = launch_exclusive_scan(a.indeg, a.off, cap + 1, a.scan_tmp, s);
   if (e != cudaSuccess) return e;
   if (a.src) {
     cudaMemsetAsync(a.fillc, 0, cap * 4, s);
-    transpose_scatter_kernel<<<grid_for(cap * 32), kThreads, 0, s>>>(a.g, a.off, a.fillc, a.src, a.heads);
+    transpose_scatter_kernel<<<grid_for(cap * 32), kThreads, 0, s>>>(a.g, a.off, a.fillc, a.src, a.heads, a.src_capacity);
     count_launches(a.sort_rows ? 2 : 1);
-    if (a.sort_rows) transpose_sort_rows_kernel<<<(unsigned)(cap < 148u * 16u ? cap : 148u * 16u), 128, 0, s>>>(cap, a.off, a.src);
+    const uint64_t sort_blocks = (uint64_t)sm_count() * 16u;
+    if (a.sort_rows) transpose_sort_rows_kernel<<<(unsigned)(cap < sort_blocks ? cap : sort_blocks), 128, 0, s>>>(cap, a.off, a.src, a.src_capacity);
   }
   return cudaGetLastError();
 }
@@ -451,13 +462,27 @@ __global__ void copy_rows_kernel(const uint32_t* __restrict__ src, uint32_t* __r
 cudaError_t launch_copy_rows(const uint32_t* src, uint32_t* dst, const uint32_t* ids, uint64_t n, uint32_t R, uint64_t cap, cudaStream_t s) {
   if (n == 0) return cudaSuccess;
   uint64_t blocks = (n + 7) / 8;
-  if (blocks > 148u * 32u) blocks = 148u * 32u;
+  if (blocks > (uint64_t)sm_count() * 32u) blocks = (uint64_t)sm_count() * 32u;
   copy_rows_kernel<<<(unsigned)blocks, 256, 0, s>>>(src, dst, ids, n, R, cap);
   count_launches(1);
   return cudaGetLastError();
 }
 cudaError_t launch_pad_adjacency(uint32_t* adj, const uint32_t* deg, uint64_t cap, uint32_t R, cudaStream_t s) {
   pad_adjacency_kernel<<<grid_for(cap * R), kThreads, 0, s>>>(adj, deg, cap, R);
+  count_launches(1);
+  return cudaGetLastError();
+}
+
+__global__ void check_graph_kernel(const uint32_t* adj, const uint32_t* deg, uint64_t cap, uint32_t R, DevState* st) {
+  const uint64_t total = cap * R;
+  for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < total; i += (uint64_t)gridDim.x * blockDim.x) {
+    const uint64_t v = i / R;
+    const uint32_t s = (uint32_t)(i - v * R), d = deg[v];
+    if ((s == 0 && d > R) || (s < d && adj[i] >= cap)) atomicMin(&st->status, -1);
+  }
+}
+cudaError_t launch_check_graph(const uint32_t* adj, const uint32_t* deg, uint64_t cap, uint32_t R, DevState* st, cudaStream_t s) {
+  check_graph_kernel<<<grid_for(cap * R), kThreads, 0, s>>>(adj, deg, cap, R, st);
   count_launches(1);
   return cudaGetLastError();
 }

@@ -7,9 +7,22 @@
 
 namespace grand {
 
-// Number of kernels launched by this library in this process (every launcher adds its own).
+// Kernel launches are counted per index: the API entry point names the counter of its handle for the
+// calling thread (LaunchScope), every launcher adds to it.
 void count_launches(unsigned n);
-unsigned long long launches_so_far();
+struct LaunchScope {
+  unsigned long long* prev;
+  explicit LaunchScope(unsigned long long* counter);
+  ~LaunchScope();
+};
+
+// Facts about the current device, looked up once per device (a process may drive several GPUs).
+int sm_count();
+// Lets `kernel` use the device's full opt-in dynamic shared memory; done once per (kernel, device).  `done` is a
+// zero-initialised per-kernel table owned by the launcher (one slot per device index).
+constexpr int kMaxDevices = 64;
+struct SmemOptIn { int done[kMaxDevices]; };
+cudaError_t allow_full_dynamic_smem(const void* kernel, SmemOptIn* done);
 
 // Row layout shared by every distance kernel: a padded row has nchunk 16-byte chunks; a team of G
 // lanes covers it with CPL chunks per lane.  layout_code selects the (G, CPL) instantiation.
@@ -33,9 +46,13 @@ struct DevState {
   unsigned long long nlive;
   unsigned long long total_in;   // sum of in-degrees of the delete batch
   unsigned long long medoid_key; // argmin scratch
-  unsigned long long counters[8];  // expansions, dist_evals, pair_dists, dirty, prunes, requests
+  unsigned long long counters[16];
 };
-enum { CTR_EXP = 0, CTR_DIST = 1, CTR_PAIR = 2, CTR_DIRTY = 3, CTR_PRUNE = 4, CTR_REQ = 5 };
+// expansions, query-to-node distances, node-to-node distances, rebuilt rows, prunes, grouped requests; then the
+// bytes the method itself has to move in the rebuild, repair-pick and forward-prune kernels (what each kernel
+// counts is stated where it counts), and the rebuilt rows that went through a prune
+enum { CTR_EXP = 0, CTR_DIST = 1, CTR_PAIR = 2, CTR_DIRTY = 3, CTR_PRUNE = 4, CTR_REQ = 5, CTR_RB_BYTES = 6, CTR_PK_BYTES = 7,
+       CTR_FP_BYTES = 8, CTR_RB_PRUNED = 9 };
 
 struct GraphView {
   const uint8_t* store;
@@ -156,6 +173,8 @@ struct TransposeArgs {
   uint32_t* scan_tmp;  // >= ceil((cap+1)/4096)+1
   bool sort_rows;
   const uint32_t* heads;  // optional bitmap: build only the rows of these nodes
+  uint64_t src_capacity;  // entries `src` can hold; edges beyond it are dropped (the caller compares the total)
+  uint32_t* bad;          // optional: set to 1 when a row names a neighbour id >= cap (such an edge is skipped)
 };
 cudaError_t launch_transpose(const TransposeArgs& a, cudaStream_t s);
 cudaError_t launch_exclusive_scan(const uint32_t* in, uint32_t* out, uint64_t n, uint32_t* tmp, cudaStream_t s);
@@ -183,6 +202,8 @@ struct DeleteArgs {
 cudaError_t launch_delete_prepare(const DeleteArgs& a, cudaStream_t s);   // in-degree prefix, total_in
 cudaError_t launch_delete_ci(const DeleteArgs& a, cudaStream_t s);        // repair candidates C_i
 cudaError_t launch_delete_visited_in(const DeleteArgs& a, uint32_t* inlist, cudaStream_t s);  // Alg. 6 as printed: z in V_i with p_i in N_out(z)
+// repair picks: the set-up kernels (dirty marks of the in-neighbours, work-unit prefix), then the pick kernel alone
+cudaError_t launch_delete_picks_prepare(const DeleteArgs& a, uint64_t total_in, cudaStream_t s);
 cudaError_t launch_delete_picks(const DeleteArgs& a, uint64_t total_in, cudaStream_t s);
 
 struct FixedDeleteArgs {
@@ -217,6 +238,8 @@ cudaError_t launch_augment_rows(const Layout& lay, uint8_t* store, const uint32_
 cudaError_t launch_copy_rows(const uint32_t* src, uint32_t* dst, const uint32_t* ids, uint64_t n, uint32_t R, uint64_t cap, cudaStream_t s);
 cudaError_t launch_pad_adjacency(uint32_t* adj, const uint32_t* deg, uint64_t cap, uint32_t R, cudaStream_t s);
 cudaError_t launch_fill_u32(uint32_t* p, uint32_t v, uint64_t n, cudaStream_t s);
+// status -1 when a degree exceeds R or a listed neighbour id is >= cap (caller-supplied graphs)
+cudaError_t launch_check_graph(const uint32_t* adj, const uint32_t* deg, uint64_t cap, uint32_t R, DevState* st, cudaStream_t s);
 
 }  // namespace grand
 

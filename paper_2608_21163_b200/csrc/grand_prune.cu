@@ -22,7 +22,7 @@ constexpr uint32_t kMaxR = 128;
 template <typename T, int G, int CPL>
 __device__ uint32_t block_prune(const uint8_t* __restrict__ store, uint32_t row_bytes, uint32_t nchunk, const AlphaParam ap,
                                 const unsigned long long* cand, uint32_t n, uint32_t R, uint32_t* out_idx,
-                                unsigned long long& npair) {
+                                unsigned long long& npair, unsigned long long& nrows) {
   using Dist = typename Elem<T>::Dist;
   const uint32_t tid = threadIdx.x, nthreads = blockDim.x;
   const int lane = tid & 31, warp = tid >> 5;
@@ -33,6 +33,7 @@ __device__ uint32_t block_prune(const uint8_t* __restrict__ store, uint32_t row_
     const unsigned long long kc = cand[c];
     const Dist Dc = key_dist<Dist>(kc);
     bool pruned = false;
+    if (tid == 0) ++nrows;  // every candidate the prune looks at has its row fetched once
     if (cnt) {
       uint4 rc[CPL];
       load_row<G, CPL>(store + (size_t)key_id(kc) * row_bytes, nchunk, t, rc);
@@ -72,7 +73,7 @@ __global__ void __launch_bounds__(kPruneThreads) forward_prune_kernel(const Prun
   const uint32_t tid = threadIdx.x, nthreads = blockDim.x;
   const uint32_t R = a.g.R;
   const AlphaParam ap{a.A_fix, a.alpha};
-  unsigned long long npair = 0;
+  unsigned long long npair = 0, nrows = 0;
   uint32_t nprune = 0;
   auto sync = [] { __syncthreads(); };
   for (uint64_t i = blockIdx.x; i < a.n; i += gridDim.x) {
@@ -92,7 +93,7 @@ __global__ void __launch_bounds__(kPruneThreads) forward_prune_kernel(const Prun
       for (uint32_t j = tid; j < cnt; j += nthreads) out_idx[j] = j;
       __syncthreads();
     } else {
-      cnt = block_prune<T, G, CPL>(a.g.store, a.lay.row_bytes, a.lay.nchunk, ap, cand, n, R, out_idx, npair);
+      cnt = block_prune<T, G, CPL>(a.g.store, a.lay.row_bytes, a.lay.nchunk, ap, cand, n, R, out_idx, npair, nrows);
       ++nprune;
     }
     for (uint32_t s = tid; s < R; s += nthreads) {
@@ -120,6 +121,7 @@ __global__ void __launch_bounds__(kPruneThreads) forward_prune_kernel(const Prun
   }
   if (npair) atomicAdd(&a.state->counters[CTR_PAIR], npair);
   if (tid == 0 && nprune) atomicAdd(&a.state->counters[CTR_PRUNE], (unsigned long long)nprune);
+  if (tid == 0 && nrows) atomicAdd(&a.state->counters[CTR_FP_BYTES], nrows * a.lay.row_bytes);
 }
 
 // The same candidate-ordered prune with one WARP per node, for short rows: a row of a few chunks keeps only a
@@ -141,7 +143,7 @@ __global__ void __launch_bounds__(kWarpPruneWarps * 32) forward_prune_warp_kerne
   const uint32_t R = a.g.R, row_bytes = a.lay.row_bytes, nchunk = a.lay.nchunk;
   const uint8_t* __restrict__ store = a.g.store;
   const AlphaParam ap{a.A_fix, a.alpha};
-  unsigned long long npair = 0;
+  unsigned long long npair = 0, nrows = 0;
   uint32_t nprune = 0;
   auto wsync = [] { __syncwarp(); };
   // (handing the nodes out through a counter was measured and is slower than this fixed assignment)
@@ -162,6 +164,7 @@ __global__ void __launch_bounds__(kWarpPruneWarps * 32) forward_prune_warp_kerne
       const unsigned long long kc = cand[c];
       const Dist Dc = key_dist<Dist>(kc);
       bool pruned = false;
+      ++nrows;  // every candidate the prune looks at has its row fetched once
       if (cnt) {
         uint4 rc[CPL];
         load_row<G, CPL>(store + (size_t)key_id(kc) * row_bytes, nchunk, t, rc);
@@ -213,6 +216,7 @@ __global__ void __launch_bounds__(kWarpPruneWarps * 32) forward_prune_warp_kerne
   }
   if (npair) atomicAdd(&a.state->counters[CTR_PAIR], npair);
   if (lane == 0 && nprune) atomicAdd(&a.state->counters[CTR_PRUNE], (unsigned long long)nprune);
+  if (lane == 0 && nrows) atomicAdd(&a.state->counters[CTR_FP_BYTES], nrows * row_bytes);
 }
 
 // The candidate-ordered prune on tensor cores, for integer rows of at most 128 bytes and R <= 64: one warp per
@@ -247,7 +251,7 @@ __global__ void __launch_bounds__(kMmaPruneWarps * 32) forward_prune_mma_kernel(
   int* bN = bU + 16;                                           // |c|^2 per block candidate
   uint32_t* out_idx = reinterpret_cast<uint32_t*>(bN + 16);
   const uint8_t* __restrict__ store = a.g.store;
-  unsigned long long npair = 0;
+  unsigned long long npair = 0, nrows = 0;
   uint32_t nprune = 0;
   auto wsync = [] { __syncwarp(); };
   const uint64_t wglobal = (uint64_t)blockIdx.x * kMmaPruneWarps + warp, wtotal = (uint64_t)gridDim.x * kMmaPruneWarps;
@@ -371,7 +375,10 @@ __global__ void __launch_bounds__(kMmaPruneWarps * 32) forward_prune_mma_kernel(
           --room;
         }
       }
-      if (lane == 0) npair += (unsigned long long)nb * cnt + (unsigned long long)nb * (nb - 1) / 2;
+      if (lane == 0) {
+        npair += (unsigned long long)nb * cnt + (unsigned long long)nb * (nb - 1) / 2;
+        nrows += nb;  // the block's candidate rows, fetched once
+      }
       // ---- the selected candidates join the members: index, norm, row
       const uint32_t nsel = __popc(sel);
       if (lane < 16 && ((sel >> lane) & 1u)) {
@@ -416,6 +423,7 @@ __global__ void __launch_bounds__(kMmaPruneWarps * 32) forward_prune_mma_kernel(
   }
   if (npair) atomicAdd(&a.state->counters[CTR_PAIR], npair);
   if (lane == 0 && nprune) atomicAdd(&a.state->counters[CTR_PRUNE], (unsigned long long)nprune);
+  if (lane == 0 && nrows) atomicAdd(&a.state->counters[CTR_FP_BYTES], nrows * row_bytes);
 }
 
 template <typename T, int METRIC, int G, int CPL>
@@ -426,15 +434,11 @@ static cudaError_t launch_forward_prune_t(const PruneArgs& a, cudaStream_t s) {
       const size_t per_warp = (forward_prune_mma_smem_per_warp(a.lay.row_bytes) + 15) / 16 * 16;
       const size_t smem = per_warp * kMmaPruneWarps;
       auto kern = forward_prune_mma_kernel<T>;
-      static bool smem_set = false;  // (one kernel serves every row layout of this element type)
-      if (!smem_set) {
-        const size_t most = (forward_prune_mma_smem_per_warp(128u) + 15) / 16 * 16 * kMmaPruneWarps;
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)most);
-        if (e != cudaSuccess) return e;
-        smem_set = true;
-      }
-      const uint64_t want = (a.n + kMmaPruneWarps - 1) / kMmaPruneWarps;
-      const unsigned blocks = (unsigned)(want < 148u * 8u ? want : 148u * 8u);
+      static SmemOptIn optin{};
+      cudaError_t e = allow_full_dynamic_smem((const void*)kern, &optin);
+      if (e != cudaSuccess) return e;
+      const uint64_t want = (a.n + kMmaPruneWarps - 1) / kMmaPruneWarps, most = (uint64_t)sm_count() * 8u;
+      const unsigned blocks = (unsigned)(want < most ? want : most);
       kern<<<blocks, kMmaPruneWarps * 32, smem, s>>>(a, (uint32_t)per_warp);
       count_launches(1);
       return cudaGetLastError();
@@ -442,14 +446,15 @@ static cudaError_t launch_forward_prune_t(const PruneArgs& a, cudaStream_t s) {
   }
   if constexpr (G * CPL <= 16) {
     if (!a.fixed_mode && a.cand_stride <= kWarpPruneCand) {
-      const uint64_t want = (a.n + kWarpPruneWarps - 1) / kWarpPruneWarps;
-      const unsigned blocks = (unsigned)(want < 148u * 16u ? want : 148u * 16u);
+      const uint64_t want = (a.n + kWarpPruneWarps - 1) / kWarpPruneWarps, most = (uint64_t)sm_count() * 16u;
+      const unsigned blocks = (unsigned)(want < most ? want : most);
       forward_prune_warp_kernel<T, G, CPL><<<blocks, kWarpPruneWarps * 32, 0, s>>>(a);
       count_launches(1);
       return cudaGetLastError();
     }
   }
-  const unsigned blocks = (unsigned)(a.n < 148u * 16u ? a.n : 148u * 16u);
+  const uint64_t most = (uint64_t)sm_count() * 16u;
+  const unsigned blocks = (unsigned)(a.n < most ? a.n : most);
   forward_prune_kernel<T, METRIC, G, CPL><<<blocks, kPruneThreads, 0, s>>>(a);
   count_launches(1);
   return cudaGetLastError();

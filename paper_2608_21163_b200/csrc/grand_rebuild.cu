@@ -4,15 +4,20 @@
 // computed for the kept neighbours (requests already carry dist(u, id)) and GrANDRobustPrune
 // (Alg. 4) runs on C.  The prune is restructured for the GPU without changing its result:
 //
-//  * p* is always the first valid candidate in key order, so only the outcomes of the tests
-//    alpha * dist(c_i, c_j) <= D_u[c_j] for i < j can ever matter.  They are independent of each
-//    other, so the warp evaluates them in parallel into a bit matrix in shared memory and then
-//    replays the sequential selection on bit masks.
+//  * Rows carry the cached distances dist(u, v) of their entries (rowd), so D_u of a kept neighbour
+//    costs no gather.
 //  * Every row remembers how long its leading run of prune output is (rowpfx).  Two members of
 //    that run both survived an earlier prune of this very node, which means the earlier one does
 //    not prune the later one; distances and D_u are recomputed to the same bits, so those tests
-//    are known to be false and only pairs with an "uncertain" member (appended since, or fresh)
-//    are evaluated.
+//    are known to be false and the sequential prune can only change at an "uncertain" member
+//    (appended since the last prune, or fresh).
+//  * The uncertain members are walked in key order: does a valid member of the run in front of it
+//    prune it (the first hit ends it)?  If not it is selected and prunes among the valid candidates
+//    behind it; the walk stops once R valid candidates stand in front.  Only tests the sequential
+//    algorithm needs are evaluated.  A full, entirely pruned row that receives one candidate takes a
+//    two-phase shortcut of the same walk.  Candidate lists with more than 2P uncertain members
+//    (possible only for R > P, or rows without a trusted run) fall back to evaluating every test
+//    alpha * dist(c_i, c_j) <= D_u[c_j], i < j, into a bit matrix and replaying the selection on masks.
 //
 // Dirty nodes are handed out through an atomic work counter because a node that prunes costs far
 // more than one that only appends.
@@ -56,7 +61,7 @@ __global__ void __launch_bounds__(kRebuildWarps * 32) rebuild_kernel(const Rebui
   const uint32_t row_bytes = a.lay.row_bytes, nchunk = a.lay.nchunk;
   const uint8_t* __restrict__ store = a.g.store;
   auto wsync = [] { __syncwarp(); };
-  unsigned long long npair = 0;
+  unsigned long long npair = 0, nbytes = 0;  // nbytes: what the method has to move for the rows this warp rebuilds
   uint32_t nprune = 0, ndone = 0;
   const uint32_t ndirty = a.state->ndirty;
 
@@ -188,6 +193,8 @@ __global__ void __launch_bounds__(kRebuildWarps * 32) rebuild_kernel(const Rebui
     }
     __syncwarp();
     const uint32_t nC = nk + nf;
+    // the row read and written back, the node's request tuples, and (below) the candidates' vectors when a prune runs
+    nbytes += 2ull * R * 4u + (unsigned long long)cntu * 12u;
     if (nC <= R) {
       for (uint32_t s = lane; s < R; s += 32) {
         row[s] = s < nk ? keep[s] : (s < nC ? key_id(cand[s]) : kInvalid);
@@ -198,6 +205,7 @@ __global__ void __launch_bounds__(kRebuildWarps * 32) rebuild_kernel(const Rebui
         a.g.rowpfx[u] = (uint8_t)kp;  // the surviving part of the pruned run still leads the row
       }
     } else {
+      nbytes += (unsigned long long)nC * row_bytes;
       // ---- D_u for the kept neighbours (those appended after the last prune are tagged uncertain)
       bool all_cached = true;
       for (uint32_t jb = 0; jb < nk; jb += 32) {
@@ -518,8 +526,12 @@ __global__ void __launch_bounds__(kRebuildWarps * 32) rebuild_kernel(const Rebui
   }
   if (npair) atomicAdd(&a.state->counters[CTR_PAIR], npair);
   if (lane == 0) {
-    if (nprune) atomicAdd(&a.state->counters[CTR_PRUNE], (unsigned long long)nprune);
+    if (nprune) {
+      atomicAdd(&a.state->counters[CTR_PRUNE], (unsigned long long)nprune);
+      atomicAdd(&a.state->counters[CTR_RB_PRUNED], (unsigned long long)nprune);
+    }
     if (ndone) atomicAdd(&a.state->counters[CTR_DIRTY], (unsigned long long)ndone);
+    if (nbytes) atomicAdd(&a.state->counters[CTR_RB_BYTES], nbytes);
   }
 }
 
@@ -528,22 +540,13 @@ static cudaError_t launch_rebuild_t(const RebuildArgs& a, cudaStream_t s) {
   const size_t per_warp = rebuild_smem_per_warp(a.g.R, a.P);
   const size_t smem = per_warp * kRebuildWarps;
   auto kern = rebuild_kernel<T, METRIC, G, CPL>;
-  static size_t smem_set = 0;
-  static int sm_count = 0;
-  if (smem > smem_set) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    smem_set = smem;
-  }
-  if (!sm_count) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
-  }
+  static SmemOptIn optin{};
+  cudaError_t e = allow_full_dynamic_smem((const void*)kern, &optin);
+  if (e != cudaSuccess) return e;
   int occ = 1;
   cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, kRebuildWarps * 32, smem);
   if (occ < 1) occ = 1;
-  uint32_t blocks = (uint32_t)sm_count * occ;
+  uint32_t blocks = (uint32_t)sm_count() * occ;
   if (blocks > a.max_blocks && a.max_blocks) blocks = a.max_blocks;
   kern<<<blocks, kRebuildWarps * 32, smem, s>>>(a, (uint32_t)per_warp);
   count_launches(1);

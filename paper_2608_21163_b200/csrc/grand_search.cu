@@ -381,23 +381,14 @@ static cudaError_t launch_beam_search_t(const SearchArgs& a, cudaStream_t s) {
   const size_t per_warp = beam_search_smem_per_warp(a.L, a.g.R, a.hash_bits);
   const size_t smem = per_warp * kSearchWarps;
   auto kern = beam_search_kernel<T, METRIC, G, CPL>;
-  static size_t smem_set = 0;
-  static int sm_count = 0;
-  if (smem > smem_set) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    smem_set = smem;
-  }
-  if (!sm_count) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
-  }
+  static SmemOptIn optin{};
+  cudaError_t e = allow_full_dynamic_smem((const void*)kern, &optin);
+  if (e != cudaSuccess) return e;
   int occ = 1;
   cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, kSearchWarps * 32, smem);
   if (occ < 1) occ = 1;
   uint64_t blocks = (a.nq + kSearchWarps - 1) / kSearchWarps;
-  const uint64_t cap = (uint64_t)sm_count * occ;
+  const uint64_t cap = (uint64_t)sm_count() * occ;
   if (blocks > cap) blocks = cap;
   if (blocks == 0) return cudaSuccess;
   kern<<<(unsigned)blocks, kSearchWarps * 32, smem, s>>>(a, (uint32_t)per_warp);

@@ -31,7 +31,7 @@ namespace {
 
 constexpr uint64_t kMaxNodes = GRAND_NOALLOC_MAX_NODES;
 constexpr uint64_t kScanWords = kMaxNodes / 2048 + 8;           // block sums of the exclusive scan
-constexpr uint64_t kScratchWords = kMaxNodes + kScanWords;      // fill cursors + scan sums
+constexpr uint64_t kScratchWords = kMaxNodes + kScanWords + 1;  // fill cursors + scan sums + one "bad id" flag
 static_assert(kScratchWords * 4 <= GRAND_NOALLOC_SCRATCH_BYTES, "scratch array smaller than its users need");
 
 static __device__ __align__(256) uint32_t g_noalloc_scratch[GRAND_NOALLOC_SCRATCH_BYTES / 4];
@@ -84,19 +84,29 @@ extern "C" int grand_reverse_graph_noalloc(const uint32_t* adj_dev, const uint32
   t.fillc = scratch;
   t.scan_tmp = scratch + kMaxNodes;
   t.sort_rows = true;
-  uint32_t E = 0;
+  t.src_capacity = src_capacity;
+  // A neighbour id at or beyond n_nodes would index outside off_dev and outside the scratch array: the kernels
+  // skip such an edge and raise this flag (one word of the scratch array, cleared here like the rest), and the call
+  // then reports an invalid argument.
+  t.bad = scratch + kMaxNodes + kScanWords;
+  if (cudaMemsetAsync(t.bad, 0, 4, s) != cudaSuccess) return GRAND_ERR_CUDA;
+  uint32_t E = 0, bad = 0;
   if (src_dev) {
     // offsets first, so that the edge count can be checked against the caller's buffer
     t.src = nullptr;
     if (grand::launch_transpose(t, s) != cudaSuccess) return GRAND_ERR_CUDA;
     if (cudaMemcpyAsync(&E, off_dev + n_nodes, 4, cudaMemcpyDeviceToHost, s) != cudaSuccess) return GRAND_ERR_CUDA;
+    if (cudaMemcpyAsync(&bad, t.bad, 4, cudaMemcpyDeviceToHost, s) != cudaSuccess) return GRAND_ERR_CUDA;
     if (cudaStreamSynchronize(s) != cudaSuccess) return GRAND_ERR_CUDA;
+    if (bad) return GRAND_ERR_INVALID_ARG;
     if (E > src_capacity) return GRAND_ERR_CAPACITY;
     t.src = src_dev;
   }
   if (grand::launch_transpose(t, s) != cudaSuccess) return GRAND_ERR_CUDA;
   if (cudaMemcpyAsync(&E, off_dev + n_nodes, 4, cudaMemcpyDeviceToHost, s) != cudaSuccess) return GRAND_ERR_CUDA;
+  if (cudaMemcpyAsync(&bad, t.bad, 4, cudaMemcpyDeviceToHost, s) != cudaSuccess) return GRAND_ERR_CUDA;
   if (cudaStreamSynchronize(s) != cudaSuccess) return GRAND_ERR_CUDA;
+  if (bad) return GRAND_ERR_INVALID_ARG;
   if (E_out_host) *E_out_host = E;
   return GRAND_OK;
 }

@@ -41,6 +41,10 @@ def test_strerror_and_argument_checks_need_no_gpu():
 
 
 def test_options_struct_layout_matches_header():
-    # 2 x u64, 10 x 32-bit fields, 3 pointers
-    assert ctypes.sizeof(binding.GrandOptions) == 16 + 40 + 24
-    assert ctypes.sizeof(binding.GrandStats) == 8 * 8 + 7 * 8 + 8
+    # 2 x u64, 9 x 32-bit fields (+4 padding), u64, one 32-bit field (+4 padding), 3 pointers
+    assert ctypes.sizeof(binding.GrandOptions) == 16 + 40 + 8 + 8 + 24
+    # 11 counters, 7 phase times, 5 launch counts
+    assert ctypes.sizeof(binding.GrandStats) == 11 * 8 + 7 * 8 + 5 * 8
+    # field order as in the header: the 64-bit edge bound sits between the two 32-bit switches
+    names = [n for n, _ in binding.GrandOptions._fields_]
+    assert names.index("visited_set_delete") < names.index("max_delete_edges") < names.index("snapshot_search")
