@@ -1,21 +1,26 @@
 #!/usr/bin/env python
-"""Benchmark of the batched dynamic-update + search hot path on the SIFT-shaped stream.
+"""Benchmark of the batched dynamic-update + search hot path.
 
-One step = one pass of the whole path over one batch of synthetic input: insert 10,000 vectors,
-delete 10,000 random live ids, search 10,000 queries (k=10) on an index built on 900,000
-128-d uint8 vectors (R=64, L=128, alpha=1.2).  Prints ONE JSON line:
+One step = one pass of the whole path over one batch of synthetic input: insert a batch, delete a batch, search a
+batch of queries (k=10) on a built index.  The headline workload is the Deep-shaped sliding window (10M x 96 fp32,
+window 8M, steps of insert 100k newest + delete 100k oldest + search 10k; R=64, L=128, alpha=1.2): the largest
+configuration by vectors and edges, and the one that runs the complete Vamana path (search, RobustPrune, reverse
+graph, consolidated repair).  The other full-size configurations follow under `per_config` with the same fields.
+Prints ONE JSON line:
 
-  value    update throughput, (inserted + deleted vectors) / time of the insert + delete calls, inputs
-           already resident in HBM, timed with CUDA events; whole job over all ranks
-  e2e      the same metric through the host-buffer C-ABI calls (host->device copy of ids + vectors and
-           the device->host status/result read-back inside the timed region)
-  roofline the beam-search kernel: gathered adjacency + vector bytes (in-kernel counters) per second
-           against the measured HBM copy bandwidth
-  cpu_baseline  the CPU oracle, as it stands, on a bounded shrink of the same stream
+  value     update throughput, (inserted + deleted vectors) / time of the insert + delete calls, inputs already
+            resident in HBM, CUDA-event timed, the library's phase events OFF; whole job over all ranks
+  e2e       the same metric through the host-buffer C-ABI calls (host->device copy of ids + vectors and the
+            device->host status/result read-back inside the timed region)
+  roofline  the dominant kernel (beam search): gathered adjacency + vector bytes (in-kernel counters) per second of
+            kernel time against the measured HBM copy bandwidth; `rooflines` has one entry per kernel of the path
+            (kernel times come from separate steps with the phase events ON, counters from those same steps)
+  cpu_baseline  the CPU oracle, as it stands, on a bounded shrink of the same stream, plus the tiny config at full
+            size; `sampled_parity` runs the oracle's search on the graph the GPU built, at full size
 
-`--impl reference` times the oracle alone (it is the reference arm of this build).  With --gpus N
-(launched by torchrun) every rank runs an independent replica of the stream: the path has no
-exchange step, so there is no data-path collective.
+`--impl reference` times the oracle alone (it is the reference arm of this build).  With --gpus N (launched by
+torchrun) every rank runs an independent replica of the stream: the path has no exchange step, so there is no
+data-path collective.
 """
 import argparse
 import json
@@ -35,10 +40,14 @@ from paper_2608_21163_b200 import synth  # noqa: E402
 
 METRIC = "update_vectors_per_sec"
 UNIT = "vectors/s"
-WORKLOAD = "sift_u8_d128"
-# DRAM bytes moved per beam-search launch divided by the algorithmic bytes of that launch, from the
-# single-pass ncu capture at full size summarised in profiles/ (L2 absorbs the rest of the gathers).
-NCU_TRAFFIC_RATIO = 0.375
+WORKLOAD = "deep_f32_d96"
+PER_CONFIG = ["sift_u8_d128", "gist_f32_d960", "embed_f32_d768_ip"]
+SWEEP_L = (10, 16, 24, 32, 48, 64, 96, 128, 192, 256, 384, 512)
+# DRAM bytes of one beam-search launch divided by the launch's algorithmic bytes, from one-pass ncu captures
+# (dram__bytes_read.sum + dram__bytes_write.sum); each ratio is valid for its workload at the named scale only.
+NCU_TRAFFIC = {
+    ("sift_u8_d128", 1.0): (0.375, "profiles/beam_search_dram_sift_u8_d128_full.txt"),
+}
 
 
 def read_peaks():
@@ -103,17 +112,23 @@ def max_over_ranks(values, dist, device):
 
 
 # ------------------------------------------------------------------ oracle arm
-def oracle_run(steps, warmup, seed=0, workload=WORKLOAD):
+ORACLE_BUILD = 20_000
+ORACLE_BATCH = 500
+
+
+def oracle_run(steps, warmup, seed=0, workload=WORKLOAD, nthreads=0):
     """The CPU oracle on a bounded shrink of the stream: build 20,000 points (untimed), then steps of
     insert 500 + delete 500 + search 500.  Returns the JSON-ready dict of the reference arm."""
     from oracle import grand_oracle as go
-    cfg = dict(synth.CONFIGS[workload])
-    per = 500
-    cfg.update(n=20_000 + (steps + warmup) * per, build=20_000, first_batch=1_000, max_build_batch=2_000,
-               ins=per, dele=per, nq=per, rounds=steps + warmup)
+    full = synth.CONFIGS[workload]
+    cfg = dict(full)
+    per = ORACLE_BATCH
+    cfg.update(n=ORACLE_BUILD + (steps + warmup) * per, build=ORACLE_BUILD, first_batch=1_000, max_build_batch=2_000,
+               ins=per, dele=per, nq=per, rounds=steps + warmup, reuse_ids=False)
     wl = synth.Workload(cfg, seed)
     st = synth.StreamState(wl)
-    o = go.Oracle(cfg["dim"], cfg["dtype"], cfg["metric"], cfg["R"], cfg["L"], cfg["alpha"], wl.capacity(), mode=cfg["mode"])
+    o = go.Oracle(cfg["dim"], cfg["dtype"], cfg["metric"], cfg["R"], cfg["L"], cfg["alpha"], wl.capacity(), mode=cfg["mode"],
+                  nthreads=nthreads)
     t0 = time.perf_counter()
     for ids, rows in st.build_batches():
         o.insert_batch(ids, wl.vectors(*rows))
@@ -123,7 +138,6 @@ def oracle_run(steps, warmup, seed=0, workload=WORKLOAD):
     for r in range(steps + warmup):
         ids, rows = st.insert_ids()
         v = wl.vectors(*rows)
-        dele = None
         t0 = time.perf_counter()
         o.insert_batch(ids, v)
         t1 = time.perf_counter()
@@ -138,77 +152,106 @@ def oracle_run(steps, warmup, seed=0, workload=WORKLOAD):
             t_upd += (t1 - t0) + (t3 - t2)
             t_search += t4 - t3
     value = 2 * per * steps / t_upd
-    sample = (f"{workload} shrunk: index built on 20,000 points (untimed, {t_build:.1f} s), then {steps} steps of "
-              f"insert {per} + delete {per} + search {per} (k=10, L={cfg['L']})")
+    sample = (f"{workload} shrunk: index built on {ORACLE_BUILD:,} points (untimed, {t_build:.1f} s) instead of {full['build']:,}, "
+              f"then {steps} steps of insert {per} + delete {per} + search {per} (k=10, L={cfg['L']})")
     return {"value": value, "unit": UNIT, "cores": o.nthreads, "kind": "oracle", "sample": sample,
-            "search_qps": per * steps / t_search, "ms_per_step": 1e3 * (t_upd + t_search) / steps}
+            "index_size_ratio": full["build"] / ORACLE_BUILD, "search_qps": per * steps / t_search,
+            "ms_per_step": 1e3 * (t_upd + t_search) / steps}
 
 
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=7)
-    ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--impl", default="grand", choices=["grand", "reference"])
-    ap.add_argument("--scale", type=float, default=1.0, help="shrink the workload (profiling captures, quick checks)")
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-sweep", action="store_true")
-    ap.add_argument("--workload", default=WORKLOAD, choices=sorted(synth.CONFIGS), help="default: the bench workload; the other "
-                    "configs are exploration runs (their lines carry their own workload name)")
-    ap.add_argument("--pattern", default="", choices=["", "sliding_window", "interleaved", "expiration_time", "clustered", "insert_heavy"],
-                    help="run one of the paper's streaming patterns (Sec. 5.2) on the SIFT-shaped data instead of the step loop")
-    ap.add_argument("--hash-bits", type=int, default=0, help="log2 size of the per-query visited cache (0 = library default)")
-    ap.add_argument("--visited-set-delete", action="store_true",
-                    help="run the delete variant that takes in-neighbours from the visited sets (dangling edges allowed)")
-    ap.add_argument("--snapshot-search", action="store_true",
-                    help="keep the adjacency twice so that searches may overlap update batches; adds an 'overlap' measurement")
-    ap.add_argument("--search-only", type=int, default=0, help="after the build run this many search launches and exit")
-    args = ap.parse_args()
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    K, W = args.steps, max(args.warmup, 0)
+def oracle_tiny_full(nthreads):
+    """The tiny config (10,000 x 32 uint8) at full size through the oracle: 8 x 1,000 build, +2,000, -1,000, 1,000 queries."""
+    from oracle import grand_oracle as go
+    cfg = synth.CONFIGS["tiny_u8_d32"]
+    wl = synth.Workload(cfg, 0)
+    st = synth.StreamState(wl)
+    o = go.Oracle(cfg["dim"], cfg["dtype"], cfg["metric"], cfg["R"], cfg["L"], cfg["alpha"], wl.capacity(), nthreads=nthreads)
+    t0 = time.perf_counter()
+    for ids, rows in st.build_batches():
+        o.insert_batch(ids, wl.vectors(*rows))
+    t1 = time.perf_counter()
+    ids, rows = st.insert_ids()
+    v = wl.vectors(*rows)
+    t2 = time.perf_counter()
+    o.insert_batch(ids, v)
+    t3 = time.perf_counter()
+    dele = st.delete_ids()
+    t4 = time.perf_counter()
+    o.delete_batch(dele)
+    t5 = time.perf_counter()
+    q = wl.queries()
+    t6 = time.perf_counter()
+    o.search(q, 10, cfg["L"])
+    t7 = time.perf_counter()
+    return {"threads": o.nthreads, "build_vectors_per_sec": cfg["build"] / (t1 - t0),
+            "update_vectors_per_sec": (len(ids) + len(dele)) / ((t3 - t2) + (t5 - t4)), "search_qps": len(q) / (t7 - t6)}
 
-    if args.impl == "reference":
-        if rank != 0:
-            return 0
-        r = oracle_run(K, W, workload=args.workload)
-        line = {"impl": "reference", "metric": METRIC, "value": r["value"], "unit": UNIT, "n_gpus": args.gpus, "steps": K,
-                "warmup": W, "ms_per_step": r["ms_per_step"], "higher_is_better": True, "scaling": "weak",
-                "vs_baseline": None, "dtype": "int32", "data": "synthetic",
-                "config": {"workload": args.workload, "sample": r["sample"]},
-                "cpu_baseline": {k: r[k] for k in ("value", "unit", "cores", "kind", "sample")},
-                "e2e": {"value": r["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
-                "search_qps": r["search_qps"], "gpu_launches": 0}
-        print(json.dumps(line))
-        return 0
 
-    import torch
-    from paper_2608_21163_b200 import binding as gb
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
-    torch.backends.cuda.matmul.allow_tf32 = False
+def sampled_parity(torch, g, cfg, base_host, queries_host, is_f32, nsample=200):
+    """The oracle's own search (with a complete visited set) on the graph the GPU built, at the bench's full size, for
+    a sample of the queries: its answers against the GPU's for the same queries, and the distances it evaluates per
+    search (every node once) against the GPU's count (its bounded visited cache may forget and evaluate twice)."""
+    from oracle import grand_oracle as go
+    t0 = time.perf_counter()
+    adj, deg, live, entry = g.export_graph()
+    cap = g.capacity
+    o = go.Oracle(cfg["dim"], cfg["dtype"], cfg["metric"], cfg["R"], cfg["L"], cfg["alpha"], cap, mode=cfg["mode"])
+    o.import_graph(adj.cpu().numpy(), deg.cpu().numpy(), live.cpu().numpy(), entry, base_host[:cap])
+    del adj, deg, live
+    q = queries_host[:nsample]
+    s0 = g.stats()
+    gi, gd = g.search(torch.from_numpy(q), 10, cfg["L"])
+    torch.cuda.synchronize()
+    s1 = g.stats()
+    gi, gd = gi.cpu().numpy(), gd.cpu().numpy()
+    oi, od = o.search(q, 10, cfg["L"], use_seen_set=True)
+    so = o.stats()
+    out = {"queries": len(q), "index_nodes_live": int(g.live_count), "seconds": None,
+           "gpu_evals_per_search": (s1["dist_evals"] - s0["dist_evals"]) / len(q),
+           "unique_evals_per_search": so["dist_evals"] / len(q),
+           "gpu_expansions_per_search": (s1["expansions"] - s0["expansions"]) / len(q),
+           "oracle_expansions_per_search": so["expansions"] / len(q)}
+    out["reevaluated_share"] = 1.0 - out["unique_evals_per_search"] / max(out["gpu_evals_per_search"], 1.0)
+    if is_f32:
+        out["mean_result_overlap"] = float(np.mean([len(set(a.tolist()) & set(b.tolist())) / 10 for a, b in zip(oi, gi)]))
+        rel = 0.0
+        for i in range(len(q)):
+            ok = gi[i] != 0xFFFFFFFF
+            b = base_host[gi[i][ok]].astype(np.float64)
+            qq = q[i].astype(np.float64)
+            if cfg["metric"] == synth.L2:
+                exact = ((b - qq) ** 2).sum(1)
+                scale = np.abs(exact)
+            else:
+                exact = -(b @ qq)
+                scale = np.linalg.norm(b, axis=1) * np.linalg.norm(qq)
+            rel = max(rel, float((np.abs(gd[i][ok] - exact) / np.maximum(scale, 1e-30)).max()))
+        out["max_relative_distance_error"] = rel
+        out["ok"] = bool(rel <= 1e-5 and out["mean_result_overlap"] > 0.95)
+    else:
+        out["ids_identical"] = bool((oi == gi).all())
+        out["distances_identical"] = bool((od == gd.astype(np.float64)).all())
+        out["ok"] = out["ids_identical"] and out["distances_identical"]
+    out["seconds"] = time.perf_counter() - t0
+    return out
 
-    if args.pattern:
-        return run_pattern(args, torch, gb, dev)
-    cfg = dict(synth.CONFIGS[args.workload])
+
+# ------------------------------------------------------------------ one workload on the GPU
+def run_workload(args, torch, gb, dev, dist, rank, world, name, scale, K, W, Kp, headline):
+    local_rank = dev.index
+    cfg = dict(synth.CONFIGS[name])
     is_f32 = cfg["dtype"] == synth.F32
     dist_dtype = torch.float32 if is_f32 else torch.int32
-    if args.scale != 1.0:
-        cfg = synth.scaled(cfg, args.scale)
-    total_steps = W + 2 * K + 1      # device-resident steps, then one untimed and K timed end-to-end steps
+    if scale != 1.0:
+        cfg = synth.scaled(cfg, scale)
+    total_steps = W + K + Kp + K + 1     # warm-up, timed, profiled, then one untimed and K timed end-to-end steps
     if args.snapshot_search:
-        total_steps += K + 1         # and the same steps once more with the searches on a second stream
+        total_steps += K + 1             # and the same steps once more with the searches on a second stream
     cfg["rounds"] = total_steps
     cfg["n"] = cfg["build"] + total_steps * cfg["ins"]
-    cfg["reuse_ids"] = False      # fresh ids every step, whatever the config's own id policy
-    seed = rank                       # replicas draw independent streams
+    cfg["reuse_ids"] = False             # fresh ids every step, whatever the config's own id policy
+    cfg["delete_first"] = False
+    seed = rank                          # replicas draw independent streams
     wl = synth.Workload(cfg, seed)
     st = synth.StreamState(wl)
     cap = wl.capacity()
@@ -243,15 +286,14 @@ def main():
         for _ in range(args.search_only):
             g.search(queries, 10, cfg["L"], out_i, out_d)
         torch.cuda.synchronize()
-        print(json.dumps({"search_only": args.search_only, "build_s": t_build}))
-        return 0
+        return {"search_only": args.search_only, "build_s": t_build}
 
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)   # > L2 (126 MB)
     out_i = torch.empty((cfg["nq"], 10), dtype=torch.uint32, device=dev)
     out_d = torch.empty((cfg["nq"], 10), dtype=dist_dtype, device=dev)
     ev = lambda: torch.cuda.Event(enable_timing=True)
 
-    def one_step(timed):
+    def one_step():
         ids, rows = st.insert_ids()
         d_ins = ids_dev(ids)
         vec = base[rows[0]:rows[0] + rows[1]]
@@ -269,9 +311,9 @@ def main():
         return (e[0].elapsed_time(e[1]), e[1].elapsed_time(e[2]), e[2].elapsed_time(e[3]), len(ids), len(dele))
 
     for _ in range(W):
-        one_step(False)
+        one_step()
     g.reset_stats()
-    g.set_profiling(True)
+    g.set_profiling(False)
     if dist:
         dist.barrier()
     torch.cuda.synchronize()
@@ -282,21 +324,35 @@ def main():
     t_ins = t_del = t_srch = 0.0
     n_upd = 0
     for _ in range(K):
-        a, b, c, ni, nd = one_step(True)
+        a, b, c, ni, nd = one_step()
         t_ins += a; t_del += b; t_srch += c; n_upd += ni + nd
     torch.cuda.synchronize()
     if dist:
         dist.barrier()
     clocks = sampler.stop() if rank == 0 else None
+    stats_timed = g.stats()
+    launches = stats_timed["kernel_launches"] - launches0
+
+    # ---- kernel times: separate steps with the library's phase events on (the events and the synchronising search
+    #      they bring would otherwise sit inside `value`)
+    g.reset_stats()
+    g.set_profiling(True)
+    if args.cuda_profiler_range:
+        torch.cuda.profiler.start()      # `ncu --profile-from-start off` then sees exactly these steps
+    for _ in range(Kp):
+        one_step()
+    torch.cuda.synchronize()
+    if args.cuda_profiler_range:
+        torch.cuda.profiler.stop()
     stats = g.stats()
-    launches = stats["kernel_launches"] - launches0
     g.set_profiling(False)
+    live_edges = int(g.export_graph()[1].view(torch.int32).to(torch.int64).sum().item())
 
     # ---- snapshot mode: the step's search on a second stream, overlapping the step's update batches
     overlap = None
     if args.snapshot_search:
         side = torch.cuda.Stream()
-        main = torch.cuda.current_stream()
+        main_s = torch.cuda.current_stream()
         t_ov = 0.0
         for it in range(K + 1):
             ids, rows = st.insert_ids()
@@ -314,7 +370,7 @@ def main():
                 es.record()
             g.insert_batch(d_ins, vec)
             g.delete_batch(d_del)
-            main.wait_event(es)
+            main_s.wait_event(es)
             e1.record()
             torch.cuda.synchronize()
             if it:
@@ -330,7 +386,7 @@ def main():
     t_e2e_upd = t_e2e_all = 0.0
     n_e2e = 0
     h2d = d2h = 0
-    for it in range(K + 1):          # the first pass sizes the library's staging buffers and is not timed
+    for it in range(K + 1):          # the first pass sizes the search call's staging buffers and is not timed
         ids, rows = st.insert_ids()
         vec_pin = pin(base_host[rows[0]:rows[0] + rows[1]])
         ids_pin = pin(ids)
@@ -351,7 +407,7 @@ def main():
         t_e2e_all += t2 - t0
         n_e2e += len(ids) + len(dele)
         h2d = ids_pin.numel() * 4 + vec_pin.numel() * vec_pin.element_size() + del_pin.numel() * 4 + q_pin.numel() * q_pin.element_size()
-        d2h = oi_pin.numel() * 4 + od_pin.numel() * 4 + 4 * 104   # results + four status blocks
+        d2h = oi_pin.numel() * 4 + od_pin.numel() * 4 + 4 * 176   # results + four status blocks
     torch.cuda.synchronize()
 
     # ---- max over ranks
@@ -360,21 +416,40 @@ def main():
     e2e_value = world * n_e2e / t_e2e_s
     search_qps = world * cfg["nq"] * K / (t_srch_ms * 1e-3)
 
-    # ---- roofline of the dominant kernel (beam search): gathered bytes / launch time
+    # ---- rooflines: algorithmic bytes (counted in the kernels) per second of kernel time (phase events of the
+    #      profiled steps, on the launching stream) against the measured HBM copy bandwidth
     peak, peak_kind = read_peaks()
-    alg_bytes = stats["expansions"] * (cfg["R"] * 4 + 4) + stats["dist_evals"] * row_bytes
-    n_sl = max(stats["n_search_launches"], 1)
-    ach = alg_bytes / (stats["ms_search"] * 1e-3) / 1e9 if stats["ms_search"] > 0 else 0.0
-    roofline = {"bound": "hbm", "kernel": "beam_search_kernel", "achieved": ach, "peak": peak, "unit": "GB/s",
-                "frac": ach / peak, "peak_kind": peak_kind,
-                "traffic": (NCU_TRAFFIC_RATIO * alg_bytes / n_sl) if NCU_TRAFFIC_RATIO else None,
-                "algorithmic_bytes_per_launch": alg_bytes / n_sl, "launches": n_sl,
-                "avg_launch_ms": stats["ms_search"] / n_sl}
+
+    def roof(kernel, nbytes, ms, launches_, what):
+        if not launches_ or ms <= 0:
+            return None
+        ach = nbytes / (ms * 1e-3) / 1e9
+        return {"bound": "hbm", "kernel": kernel, "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
+                "peak_kind": peak_kind, "traffic": None, "algorithmic_bytes_per_launch": nbytes / launches_,
+                "launches": launches_, "avg_launch_ms": ms / launches_, "bytes_counted": what}
+
+    search_bytes = stats["expansions"] * (cfg["R"] * 4 + 4) + stats["dist_evals"] * row_bytes
+    rooflines = {
+        "beam_search": roof("beam_search_kernel", search_bytes, stats["ms_search"], stats["n_search_launches"],
+                            "expansions x (R x 4 + 4) adjacency bytes + evaluated nodes x padded row bytes"),
+        "rebuild": roof("rebuild_kernel", stats["rebuild_bytes"], stats["ms_rebuild"], stats["n_rebuild_launches"],
+                        "per rebuilt row: row read + write (2 x R x 4), request tuples (12 each), and one vector per candidate when a prune runs"),
+        "delete_picks": roof("delete_picks_*_kernel", stats["picks_bytes"], stats["ms_picks"], stats["n_picks_launches"],
+                             "one vector per (deleted node, surviving in-/out-neighbour) pair + the repair candidates' vectors per deleted node"),
+        "forward_prune": roof("forward_prune_*_kernel", stats["prune_bytes"], stats["ms_prune"], stats["n_prune_launches"],
+                              "one vector per candidate the prune looks at"),
+        "reverse_graph": roof("transpose_hist/scatter_kernel", stats["n_transpose_launches"] * 2 * (cap * 4 + live_edges * 4),
+                              stats["ms_transpose"], stats["n_transpose_launches"],
+                              "two passes over the degrees and the live adjacency entries (scan and scatter of the batch's rows not counted)"),
+    }
+    tr = NCU_TRAFFIC.get((name, float(scale)))
+    if tr and rooflines["beam_search"]:
+        rooflines["beam_search"]["traffic"] = tr[0] * rooflines["beam_search"]["algorithmic_bytes_per_launch"]
+        rooflines["beam_search"]["traffic_source"] = f"{tr[0]} x algorithmic bytes, ratio from {tr[1]}"
 
     if rank != 0:
-        if dist:
-            dist.destroy_process_group()
-        return 0
+        g.close()
+        return None
 
     extra = {}
     if not args.no_sweep:
@@ -382,7 +457,7 @@ def main():
         live = np.flatnonzero(st.live)
         truth = brute_topk_gpu(torch, base, torch.from_numpy(live).to(dev), queries, 10, cfg["metric"], is_f32)
         sweep = []
-        for L in (10, 16, 24, 32, 48, 64, 96, 128):
+        for L in SWEEP_L:
             reps = []
             for _ in range(3):
                 flush.zero_(); torch.cuda.synchronize()
@@ -394,35 +469,136 @@ def main():
             rec = recall_gpu(torch, found, truth)
             sweep.append({"L": L, "recall_at_10": rec, "qps": cfg["nq"] / (min(reps) * 1e-3)})
         ok = [s for s in sweep if s["recall_at_10"] >= 0.95]
+        best = max(sweep, key=lambda s: s["recall_at_10"])
         extra["search_sweep"] = sweep
-        extra["search_qps_at_recall95"] = ok[0] if ok else None
-        extra["recall_at_10_config_L"] = sweep[-1]["recall_at_10"]
+        extra["search_qps_at_recall95"] = dict(ok[0], reached=True) if ok else \
+            {"reached": False, "best_recall_at_10": best["recall_at_10"], "L": best["L"], "qps": best["qps"]}
+        extra["recall_at_10_config_L"] = [s for s in sweep if s["L"] == cfg["L"]][0]["recall_at_10"]
+        del truth
 
-    cpu = None
     if not args.no_cpu_baseline:
-        r = oracle_run(steps=30, warmup=1, workload=args.workload)
-        cpu = {k: r[k] for k in ("value", "unit", "cores", "kind", "sample")}
-        cpu["search_qps"] = r["search_qps"]
+        sp = sampled_parity(torch, g, cfg, base_host, queries_host, is_f32)
+        extra["sampled_parity"] = sp
+        bs = rooflines["beam_search"]
+        if bs:
+            bs["achieved_on_unique_rows"] = bs["achieved"] * (1.0 - max(sp["reevaluated_share"], 0.0))
 
     ms_per_step = (t_upd_ms + t_srch_ms) / K
-    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
-            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "f32" if is_f32 else "int32", "data": "synthetic",
-            "config": {"workload": args.workload, "scale": args.scale, "built_on": cfg["build"], "dim": cfg["dim"], "R": cfg["R"],
-                       "L": cfg["L"], "alpha": cfg["alpha"], "step": f"insert {cfg['ins']} + delete {cfg['dele']} + search {cfg['nq']} (k=10)",
-                       "l2": "index (vectors + adjacency) larger than L2, and a 256 MiB flush between steps",
-                       "delete": "visited-set (Alg. 6 as printed)" if args.visited_set_delete else "exact in-neighbours",
-                       "parallelism": f"replicas x{world}"},
-            "overlap": overlap,
-            "search_qps": search_qps,
-            "insert_vectors_per_sec": world * (n_upd / 2) / (t_ins * 1e-3), "delete_vectors_per_sec": world * (n_upd / 2) / (t_del * 1e-3),
-            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                    "ms_per_step": 1e3 * t_e2e_all / K},
-            "gpu_launches": launches, "clocks": clocks, "roofline": roofline, "cpu_baseline": cpu,
-            "phases_ms_per_step": {k[3:]: stats[k] / K for k in stats if k.startswith("ms_")},
-            "counters_per_step": {k: stats[k] / K for k in ("expansions", "dist_evals", "pair_dists", "dirty_nodes", "prunes", "requests")},
-            "build": {"vectors": cfg["build"], "seconds": t_build, "vectors_per_sec": cfg["build"] / t_build, "datagen_s": t_gen}}
-    line.update(extra)
+    res = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+           "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+           "dtype": "f32" if is_f32 else "int32", "data": "synthetic",
+           "config": {"workload": name, "scale": scale, "built_on": cfg["build"], "dim": cfg["dim"], "R": cfg["R"],
+                      "L": cfg["L"], "alpha": cfg["alpha"], "mode": "fixed-degree" if cfg["mode"] else "vamana",
+                      "metric": "ip" if cfg["metric"] else "l2",
+                      "step": f"insert {cfg['ins']} + delete {cfg['dele']} + search {cfg['nq']} (k=10)",
+                      "l2": "index (vectors + adjacency) larger than L2, and a 256 MiB flush between steps",
+                      "delete": "visited-set (Alg. 6 as printed)" if args.visited_set_delete else "exact in-neighbours",
+                      "kernel_times": f"from {Kp} further steps with the library's phase events on; `value` is timed with them off",
+                      "parallelism": f"replicas x{world}"},
+           "overlap": overlap,
+           "search_qps": search_qps,
+           "insert_vectors_per_sec": world * (n_upd / 2) / (t_ins * 1e-3), "delete_vectors_per_sec": world * (n_upd / 2) / (t_del * 1e-3),
+           "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                   "ms_per_step": 1e3 * t_e2e_all / K},
+           "gpu_launches": launches, "clocks": clocks, "roofline": rooflines["beam_search"], "rooflines": rooflines,
+           "phases_ms_per_step": {k[3:]: stats[k] / Kp for k in stats if k.startswith("ms_")},
+           "counters_per_step": {k: stats_timed[k] / K for k in ("expansions", "dist_evals", "pair_dists", "dirty_nodes", "prunes",
+                                                                 "rebuild_prunes", "requests", "rebuild_bytes", "picks_bytes", "prune_bytes")},
+           "build": {"vectors": cfg["build"], "seconds": t_build, "vectors_per_sec": cfg["build"] / t_build, "datagen_s": t_gen}}
+    if not headline:
+        for k in ("n_gpus", "higher_is_better", "scaling", "vs_baseline", "data", "overlap"):
+            res.pop(k)
+    res.update(extra)
+    g.close()
+    del g, base, queries, flush
+    torch.cuda.empty_cache()
+    return res
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=7)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="grand", choices=["grand", "reference"])
+    ap.add_argument("--scale", type=float, default=1.0, help="shrink the workload (profiling captures, quick checks)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sweep", action="store_true")
+    ap.add_argument("--no-per-config", action="store_true", help="run the headline workload only")
+    ap.add_argument("--profiled-steps", type=int, default=3, help="extra steps with the phase events on (kernel times)")
+    ap.add_argument("--workload", default=WORKLOAD, choices=sorted(synth.CONFIGS), help="headline workload of the line")
+    ap.add_argument("--pattern", default="", choices=["", "sliding_window", "interleaved", "expiration_time", "clustered", "insert_heavy"],
+                    help="run one of the paper's streaming patterns (Sec. 5.2) on the SIFT-shaped data instead of the step loop")
+    ap.add_argument("--hash-bits", type=int, default=0, help="log2 size of the per-query visited cache (0 = library default)")
+    ap.add_argument("--visited-set-delete", action="store_true",
+                    help="run the delete variant that takes in-neighbours from the visited sets (dangling edges allowed)")
+    ap.add_argument("--snapshot-search", action="store_true",
+                    help="keep the adjacency twice so that searches may overlap update batches; adds an 'overlap' measurement")
+    ap.add_argument("--search-only", type=int, default=0, help="after the build run this many search launches and exit")
+    ap.add_argument("--cuda-profiler-range", action="store_true",
+                    help="bracket the profiled steps with cudaProfilerStart/Stop (for captures limited to those steps)")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    K, W = max(args.steps, 1), max(args.warmup, 0)
+
+    if args.impl == "reference":
+        if rank != 0:
+            return 0
+        r = oracle_run(K, W, workload=args.workload)
+        is_f32 = synth.CONFIGS[args.workload]["dtype"] == synth.F32
+        line = {"impl": "reference", "metric": METRIC, "value": r["value"], "unit": UNIT, "n_gpus": args.gpus, "steps": K,
+                "warmup": W, "ms_per_step": r["ms_per_step"], "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "f64" if is_f32 else "int64", "data": "synthetic",
+                "config": {"workload": args.workload, "sample": r["sample"], "index_size_ratio": r["index_size_ratio"]},
+                "cpu_baseline": {k: r[k] for k in ("value", "unit", "cores", "kind", "sample", "index_size_ratio")},
+                "e2e": {"value": r["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                "search_qps": r["search_qps"], "gpu_launches": 0}
+        print(json.dumps(line))
+        return 0
+
+    import torch
+    from paper_2608_21163_b200 import binding as gb
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    torch.backends.cuda.matmul.allow_tf32 = False
+
+    if args.pattern:
+        return run_pattern(args, torch, gb, dev)
+
+    line = run_workload(args, torch, gb, dev, dist, rank, world, args.workload, args.scale, K, W, max(args.profiled_steps, 1), True)
+    if args.search_only:
+        print(json.dumps(line))
+        return 0
+    if rank != 0:
+        if dist:
+            dist.destroy_process_group()
+        return 0
+
+    # ---- the other full-size configurations, same fields, a short run each (one GPU, rank 0 of a single-rank job)
+    if world == 1 and not args.no_per_config and args.scale == 1.0:
+        per = {}
+        for name in PER_CONFIG:
+            if name == args.workload:
+                continue
+            per[name] = run_workload(args, torch, gb, dev, None, 0, 1, name, 1.0, 3, 3, 2, False)
+        line["per_config"] = per
+
+    # ---- the oracle on the host cores (rank 0, one-GPU runs only): a bounded shrink of the headline stream, and the
+    #      tiny config at full size with all threads and with one
+    line["cpu_baseline"] = None
+    if world == 1 and not args.no_cpu_baseline:
+        r = oracle_run(steps=6, warmup=1, workload=args.workload)
+        cpu = {k: r[k] for k in ("value", "unit", "cores", "kind", "sample", "index_size_ratio", "search_qps")}
+        cpu["tiny_u8_d32_full_size"] = [oracle_tiny_full(0), oracle_tiny_full(1)]
+        line["cpu_baseline"] = cpu
     print(json.dumps(line))
     if dist:
         dist.destroy_process_group()
@@ -491,20 +667,31 @@ def _contiguous(ids):
 
 
 def brute_topk_gpu(torch, base, live_ids, queries, k, metric=0, is_f32=False):
-    """Ground truth for recall (harness only).  uint8 + squared L2: exact, ties by id.  fp32: fp32 matmul."""
+    """Ground truth for recall (harness only).  uint8 + squared L2: exact, ties by id.  fp32: fp32 matmul over
+    column blocks of the live set (bounded memory), candidates merged per block."""
+    nq = queries.shape[0]
     if is_f32:
-        out = []
-        x = base[live_ids]
-        xn = (x * x).sum(1)
-        for lo in range(0, queries.shape[0], 128):
-            q = queries[lo:lo + 128]
-            d = -(q @ x.T) if metric == 1 else (xn[None, :] - 2 * (q @ x.T))
-            out.append(live_ids[torch.topk(d, k, dim=1, largest=False).indices])
-        return torch.cat(out)
+        best_d = torch.full((nq, k), float("inf"), device=base.device)
+        best_i = torch.zeros((nq, k), dtype=torch.int64, device=base.device)
+        step = 1 << 20
+        for lo in range(0, live_ids.numel(), step):
+            ids = live_ids[lo:lo + step]
+            x = base[ids]
+            xn = (x * x).sum(1)
+            for qlo in range(0, nq, 512):
+                q = queries[qlo:qlo + 512]
+                d = -(q @ x.T) if metric == 1 else (xn[None, :] - 2 * (q @ x.T))
+                dd, ii = torch.topk(d, min(k, d.shape[1]), dim=1, largest=False)
+                cat_d = torch.cat([best_d[qlo:qlo + 512], dd], 1)
+                cat_i = torch.cat([best_i[qlo:qlo + 512], ids[ii]], 1)
+                sel = torch.topk(cat_d, k, dim=1, largest=False).indices
+                best_d[qlo:qlo + 512] = torch.gather(cat_d, 1, sel)
+                best_i[qlo:qlo + 512] = torch.gather(cat_i, 1, sel)
+        return best_i
     x = base[live_ids].to(torch.float32)
     xn = (x * x).sum(1).to(torch.int64)
     out = []
-    for lo in range(0, queries.shape[0], 256):
+    for lo in range(0, nq, 256):
         q = queries[lo:lo + 256].to(torch.float32)
         dot = (q @ x.T).to(torch.int64)                      # exact: |dot| < 2^24
         d = (q * q).sum(1).to(torch.int64)[:, None] + xn[None, :] - 2 * dot

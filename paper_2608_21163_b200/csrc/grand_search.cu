@@ -81,7 +81,11 @@ __global__ void __launch_bounds__(kSearchWarps * 32, search_min_blocks<G, CPL>()
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int t = lane % G, team = lane / G;
   const uint32_t lt_mask = (1u << lane) - 1u;
-  const uint32_t L = a.L, R = a.g.R, H = 1u << a.hash_bits;
+#ifdef GRAND_SPEC_R
+  const uint32_t L = GRAND_SPEC_L, R = GRAND_SPEC_R, HB = GRAND_SPEC_HB, H = 1u << HB;
+#else
+  const uint32_t L = a.L, R = a.g.R, HB = a.hash_bits, H = 1u << HB;
+#endif
   const uint32_t Lp = (L + 1u) & ~1u, Rp = (R + 1u) & ~1u;
   unsigned char* base = smem_raw + (size_t)warp * per_warp_bytes;
   unsigned long long* beam = reinterpret_cast<unsigned long long*>(base);
@@ -93,7 +97,11 @@ __global__ void __launch_bounds__(kSearchWarps * 32, search_min_blocks<G, CPL>()
 
   const uint32_t nchunk = a.lay.nchunk, row_bytes = a.lay.row_bytes;
   const uint8_t* __restrict__ store = a.g.store;
+#ifdef GRAND_SPEC_R
+  constexpr bool tags16 = true;
+#else
   const bool tags16 = a.g.cap <= (1ull << (a.hash_bits + 14));
+#endif
   unsigned long long n_exp = 0, n_dist = 0;
 
   const uint64_t wglobal = (uint64_t)blockIdx.x * kSearchWarps + warp;
@@ -136,6 +144,10 @@ __global__ void __launch_bounds__(kSearchWarps * 32, search_min_blocks<G, CPL>()
 
     uint32_t beam_n = 0, nvis = 0, cursor = 0;
     unsigned long long alt_key = kKeyMax;  // best unexpanded entry besides the one being expanded
+#ifdef GRAND_ROWSPEC
+    uint32_t nrow[4] = {kInvalid, kInvalid, kInvalid, kInvalid};  // adjacency row loaded ahead for the likeliest next expansion
+    uint32_t nrow_id = kInvalid;
+#endif
 
     // Evaluate cid[0..n) against the query and merge the survivors into the worklist.
     auto process = [&](uint32_t n) {
@@ -200,7 +212,16 @@ __global__ void __launch_bounds__(kSearchWarps * 32, search_min_blocks<G, CPL>()
       if (m == 0) return;
       if (!a.boot_ids) {  // a new entry closer than every unexpanded one will be expanded next
         best = warp_min_key(best);
+#ifdef GRAND_ROWSPEC
+        if (best < key_clean(alt_key)) {
+          nrow_id = key_id(best);
+          const uint32_t* __restrict__ nr = a.g.adj + (size_t)nrow_id * R;
+#pragma unroll
+          for (int c = 0; c < 4; ++c) nrow[c] = (uint32_t)(c * 32 + lane) < R ? __ldg(nr + c * 32 + lane) : kInvalid;
+        }
+#else
         if (best < key_clean(alt_key)) prefetch_row(a.g.adj + (size_t)key_id(best) * R, R, lane);
+#endif
       }
       // rank the survivors among themselves (m is small)
       for (uint32_t j = lane; j < m; j += 32) {
@@ -270,7 +291,7 @@ __global__ void __launch_bounds__(kSearchWarps * 32, search_min_blocks<G, CPL>()
     } else if (a.entry != kInvalid) {
       if (lane == 0) {
         cid[0] = a.entry;
-        visit_fresh(hash, a.hash_bits, tags16, a.entry);
+        visit_fresh(hash, HB, tags16, a.entry);
       }
       __syncwarp();
       process(1);
@@ -305,17 +326,35 @@ __global__ void __launch_bounds__(kSearchWarps * 32, search_min_blocks<G, CPL>()
         // Rows are padded with the invalid id, so the whole row is read without waiting for deg[u].
         const uint32_t* __restrict__ row = a.g.adj + (size_t)u * R;
         uint32_t vrow[4];
+#ifdef GRAND_ROWSPEC
+        if (u == nrow_id) {
+#pragma unroll
+          for (int c = 0; c < 4; ++c) vrow[c] = nrow[c];
+        } else {
+#pragma unroll
+          for (int c = 0; c < 4; ++c) vrow[c] = (uint32_t)(c * 32 + lane) < R ? __ldg(row + c * 32 + lane) : kInvalid;
+        }
+        // the row of the likeliest next expansion is loaded ahead (process() replaces it when a closer candidate turns up)
+        nrow_id = kInvalid;
+        if (alt_key != kKeyMax) {
+          nrow_id = key_id(alt_key);
+          const uint32_t* __restrict__ nr = a.g.adj + (size_t)nrow_id * R;
+#pragma unroll
+          for (int c = 0; c < 4; ++c) nrow[c] = (uint32_t)(c * 32 + lane) < R ? __ldg(nr + c * 32 + lane) : kInvalid;
+        }
+#else
 #pragma unroll
         for (int c = 0; c < 4; ++c) vrow[c] = (uint32_t)(c * 32 + lane) < R ? __ldg(row + c * 32 + lane) : kInvalid;
         // While that load is in flight: pull the adjacency row of the likeliest next expansion towards L2
         // (process() does the same for a closer new candidate).
         if (alt_key != kKeyMax) prefetch_row(a.g.adj + (size_t)key_id(alt_key) * R, R, lane);
+#endif
         uint32_t n = 0;
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
           if ((uint32_t)(c * 32) < R) {
             const uint32_t v = vrow[c];
-            const bool fresh = v != kInvalid && (!a.check_live || bit_test(a.g.live, v)) && visit_fresh(hash, a.hash_bits, tags16, v);
+            const bool fresh = v != kInvalid && (!a.check_live || bit_test(a.g.live, v)) && visit_fresh(hash, HB, tags16, v);
             const unsigned bal = __ballot_sync(FULL, fresh);
             if (fresh) cid[n + __popc(bal & lt_mask)] = v;
             n += __popc(bal);

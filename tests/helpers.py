@@ -66,8 +66,11 @@ def run_stream(cfg, seed=0, check_each=True, oracle=True, gpu=True, opts=None, o
         g = gb.GrandIndex(cfg["dim"], cfg["dtype"], cfg["metric"], cfg["R"], cfg["L"], cfg["alpha"], capacity=cap,
                           max_batch=max(cfg.get("first_batch", 1), cfg["max_build_batch"], cfg["ins"], cfg["dele"], 1), mode=cfg["mode"], **opts)
 
+    st.row_of = np.full(cap, -1, np.int64)     # id -> row of the generated base array that the id holds now
+
     def ins(ids, rows, what):
         v = wl.vectors(*rows)
+        st.row_of[ids] = np.arange(rows[0], rows[0] + rows[1])
         if o:
             o.insert_batch(ids, v)
         if g:

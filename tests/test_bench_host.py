@@ -19,9 +19,10 @@ def test_reference_arm_prints_contract_line():
     assert r.returncode == 0, r.stderr[-2000:]
     line = json.loads(r.stdout.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["metric"] == "update_vectors_per_sec" and line["unit"] == "vectors/s"
-    assert line["value"] > 0 and line["higher_is_better"] is True and line["config"]["workload"] == "sift_u8_d128"
+    assert line["value"] > 0 and line["higher_is_better"] is True and line["config"]["workload"] == "deep_f32_d96"
     assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] >= 1
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["e2e"]["value"] == line["value"]
+    assert line["cpu_baseline"]["index_size_ratio"] == 400.0          # 8M built at full size, 20,000 in the sample
 
 
 def test_reference_arm_other_ranks_exit_silently():

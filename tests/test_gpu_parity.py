@@ -159,7 +159,8 @@ def test_tiny_config_stream_bit_exact():
 
 
 def test_sift_shaped_shrink_bit_exact():
-    """SIFT-shaped bytes (d=128, R=64, L=128) shrunk to 20k points: several insert/delete rounds."""
+    """SIFT-shaped bytes (d=128, R=64, L=128) shrunk to 20k points: several insert/delete rounds, the graph compared
+    after every batch."""
     cfg = small_cfg("sift_u8_d128", 0.02, rounds=3)
     o, g, wl, st = run_stream(cfg, seed=0)
     check_search(o, g, wl, cfg)
@@ -167,6 +168,48 @@ def test_sift_shaped_shrink_bit_exact():
     for L in (10, 32, 200):
         oi, od = o.search(q, 10, L)
         gi, gd = gpu_search(g, q, 10, L)
+        assert (oi == gi).all() and (od == gd.astype(np.float64)).all()
+
+
+def test_sift_shaped_100k_points_bit_exact():
+    """The same stream at 100,000 points (90,000 built in batches of up to 1,000, then three rounds of insert 1,000 +
+    delete 1,000): the graph after the build and after every round, then 1,000 searches, all bit for bit."""
+    cfg = small_cfg("sift_u8_d128", 0.1, rounds=3)
+    checked = []
+
+    def on_round(r, o, g, wl, st):
+        assert_same_graph(o, g, f"round {r}")
+        checked.append(r)
+
+    o, g, wl, st = run_stream(cfg, seed=0, check_each=False, on_round=on_round)
+    assert checked == [0, 1, 2] and o.live_count == 90_000
+    check_search(o, g, wl, cfg)
+    assert o.stats()["dead_edges_seen"] == 0
+
+
+def test_ids_above_the_tag_range_of_the_visited_cache_bit_exact():
+    """A capacity above 2^(hash_bits + 14) ids no longer fits the 16-bit tags of the visited cache: the search falls
+    back to a direct-mapped table of full ids.  A few thousand live ids spread over a capacity just above 2^22
+    (hash_bits = 8) take that path through inserts, a delete and searches."""
+    torch = torch_()
+    from paper_2608_21163_b200 import binding as gb
+    cap, dim, R, L, n = (1 << 22) + 4096, 16, 8, 24, 4000
+    ids_all = np.unique(np.linspace(0, cap - 1, n).astype(np.uint32))
+    assert ids_all[-1] >= (1 << 22) and len(ids_all) == n
+    vecs = synth.uniform_u8(41, "base", 0, n, dim)
+    o = go.Oracle(dim, go.U8, go.L2, R, L, 1.2, cap)
+    g = gb.GrandIndex(dim, gb.U8, gb.L2, R, L, 1.2, capacity=cap, max_batch=500, hash_bits=8)
+    for lo in range(0, n, 500):
+        o.insert_batch(ids_all[lo:lo + 500], vecs[lo:lo + 500])
+        g.insert_batch(torch.from_numpy(ids_all[lo:lo + 500]), torch.from_numpy(vecs[lo:lo + 500]))
+    assert_same_graph(o, g, "sparse ids, build")
+    dele = synth.choose_ids(41, "del", ids_all, 400)
+    o.delete_batch(dele); g.delete_batch(torch.from_numpy(dele))
+    assert_same_graph(o, g, "sparse ids, delete")
+    q = synth.uniform_u8(41, "query", 0, 300, dim)
+    for k, Ls in [(10, 24), (5, 100)]:
+        oi, od = o.search(q, k, Ls)
+        gi, gd = gpu_search(g, q, k, Ls)
         assert (oi == gi).all() and (od == gd.astype(np.float64)).all()
 
 
@@ -276,14 +319,16 @@ def test_fixed_degree_mode_bit_exact_on_bytes():
 
 
 # ------------------------------------------------------------------ fp32 streams: tolerance + recall
-@pytest.mark.parametrize("name,scale", [("deep_f32_d96", 0.002), ("gist_f32_d960", 0.004), ("embed_f32_d768_ip", 0.001)])
+# Sizes: the largest shrinks whose oracle build finishes in about a minute on the test box's host cores
+# (Deep-shaped 100,000 points, GIST-shaped 30,000, embedding-shaped 165,000).
+@pytest.mark.parametrize("name,scale", [("deep_f32_d96", 0.01), ("gist_f32_d960", 0.025), ("embed_f32_d768_ip", 0.03)])
 def test_fp32_streams_recall_matches_oracle(name, scale):
     cfg = small_cfg(name, scale, rounds=2, nq=200)
     cfg["first_batch"] = min(cfg["first_batch"], 500)
     cfg["max_build_batch"] = max(cfg["max_build_batch"], 500)
-    o, g, wl, st = run_stream(cfg, seed=0, check_each=False, oracle=True, gpu=False)
+    o, _, wl, st = run_stream(cfg, seed=0, check_each=False, oracle=True, gpu=False)
     _, g, _, st2 = run_stream(cfg, seed=0, check_each=False, oracle=False, gpu=True)
-    assert (st.live == st2.live).all()
+    assert (st.live == st2.live).all() and (st.row_of == st2.row_of).all()
     # structural invariants of the GPU graph
     adj, deg, live, entry = gpu_graph(g)
     mask = go.live_mask(live, len(deg))
@@ -291,31 +336,25 @@ def test_fp32_streams_recall_matches_oracle(name, scale):
     for v in np.flatnonzero(mask)[:2000]:
         r = adj[v, :deg[v]]
         assert mask[r].all() and v not in r and len(set(r.tolist())) == len(r)
-    n_rows = st.next_row
+    # the vector every live id holds now (ids are reused in the GIST-shaped stream: the row map says which)
+    live_ids = np.flatnonzero(st.live).astype(np.uint32)
+    gen = wl.vectors(0, st.next_row)
     base = np.zeros((wl.capacity(), cfg["dim"]), np.float32)
-    # regenerate what is live now (ids map to rows 1:1 unless ids are reused)
-    if not cfg["reuse_ids"]:
-        base[:n_rows] = wl.vectors(0, n_rows)
-        live_ids = np.flatnonzero(st.live).astype(np.uint32)
-        q = wl.queries()
-        truth = brute_force_topk(base, live_ids, q, 10, cfg["metric"])
-        oi, _ = o.search(q, 10, cfg["L"])
-        gi, gd = gpu_search(g, q, 10, cfg["L"])
-        r_o, r_g = recall_at_k(oi, truth), recall_at_k(gi, truth)
-        assert abs(r_o - r_g) <= 0.005, (r_o, r_g)
-        assert r_g > 0.8
-        for i in range(0, len(q), 7):
-            b = base[gi[i]].astype(np.float64)
-            qq = q[i].astype(np.float64)
-            exact = ((b - qq) ** 2).sum(1) if cfg["metric"] == go.L2 else -(b @ qq)
-            scale_ = np.abs(exact) if cfg["metric"] == go.L2 else np.linalg.norm(b, axis=1) * np.linalg.norm(qq)
-            assert (np.abs(gd[i] - exact) <= 1e-5 * scale_).all()
-    else:
-        q = wl.queries()
-        oi, _ = o.search(q, 10, cfg["L"])
-        gi, _ = gpu_search(g, q, 10, cfg["L"])
-        overlap = np.mean([len(set(a.tolist()) & set(b.tolist())) / 10 for a, b in zip(oi, gi)])
-        assert overlap > 0.97, overlap
+    base[live_ids] = gen[st.row_of[live_ids]]
+    q = wl.queries()
+    truth = brute_force_topk(base, live_ids, q, 10, cfg["metric"])
+    oi, _ = o.search(q, 10, cfg["L"])
+    gi, gd = gpu_search(g, q, 10, cfg["L"])
+    r_o, r_g = recall_at_k(oi, truth), recall_at_k(gi, truth)
+    print(f"{name} x{scale}: {len(live_ids)} live points, recall@10 oracle {r_o:.4f} gpu {r_g:.4f}")
+    assert abs(r_o - r_g) <= 0.005, (r_o, r_g)
+    assert r_g > 0.6
+    for i in range(0, len(q), 3):
+        b = base[gi[i]].astype(np.float64)
+        qq = q[i].astype(np.float64)
+        exact = ((b - qq) ** 2).sum(1) if cfg["metric"] == go.L2 else -(b @ qq)
+        scale_ = np.abs(exact) if cfg["metric"] == go.L2 else np.linalg.norm(b, axis=1) * np.linalg.norm(qq)
+        assert (np.abs(gd[i] - exact) <= 1e-5 * scale_).all()
 
 
 # ------------------------------------------------------------------ errors, host API, determinism
@@ -467,7 +506,10 @@ def test_mips_reduction_vamana_ip_matches_oracle():
     for i in range(len(q)):
         b = base[gi[i]].astype(np.float64)
         exact = -(b @ q[i].astype(np.float64))
-        assert (np.abs(gd[i] - exact) <= 1e-5 * np.linalg.norm(b, axis=1) * np.linalg.norm(q[i]) + 2e-6).all()
+        # the reduction reports (d - |q|^2 - M^2) / 2 with d the squared L2 distance of the augmented rows: the
+        # rounding error of d is relative to d <= |q|^2 + M^2 + 2 |q.x|, not to |q||x|, so that is the scale
+        # 1e-5 applies to here (M = 1)
+        assert (np.abs(gd[i] - exact) <= 1e-5 * 0.5 * ((q[i].astype(np.float64) ** 2).sum() + 1.0 + 2 * np.abs(exact))).all()
         assert (np.diff(gd[i]) >= -1e-6).all()
     with pytest.raises(gb.GrandError) as e:
         g.insert_batch(torch.from_numpy(dele[:2]), torch.from_numpy((base[:2] * 9).astype(np.float32)))
