@@ -139,6 +139,7 @@ struct grand_index {
   uint64_t max_requests = 0;       // request tuples a batch may emit (buffers below are sized for it at creation)
   uint64_t max_delete_edges = 0;   // in-neighbour entries a delete batch may touch
   Buf req_tgt, req_key, seg_keys, dirty;              // sized at creation for max_requests
+  Buf work;                                           // the dirty list split by the kind of rebuild a node needs (Vamana mode)
   Buf t_indeg, t_off, t_fill, t_src;                  // reverse graph of a delete batch, sized at creation
   Buf x_indeg, x_off, x_fill, x_src;                  // full reverse graph for grand_reverse_graph (introspection; grown on demand)
   Buf st_ids, st_vecs, st_out_ids, st_out_d;          // staging of the *_host entry points (updates: sized at creation)
@@ -264,6 +265,8 @@ int write_state_head(grand_index* idx, cudaStream_t s) {
   idx->h_state->ndirty = 0;
   idx->h_state->cursor = 0;
   idx->h_state->work = 0;
+  idx->h_state->nheavy = 0;
+  idx->h_state->nlight = 0;
   idx->h_state->nlive = idx->nlive;
   idx->h_state->total_in = 0;
   CK(cudaMemcpyAsync(idx->d_state, idx->h_state, offsetof(DevState, medoid_key), cudaMemcpyHostToDevice, s));
@@ -305,6 +308,7 @@ int ensure_requests(grand_index* idx, uint64_t nreq, cudaStream_t s) {
   if ((rc = ensure(idx, idx->req_key, nreq * 8, s))) return rc;
   if ((rc = ensure(idx, idx->seg_keys, nreq * 8, s))) return rc;
   if ((rc = ensure(idx, idx->dirty, nreq * 4, s))) return rc;
+  if (idx->mode == GRAND_MODE_VAMANA && !idx->approx && (rc = ensure(idx, idx->work, nreq * 4, s))) return rc;
   return GRAND_OK;
 }
 
@@ -497,7 +501,7 @@ int grand_destroy(grand_index* idx) {
   if (!idx) return GRAND_OK;
   cudaDeviceSynchronize();
   for (void* p : idx->owned) idx->dev_free(p, idx->user);
-  for (Buf* b : {&idx->req_tgt, &idx->req_key, &idx->seg_keys, &idx->dirty, &idx->sync_dirty, &idx->t_indeg, &idx->t_off, &idx->t_fill, &idx->t_src,
+  for (Buf* b : {&idx->req_tgt, &idx->req_key, &idx->seg_keys, &idx->dirty, &idx->work, &idx->sync_dirty, &idx->t_indeg, &idx->t_off, &idx->t_fill, &idx->t_src,
                  &idx->x_indeg, &idx->x_off, &idx->x_fill, &idx->x_src, &idx->st_ids, &idx->st_vecs, &idx->st_out_ids, &idx->st_out_d})
     if (b->p) idx->dev_free(b->p, idx->user);
   for (auto e : idx->ctr_done)
@@ -508,6 +512,23 @@ int grand_destroy(grand_index* idx) {
   for (auto& rd : idx->readers) for (auto e : rd) cudaEventDestroy(e);
   delete idx;
   return GRAND_OK;
+}
+
+// Vamana mode (exact delete): the dirty list is split into nodes that need the full rebuild and nodes whose row
+// cannot overflow; the rebuild then reads the split list.
+static void split_group_args(const grand_index* idx, GroupArgs& a) {
+  if (!idx->work.p) return;
+  a.work = (uint32_t*)idx->work.p;
+  a.work_cap = (uint32_t)(idx->work.bytes / 4);
+  a.light_max = 8;
+  a.deg = idx->deg;
+  a.R = idx->R;
+}
+static void split_rebuild_args(const grand_index* idx, RebuildArgs& a) {
+  if (!idx->work.p) return;
+  a.dirty = (const uint32_t*)idx->work.p;
+  a.split = 1;
+  a.dirty_cap = (uint32_t)(idx->work.bytes / 4);
 }
 
 // An update call that gives up after validation has marked its ids: clear the marks, drain the stream, report.
@@ -589,6 +610,7 @@ int grand_insert_batch(grand_index* idx, const uint32_t* ids, const void* vecs, 
     a.req_tgt = (uint32_t*)idx->req_tgt.p; a.req_key = (unsigned long long*)idx->req_key.p; a.nreq = n * R;
     a.cnt = idx->cnt; a.fill = idx->fill; a.start = idx->start; a.flag = idx->flag;
     a.dirty = (uint32_t*)idx->dirty.p; a.seg_keys = (unsigned long long*)idx->seg_keys.p; a.state = idx->d_state;
+    split_group_args(idx, a);
     CKB(launch_group_requests(a, s));
   }
   {
@@ -609,6 +631,7 @@ int grand_insert_batch(grand_index* idx, const uint32_t* ids, const void* vecs, 
       a.cnt = idx->cnt; a.fill = idx->fill; a.start = idx->start; a.flag = idx->flag;
       a.dirty = (uint32_t*)idx->dirty.p; a.seg_keys = (unsigned long long*)idx->seg_keys.p;
       a.max_blocks = (uint32_t)mbk; a.state = idx->d_state;
+      split_rebuild_args(idx, a);
       CKB(launch_rebuild(a, s));
       idx->stats.n_rebuild_launches++;
     }
@@ -746,6 +769,7 @@ int grand_delete_batch(grand_index* idx, const uint32_t* ids, uint64_t n, grand_
       a.req_tgt = d.req_tgt; a.req_key = d.req_key; a.nreq = nreq;
       a.cnt = idx->cnt; a.fill = idx->fill; a.start = idx->start; a.flag = idx->flag;
       a.dirty = d.dirty; a.seg_keys = (unsigned long long*)idx->seg_keys.p; a.state = idx->d_state;
+      split_group_args(idx, a);
       CKB(launch_group_requests(a, s));
     }
     {
@@ -757,6 +781,7 @@ int grand_delete_batch(grand_index* idx, const uint32_t* ids, uint64_t n, grand_
       a.dirty = d.dirty; a.seg_keys = (unsigned long long*)idx->seg_keys.p;
       const uint64_t most = (uint64_t)sm_count() * 16u;
       a.max_blocks = (uint32_t)(nreq < most ? nreq : most); a.state = idx->d_state;
+      split_rebuild_args(idx, a);
       CKB(launch_rebuild(a, s));
       idx->stats.n_rebuild_launches++;
     }

@@ -54,6 +54,20 @@ __global__ void group_alloc_kernel(const GroupArgs a) {
     if (lane == 31) base = atomicAdd(&a.state->cursor, inc);
     base = __shfl_sync(0xFFFFFFFFu, base, 31);
     if (k < nd) a.start[u] = base + inc - c;
+    if (a.work) {
+      const bool light = k < nd && c <= a.light_max && a.deg[u] + c <= a.R;
+      const unsigned lb = __ballot_sync(0xFFFFFFFFu, light), hb = __ballot_sync(0xFFFFFFFFu, k < nd && !light);
+      uint32_t lbase = 0, hbase = 0;
+      if (lane == 0) {
+        if (lb) lbase = atomicAdd(&a.state->nlight, (uint32_t)__popc(lb));
+        if (hb) hbase = atomicAdd(&a.state->nheavy, (uint32_t)__popc(hb));
+      }
+      lbase = __shfl_sync(0xFFFFFFFFu, lbase, 0);
+      hbase = __shfl_sync(0xFFFFFFFFu, hbase, 0);
+      const uint32_t lt = (1u << lane) - 1u;
+      if (light) a.work[a.work_cap - 1u - (lbase + __popc(lb & lt))] = u;
+      else if (k < nd) a.work[hbase + __popc(hb & lt)] = u;
+    }
   }
 }
 __global__ void group_scatter_kernel(const GroupArgs a) {

@@ -42,6 +42,8 @@ struct DevState {
   uint32_t ndirty;       // length of the dirty list
   uint32_t cursor;       // segment allocator for grouped requests
   uint32_t work;         // dynamic work counter of the rebuild kernel
+  uint32_t nheavy;       // dirty nodes listed for the warp-per-node rebuild (front of the work list) ...
+  uint32_t nlight;       // ... and for the team-per-node append / compaction (back of the work list)
   uint32_t pad_;
   unsigned long long nlive;
   unsigned long long total_in;   // sum of in-degrees of the delete batch
@@ -130,6 +132,14 @@ struct GroupArgs {
   uint32_t* dirty;  // dirty list
   unsigned long long* seg_keys;  // grouped keys
   DevState* state;
+  // Optional split of the dirty list for the Vamana rebuild (work == nullptr: no split).  A node whose row cannot
+  // overflow (deg + requests <= R) with at most light_max requests only needs its requests appended (and, in a delete
+  // batch, its row compacted): such nodes are listed from the back of `work`, all others from the front.
+  uint32_t* work;
+  uint32_t work_cap;
+  uint32_t light_max;
+  const uint32_t* deg;
+  uint32_t R;
 };
 cudaError_t launch_group_requests(const GroupArgs& a, cudaStream_t s);
 
@@ -143,7 +153,9 @@ struct RebuildArgs {
   const uint32_t* livemap; // visited-set delete mode: kept neighbours must be live ...
   const uint32_t* newmap;  // ... or members of the running insert batch (not published yet)
   uint32_t* cnt; uint32_t* fill; uint32_t* start; uint32_t* flag;
-  const uint32_t* dirty;
+  const uint32_t* dirty;   // the nodes to rebuild: state->ndirty entries, or, with `split`, the work list
+  uint32_t split;          // 1: `dirty` is a work list (heavy nodes from the front, light nodes from the back, dirty_cap entries)
+  uint32_t dirty_cap;
   unsigned long long* seg_keys;
   uint32_t max_blocks;
   DevState* state;

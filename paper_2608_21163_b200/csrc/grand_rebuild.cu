@@ -63,7 +63,7 @@ __global__ void __launch_bounds__(kRebuildWarps * 32) rebuild_kernel(const Rebui
   auto wsync = [] { __syncwarp(); };
   unsigned long long npair = 0, nbytes = 0;  // nbytes: what the method has to move for the rows this warp rebuilds
   uint32_t nprune = 0, ndone = 0;
-  const uint32_t ndirty = a.state->ndirty;
+  const uint32_t ndirty = a.split ? a.state->nheavy : a.state->ndirty;  // (split: the front of the work list)
 
   // one prune test: rows of candidates i < j (sorted positions), result into the bit matrix
   auto pair_test = [&](bool act, uint32_t i, uint32_t j, uint32_t& jprev, uint4 (&rj)[CPL]) {
@@ -535,6 +535,121 @@ __global__ void __launch_bounds__(kRebuildWarps * 32) rebuild_kernel(const Rebui
   }
 }
 
+// ---- dirty nodes whose row cannot overflow (deg + requests <= R, at most kLightReq requests): nothing is pruned,
+// the requests are appended in key order behind the kept part of the row, and in a delete batch the row is
+// compacted first.  A team of 8 lanes owns one node (four nodes per warp); the row travels through registers
+// (R <= 128: 16 slots per lane), the requests sit one per lane and are ranked against each other with shuffles.
+// The result is exactly what rebuild_kernel's "|C| <= R" branch stores.
+constexpr uint32_t kLightReq = 8;
+constexpr int kLightWarps = 4;
+
+__global__ void __launch_bounds__(kLightWarps * 32) rebuild_light_kernel(const RebuildArgs a) {
+  constexpr unsigned FULL = 0xFFFFFFFFu;
+  constexpr int TS = 8, SL = 16;  // team size, row slots per lane
+  const int lane = threadIdx.x & 31, t = lane & (TS - 1), tsh = lane & ~(TS - 1);
+  const uint32_t R = a.g.R, nlight = a.state->nlight;
+  const uint32_t below = (1u << t) - 1u;
+  const uint64_t team0 = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) / TS, nteams = ((uint64_t)gridDim.x * blockDim.x) / TS;
+  unsigned long long nbytes = 0;
+  uint32_t ndone = 0;
+  // warp-uniform trip count: the four teams of a warp run in lockstep (team votes are bytes of warp ballots)
+  for (uint64_t k0 = team0 - (uint64_t)(lane / TS); k0 < nlight; k0 += nteams) {
+    const uint64_t k = k0 + (uint64_t)(lane / TS);
+    const bool act = k < nlight;
+    const uint32_t u = act ? a.dirty[a.dirty_cap - 1u - (uint32_t)k] : 0u;
+    const uint32_t cntu = act ? a.cnt[u] : 0u;
+    const uint32_t startu = act ? a.start[u] : 0u;
+    const uint32_t du = act ? min(a.g.deg[u], R) : 0u;
+    const uint32_t pfx = act ? min((uint32_t)a.g.rowpfx[u], du) : 0u;
+    uint32_t* row = a.g.adj + (size_t)u * R;
+    uint32_t* rowd = a.g.rowd ? a.g.rowd + (size_t)u * R : nullptr;
+    // the request of this lane
+    unsigned long long key = kKeyMax;
+    if ((uint32_t)t < cntu) key = a.seg_keys[startu + t];
+    // the row, slot j * 8 + t in register j
+    uint32_t rv[SL], rd[SL];
+#pragma unroll
+    for (int j = 0; j < SL; ++j) {
+      const uint32_t sl = (uint32_t)j * TS + t;
+      rv[j] = sl < du ? row[sl] : kInvalid;
+      rd[j] = (rowd && sl < du) ? rowd[sl] : kInvalid;
+    }
+    // ---- keep = N_out(u) \ B, stable, written straight back (every slot is in a register by now)
+    uint32_t nk = 0, kp = 0, okbits = 0;
+#pragma unroll
+    for (int j = 0; j < SL; ++j) {
+      if ((uint32_t)j * TS < R) {  // (uniform)
+        const uint32_t sl = (uint32_t)j * TS + t;
+        const bool ok = sl < du && !(a.delmap && bit_test(a.delmap, rv[j]));
+        const unsigned tb = (__ballot_sync(FULL, ok) >> tsh) & 0xFFu;
+        if (ok) {
+          const uint32_t pos = nk + __popc(tb & below);
+          okbits |= 1u << j;
+          if (a.delmap) {  // (an insert batch leaves the kept part where it is)
+            row[pos] = rv[j];
+            if (rowd) rowd[pos] = rd[j];
+          }
+        }
+        const uint32_t inpfx = pfx > (uint32_t)j * TS ? min(pfx - (uint32_t)j * TS, (uint32_t)TS) : 0u;
+        kp += __popc(tb & ((1u << inpfx) - 1u));
+        nk += __popc(tb);
+      }
+    }
+    // ---- requests: rank by key, drop repeats, keep the first P, drop what the row already holds and u itself
+    uint32_t less = 0, eqb = 0;  // bit s: request s has a smaller key / the same key and a lower lane
+    const uint32_t klo = (uint32_t)key, khi = (uint32_t)(key >> 32);
+    const uint32_t cmax = __reduce_max_sync(FULL, cntu);  // most requests of any of the warp's four nodes
+#pragma unroll
+    for (int s2 = 0; s2 < TS; ++s2) {
+      if ((uint32_t)s2 >= cmax) break;
+      const unsigned long long ks = ((unsigned long long)__shfl_sync(FULL, khi, s2, TS) << 32) | __shfl_sync(FULL, klo, s2, TS);
+      if (ks < key) less |= 1u << s2;
+      if (ks == key && s2 < t) eqb |= 1u << s2;
+    }
+    const bool have = (uint32_t)t < cntu;
+    const bool first = have && eqb == 0;  // not a repeat of an earlier lane's request
+    const unsigned firstb = (__ballot_sync(FULL, first) >> tsh) & 0xFFu;
+    const uint32_t id = key_id(key);
+    bool inrow = false;
+#pragma unroll
+    for (int s2 = 0; s2 < TS; ++s2) {
+      if ((uint32_t)s2 >= cmax) break;
+      const uint32_t ids = __shfl_sync(FULL, id, s2, TS);
+      bool hit = false;
+#pragma unroll
+      for (int j = 0; j < SL; ++j) hit |= ((okbits >> j) & 1u) && rv[j] == ids;
+      const unsigned hb = (__ballot_sync(FULL, hit) >> tsh) & 0xFFu;
+      if (s2 == t) inrow = hb != 0;
+    }
+    const bool fresh = first && __popc(less & firstb) < a.P && id != u && !inrow;
+    const unsigned freshb = (__ballot_sync(FULL, fresh) >> tsh) & 0xFFu;
+    const uint32_t nC = nk + __popc(freshb);
+    if (fresh) {
+      const uint32_t pos = nk + __popc(less & freshb);
+      row[pos] = id;
+      if (rowd) rowd[pos] = khi;
+    }
+    // a compacted row ends earlier than before: the slots behind it go back to the invalid id
+    for (uint32_t sl = nC + t; sl < du; sl += TS) {
+      row[sl] = kInvalid;
+      if (rowd) rowd[sl] = kInvalid;
+    }
+    if (act && t == 0) {
+      a.g.deg[u] = nC;
+      a.g.rowpfx[u] = (uint8_t)kp;
+      a.cnt[u] = 0;
+      a.fill[u] = 0;
+      a.flag[u] = 0;
+      nbytes += 2ull * R * 4u + (unsigned long long)cntu * 12u;
+      ++ndone;
+    }
+  }
+  if (ndone) {
+    atomicAdd(&a.state->counters[CTR_DIRTY], (unsigned long long)ndone);
+    atomicAdd(&a.state->counters[CTR_RB_BYTES], nbytes);
+  }
+}
+
 template <typename T, int METRIC, int G, int CPL>
 static cudaError_t launch_rebuild_t(const RebuildArgs& a, cudaStream_t s) {
   const size_t per_warp = rebuild_smem_per_warp(a.g.R, a.P);
@@ -548,6 +663,13 @@ static cudaError_t launch_rebuild_t(const RebuildArgs& a, cudaStream_t s) {
   if (occ < 1) occ = 1;
   uint32_t blocks = (uint32_t)sm_count() * occ;
   if (blocks > a.max_blocks && a.max_blocks) blocks = a.max_blocks;
+  if (a.split) {
+    // the light nodes first (their launch is short); neither kernel touches a node of the other's list
+    uint32_t lb = (uint32_t)sm_count() * 8u;
+    if (lb > a.max_blocks && a.max_blocks) lb = a.max_blocks;
+    rebuild_light_kernel<<<lb, kLightWarps * 32, 0, s>>>(a);
+    count_launches(1);
+  }
   kern<<<blocks, kRebuildWarps * 32, smem, s>>>(a, (uint32_t)per_warp);
   count_launches(1);
   return cudaGetLastError();

@@ -70,9 +70,15 @@ constexpr int search_min_blocks() {
   return G == 32 ? (CPL >= 8 ? 3 : CPL >= 4 ? 5 : 8) : (CPL >= 6 ? 6 : 7);
 }
 
-template <typename T, int METRIC, int G, int CPL>
+// RC / LC: degree bound and worklist size as compile-time constants (0 = taken from the arguments).  On short rows
+// the kernel is bound by instruction issue, and the common parameter pairs get an instantiation whose loops over the
+// row and over the worklist are unrolled, whose worklist chunks travel through registers during a merge, and which
+// loads the adjacency row of the next expansion into registers one expansion ahead.
+template <typename T, int METRIC, int G, int CPL, int RC, int LC>
 __global__ void __launch_bounds__(kSearchWarps * 32, search_min_blocks<G, CPL>()) beam_search_kernel(const SearchArgs a, const uint32_t per_warp_bytes) {
   using Dist = typename Elem<T>::Dist;
+  constexpr int RW = RC ? (RC + 31) / 32 : 4;   // 32-id words of an adjacency row per lane
+  constexpr int LW = LC ? (LC + 31) / 32 : 1;   // worklist chunks (used only when LC is given)
   constexpr int NT = 32 / G;                                   // teams per warp
   constexpr int U = CPL == 1 ? 4 : ((CPL == 2 || G == 32) ? 2 : 1);  // vectors in flight per team
   constexpr unsigned FULL = 0xFFFFFFFFu;
@@ -81,11 +87,7 @@ __global__ void __launch_bounds__(kSearchWarps * 32, search_min_blocks<G, CPL>()
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int t = lane % G, team = lane / G;
   const uint32_t lt_mask = (1u << lane) - 1u;
-#ifdef GRAND_SPEC_R
-  const uint32_t L = GRAND_SPEC_L, R = GRAND_SPEC_R, HB = GRAND_SPEC_HB, H = 1u << HB;
-#else
-  const uint32_t L = a.L, R = a.g.R, HB = a.hash_bits, H = 1u << HB;
-#endif
+  const uint32_t L = LC ? (uint32_t)LC : a.L, R = RC ? (uint32_t)RC : a.g.R, HB = a.hash_bits, H = 1u << HB;
   const uint32_t Lp = (L + 1u) & ~1u, Rp = (R + 1u) & ~1u;
   unsigned char* base = smem_raw + (size_t)warp * per_warp_bytes;
   unsigned long long* beam = reinterpret_cast<unsigned long long*>(base);
@@ -97,11 +99,7 @@ __global__ void __launch_bounds__(kSearchWarps * 32, search_min_blocks<G, CPL>()
 
   const uint32_t nchunk = a.lay.nchunk, row_bytes = a.lay.row_bytes;
   const uint8_t* __restrict__ store = a.g.store;
-#ifdef GRAND_SPEC_R
-  constexpr bool tags16 = true;
-#else
   const bool tags16 = a.g.cap <= (1ull << (a.hash_bits + 14));
-#endif
   unsigned long long n_exp = 0, n_dist = 0;
 
   const uint64_t wglobal = (uint64_t)blockIdx.x * kSearchWarps + warp;
@@ -144,10 +142,15 @@ __global__ void __launch_bounds__(kSearchWarps * 32, search_min_blocks<G, CPL>()
 
     uint32_t beam_n = 0, nvis = 0, cursor = 0;
     unsigned long long alt_key = kKeyMax;  // best unexpanded entry besides the one being expanded
-#ifdef GRAND_ROWSPEC
-    uint32_t nrow[4] = {kInvalid, kInvalid, kInvalid, kInvalid};  // adjacency row loaded ahead for the likeliest next expansion
+    uint32_t nrow[RW];              // (RC given) adjacency row loaded ahead for the likeliest next expansion
     uint32_t nrow_id = kInvalid;
-#endif
+#pragma unroll
+    for (int c = 0; c < RW; ++c) nrow[c] = kInvalid;
+    auto load_adj_row = [&](uint32_t id, uint32_t (&dst)[RW]) {
+      const uint32_t* __restrict__ rp = a.g.adj + (size_t)id * R;
+#pragma unroll
+      for (int c = 0; c < RW; ++c) dst[c] = (uint32_t)(c * 32 + lane) < R ? __ldg(rp + c * 32 + lane) : kInvalid;
+    };
 
     // Evaluate cid[0..n) against the query and merge the survivors into the worklist.
     auto process = [&](uint32_t n) {
@@ -185,6 +188,44 @@ __global__ void __launch_bounds__(kSearchWarps * 32, search_min_blocks<G, CPL>()
       n_dist += n;
       if (nkept == 0) return;  // the common case late in a search: nothing enters the worklist
       __syncwarp();
+      if constexpr (LC > 0) {
+        if (nkept == 1) {
+          // one key: its rank is a count over the worklist chunks, which then move up by one through registers
+          const unsigned long long key = ckey[0];
+          unsigned long long e[LW];
+          uint32_t b = 0;
+          unsigned dup = 0;
+#pragma unroll
+          for (int c = 0; c < LW; ++c) {
+            const uint32_t i = (uint32_t)c * 32 + lane;
+            const bool in = i < beam_n;
+            e[c] = in ? beam[i] : 0ull;
+            const unsigned long long ec = key_clean(e[c]);
+            b += __popc(__ballot_sync(FULL, in && ec < key));
+            dup |= __ballot_sync(FULL, in && ec == key);
+          }
+          if (dup) return;  // already in the worklist
+          if (!a.boot_ids && key < key_clean(alt_key)) {  // it will be expanded next
+            if constexpr (RC > 0) {
+              nrow_id = key_id(key);
+              load_adj_row(nrow_id, nrow);
+            } else {
+              prefetch_row(a.g.adj + (size_t)key_id(key) * R, R, lane);
+            }
+          }
+          __syncwarp();
+#pragma unroll
+          for (int c = 0; c < LW; ++c) {
+            const uint32_t i = (uint32_t)c * 32 + lane;
+            if (i < beam_n && i >= b && i + 1 < L) beam[i + 1] = e[c];
+          }
+          if (lane == 0) beam[b] = key;
+          __syncwarp();
+          beam_n = min(L, beam_n + 1);
+          cursor = min(cursor, b);
+          return;
+        }
+      }
       // 2. drop keys that are already in the worklist; compact the rest in place (a write never passes the
       //    reader of its own chunk) and remember their ranks
       uint32_t m = 0;
@@ -212,16 +253,14 @@ __global__ void __launch_bounds__(kSearchWarps * 32, search_min_blocks<G, CPL>()
       if (m == 0) return;
       if (!a.boot_ids) {  // a new entry closer than every unexpanded one will be expanded next
         best = warp_min_key(best);
-#ifdef GRAND_ROWSPEC
         if (best < key_clean(alt_key)) {
-          nrow_id = key_id(best);
-          const uint32_t* __restrict__ nr = a.g.adj + (size_t)nrow_id * R;
-#pragma unroll
-          for (int c = 0; c < 4; ++c) nrow[c] = (uint32_t)(c * 32 + lane) < R ? __ldg(nr + c * 32 + lane) : kInvalid;
+          if constexpr (RC > 0) {
+            nrow_id = key_id(best);
+            load_adj_row(nrow_id, nrow);
+          } else {
+            prefetch_row(a.g.adj + (size_t)key_id(best) * R, R, lane);
+          }
         }
-#else
-        if (best < key_clean(alt_key)) prefetch_row(a.g.adj + (size_t)key_id(best) * R, R, lane);
-#endif
       }
       // rank the survivors among themselves (m is small)
       for (uint32_t j = lane; j < m; j += 32) {
@@ -236,7 +275,37 @@ __global__ void __launch_bounds__(kSearchWarps * 32, search_min_blocks<G, CPL>()
       //    down, so an entry that is still unread is never overwritten).  Entry i moves up by the
       //    number of survivors whose rank is <= i.
       const uint32_t minb = csb[0];
-      if (beam_n > minb) {
+      if constexpr (LC > 0) {
+        // every chunk is read into registers before any entry is written: no ordering between chunks is needed
+        unsigned long long e[LW];
+        uint32_t np[LW];
+#pragma unroll
+        for (int c = 0; c < LW; ++c) {
+          const uint32_t i = (uint32_t)c * 32 + lane;
+          np[c] = kInvalid;
+          e[c] = 0ull;
+          if (i < beam_n && i >= minb) {
+            e[c] = beam[i];
+            uint32_t sft = 0;
+            if (m <= 8) {
+              for (uint32_t r = 0; r < m; ++r) sft += csb[r] <= i;
+            } else {
+              uint32_t lo = 0, hi = m;  // first r with csb[r] > i
+              while (lo < hi) {
+                const uint32_t mid = (lo + hi) >> 1;
+                if (csb[mid] <= i) lo = mid + 1; else hi = mid;
+              }
+              sft = lo;
+            }
+            np[c] = i + sft;
+          }
+        }
+        __syncwarp();
+#pragma unroll
+        for (int c = 0; c < LW; ++c)
+          if (np[c] < L) beam[np[c]] = e[c];
+        __syncwarp();
+      } else if (beam_n > minb) {
         const int top = (int)((beam_n - 1) >> 5), low = (int)(minb >> 5);
         for (int ch = top; ch >= low; --ch) {
           const uint32_t i = (uint32_t)ch * 32 + lane;
@@ -324,34 +393,29 @@ __global__ void __launch_bounds__(kSearchWarps * 32, search_min_blocks<G, CPL>()
         ++nvis;
         const uint32_t u = key_id(ek);
         // Rows are padded with the invalid id, so the whole row is read without waiting for deg[u].
-        const uint32_t* __restrict__ row = a.g.adj + (size_t)u * R;
-        uint32_t vrow[4];
-#ifdef GRAND_ROWSPEC
-        if (u == nrow_id) {
+        uint32_t vrow[RW];
+        if constexpr (RC > 0) {
+          if (u == nrow_id) {
 #pragma unroll
-          for (int c = 0; c < 4; ++c) vrow[c] = nrow[c];
+            for (int c = 0; c < RW; ++c) vrow[c] = nrow[c];
+          } else {
+            load_adj_row(u, vrow);
+          }
+          // the row of the likeliest next expansion is loaded ahead (process() replaces it when a closer candidate turns up)
+          nrow_id = kInvalid;
+          if (alt_key != kKeyMax) {
+            nrow_id = key_id(alt_key);
+            load_adj_row(nrow_id, nrow);
+          }
         } else {
-#pragma unroll
-          for (int c = 0; c < 4; ++c) vrow[c] = (uint32_t)(c * 32 + lane) < R ? __ldg(row + c * 32 + lane) : kInvalid;
+          load_adj_row(u, vrow);
+          // While that load is in flight: pull the adjacency row of the likeliest next expansion towards L2
+          // (process() does the same for a closer new candidate).
+          if (alt_key != kKeyMax) prefetch_row(a.g.adj + (size_t)key_id(alt_key) * R, R, lane);
         }
-        // the row of the likeliest next expansion is loaded ahead (process() replaces it when a closer candidate turns up)
-        nrow_id = kInvalid;
-        if (alt_key != kKeyMax) {
-          nrow_id = key_id(alt_key);
-          const uint32_t* __restrict__ nr = a.g.adj + (size_t)nrow_id * R;
-#pragma unroll
-          for (int c = 0; c < 4; ++c) nrow[c] = (uint32_t)(c * 32 + lane) < R ? __ldg(nr + c * 32 + lane) : kInvalid;
-        }
-#else
-#pragma unroll
-        for (int c = 0; c < 4; ++c) vrow[c] = (uint32_t)(c * 32 + lane) < R ? __ldg(row + c * 32 + lane) : kInvalid;
-        // While that load is in flight: pull the adjacency row of the likeliest next expansion towards L2
-        // (process() does the same for a closer new candidate).
-        if (alt_key != kKeyMax) prefetch_row(a.g.adj + (size_t)key_id(alt_key) * R, R, lane);
-#endif
         uint32_t n = 0;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
+        for (int c = 0; c < RW; ++c) {
           if ((uint32_t)(c * 32) < R) {
             const uint32_t v = vrow[c];
             const bool fresh = v != kInvalid && (!a.check_live || bit_test(a.g.live, v)) && visit_fresh(hash, HB, tags16, v);
@@ -415,11 +479,11 @@ __global__ void __launch_bounds__(kSearchWarps * 32, search_min_blocks<G, CPL>()
   }
 }
 
-template <typename T, int METRIC, int G, int CPL>
-static cudaError_t launch_beam_search_t(const SearchArgs& a, cudaStream_t s) {
+template <typename T, int METRIC, int G, int CPL, int RC, int LC>
+static cudaError_t launch_beam_search_rl(const SearchArgs& a, cudaStream_t s) {
   const size_t per_warp = beam_search_smem_per_warp(a.L, a.g.R, a.hash_bits);
   const size_t smem = per_warp * kSearchWarps;
-  auto kern = beam_search_kernel<T, METRIC, G, CPL>;
+  auto kern = beam_search_kernel<T, METRIC, G, CPL, RC, LC>;
   static SmemOptIn optin{};
   cudaError_t e = allow_full_dynamic_smem((const void*)kern, &optin);
   if (e != cudaSuccess) return e;
@@ -433,6 +497,16 @@ static cudaError_t launch_beam_search_t(const SearchArgs& a, cudaStream_t s) {
   kern<<<(unsigned)blocks, kSearchWarps * 32, smem, s>>>(a, (uint32_t)per_warp);
   count_launches(1);
   return cudaGetLastError();
+}
+
+template <typename T, int METRIC, int G, int CPL>
+static cudaError_t launch_beam_search_t(const SearchArgs& a, cudaStream_t s) {
+  // short rows (teams of at most 8 lanes) with the usual parameter pairs take the unrolled instantiations
+  if constexpr (G <= 8) {
+    if (a.g.R == 64 && a.L == 128) return launch_beam_search_rl<T, METRIC, G, CPL, 64, 128>(a, s);
+    if (a.g.R == 32 && a.L == 64) return launch_beam_search_rl<T, METRIC, G, CPL, 32, 64>(a, s);
+  }
+  return launch_beam_search_rl<T, METRIC, G, CPL, 0, 0>(a, s);
 }
 
 cudaError_t launch_beam_search(const SearchArgs& a, cudaStream_t s) {
