@@ -574,10 +574,198 @@ __global__ void __launch_bounds__(kMmaWarps * 32) delete_picks_mma_kernel(const 
   if (nrows) atomicAdd(&a.state->counters[CTR_PK_BYTES], nrows * row_bytes);
 }
 
-// Which pick kernel serves this index: 2 = tensor-core tiles (integer rows up to 256 bytes, k_repair <= 56),
-// 1 = candidate rows staged in shared memory, 0 = rows straight from L2.
+// ---- register-tiled variant for fp32 rows of at most 384 bytes (teams of at most 4 lanes).  The pairs (x, y) of one
+// deleted node form a dense block of distances, x among its surviving in- and out-neighbours and y in C_i.  A work
+// unit stages up to kTileUnitPairs x rows and the candidate rows in shared memory; a thread owns a tile of 2 x rows by
+// 4 candidates, so six 16-byte shared-memory loads feed 64 arithmetic instructions, where a team per pair needs one
+// load per eight (the staged kernel spends its time on the shared-memory pipe and on per-pair bookkeeping).
+// Every distance is summed in exactly the order a team of G lanes uses (lane t of a team takes chunks t, t + G, ...
+// in sequence, then the lanes' partial sums fold pairwise), so the keys are bit for bit the ones the other kernels
+// compute for the same pair.  Each thread keeps the c smallest keys of its part of a row; the four threads that share
+// a row then merge their heads.
+// 16 bytes global -> shared without a round trip through registers; the copies of one thread complete in order of
+// issue and are awaited together
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
+  const unsigned sa = (unsigned)__cvta_generic_to_shared(smem_dst);
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sa), "l"(gsrc));
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
+constexpr uint32_t kTileUnitPairs = 64;
+constexpr int kTileWarps = 4;
+constexpr int kTileMaxC = 4;
+
+static size_t delete_picks_tile_smem(uint32_t nchunk, uint32_t k_repair) {
+  const size_t rs = (size_t)(nchunk | 1u) * 16u, kr16 = (k_repair + 15u) & ~15u;
+  return (kTileUnitPairs + kr16) * rs + kr16 * 8 + kTileUnitPairs * 4;
+}
+
+template <int G, int CPL>
+__global__ void __launch_bounds__(kTileWarps * 32) delete_picks_tile_kernel(const DeleteArgs a, const uint64_t total_in) {
+  constexpr unsigned FULL = 0xFFFFFFFFu;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int xr = lane >> 2, cg = lane & 3;
+  const uint32_t R = a.g.R, c = a.c, kr = a.k_repair, kr16 = (kr + 15u) & ~15u;
+  const uint32_t row_bytes = a.lay.row_bytes, nchunk = a.lay.nchunk;
+  const uint32_t rs = (nchunk | 1u) * 16u;  // odd number of chunks: rows of neighbouring lanes fall on different banks
+  uint8_t* xrow = smem_raw;
+  uint8_t* crow = xrow + (size_t)kTileUnitPairs * rs;
+  unsigned long long* ckeys = reinterpret_cast<unsigned long long*>(crow + (size_t)kr16 * rs);
+  uint32_t* xid = reinterpret_cast<uint32_t*>(ckeys + kr16);
+  const uint32_t nunits = a.unit_off[a.n];
+  unsigned long long npair = 0, nrows = 0;
+  for (uint32_t unit = blockIdx.x; unit < nunits; unit += gridDim.x) {
+    uint32_t lo = 0, hi = (uint32_t)a.n;  // largest i with unit_off[i] <= unit
+    while (hi - lo > 1) {
+      const uint32_t mid = (lo + hi) >> 1;
+      if (a.unit_off[mid] <= unit) lo = mid; else hi = mid;
+    }
+    const uint32_t i = lo, p = a.ids[i];
+    const uint32_t nin = a.pair_off[i + 1] - a.pair_off[i];
+    const uint32_t q0 = (unit - a.unit_off[i]) * kTileUnitPairs, q1 = min(nin + R, q0 + kTileUnitPairs);
+    const uint32_t M = q1 - q0, nc = min(a.Ci_n[i], kr);
+    __syncthreads();  // the previous unit's readers are done with the staged rows
+    for (uint32_t j = threadIdx.x; j < kr16; j += blockDim.x) ckeys[j] = j < nc ? a.Ci[(size_t)i * kr + j] : kKeyMax;
+    // the candidate rows are on their way (asynchronous copies) while the x ids are resolved
+    for (uint32_t e = threadIdx.x; e < kr16 * nchunk; e += blockDim.x) {
+      const uint32_t j = e / nchunk, ch = e - j * nchunk;
+      uint4* dst = reinterpret_cast<uint4*>(crow + (size_t)j * rs) + ch;
+      if (j < nc) cp_async16(dst, reinterpret_cast<const uint4*>(a.g.store + (size_t)key_id(a.Ci[(size_t)i * kr + j]) * row_bytes) + ch);
+      else *dst = make_uint4(0, 0, 0, 0);
+    }
+    for (uint32_t j = threadIdx.x; j < kTileUnitPairs; j += blockDim.x) {
+      const uint32_t q = q0 + j;
+      uint32_t x = kInvalid;
+      if (j < M) {
+        if (q < nin) {
+          x = a.src[in_base(a, i) + q];
+        } else if (q - nin < a.g.deg[p]) {
+          x = a.g.adj[(size_t)p * R + (q - nin)];
+        }
+        if (x != kInvalid && (bit_test(a.delmap, x) || (a.livemap && !bit_test(a.livemap, x)))) x = kInvalid;
+      }
+      xid[j] = x;
+    }
+    __syncthreads();
+    for (uint32_t e = threadIdx.x; e < kTileUnitPairs * nchunk; e += blockDim.x) {
+      const uint32_t j = e / nchunk, ch = e - j * nchunk;
+      const uint32_t x = xid[j];
+      uint4* dst = reinterpret_cast<uint4*>(xrow + (size_t)j * rs) + ch;
+      if (x != kInvalid) cp_async16(dst, reinterpret_cast<const uint4*>(a.g.store + (size_t)x * row_bytes) + ch);
+      else *dst = make_uint4(0, 0, 0, 0);
+    }
+    cp_async_wait_all();
+    __syncthreads();
+    // this thread's two x rows and its running picks for them
+    const uint32_t r0 = (uint32_t)warp * 16u + (uint32_t)xr * 2u;
+    const uint4* xp0 = reinterpret_cast<const uint4*>(xrow + (size_t)r0 * rs);
+    const uint4* xp1 = reinterpret_cast<const uint4*>(xrow + (size_t)(r0 + 1) * rs);
+    const uint32_t x0 = xid[r0], x1 = xid[r0 + 1];
+    unsigned long long best[2][kTileMaxC];
+#pragma unroll
+    for (int h = 0; h < 2; ++h)
+#pragma unroll
+      for (int r = 0; r < kTileMaxC; ++r) best[h][r] = kKeyMax;
+    if ((uint32_t)warp * 16u < M) {  // (uniform per warp: a warp without pairs only keeps the barriers company)
+      for (uint32_t cb = 0; cb < nc; cb += 16) {
+        float acc[2][4][G];
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+#pragma unroll
+          for (int jj = 0; jj < 4; ++jj)
+#pragma unroll
+            for (int t = 0; t < G; ++t) acc[h][jj][t] = 0.0f;
+        const uint4* cp = reinterpret_cast<const uint4*>(crow + (size_t)(cb + cg) * rs);
+        const uint32_t cstep = 4u * (rs / 16u);  // candidate cb + cg + 4 jj
+        // (candidate rows beyond nc are staged as zeros and carry the invalid key: a block is always swept whole -
+        // skipping the empty groups of the last block was measured and is slower)
+#pragma unroll
+        for (int cc = 0; cc < CPL; ++cc) {
+#pragma unroll
+          for (int t = 0; t < G; ++t) {
+            const uint32_t ch = (uint32_t)(t + cc * G);
+            if (ch < nchunk) {  // (uniform)
+              const uint4 xa = xp0[ch], xb = xp1[ch];
+#pragma unroll
+              for (int jj = 0; jj < 4; ++jj) {
+                const uint4 yv = cp[(size_t)jj * cstep + ch];
+                acc_chunk<float, kMetricL2>(xa, yv, acc[0][jj][t]);
+                acc_chunk<float, kMetricL2>(xb, yv, acc[1][jj][t]);
+              }
+            }
+          }
+        }
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj) {
+          const unsigned long long kc = ckeys[cb + cg + 4 * jj];
+          const uint32_t y = key_id(kc);
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            float d;
+            if constexpr (G == 4) d = (acc[h][jj][0] + acc[h][jj][2]) + (acc[h][jj][1] + acc[h][jj][3]);
+            else if constexpr (G == 2) d = acc[h][jj][0] + acc[h][jj][1];
+            else d = acc[h][jj][0];
+            const uint32_t x = h ? x1 : x0;
+            unsigned long long key = (kc != kKeyMax && y != x) ? make_key(d, y) : kKeyMax;
+            // keep the c smallest seen so far, ascending
+#pragma unroll
+            for (int r = 0; r < kTileMaxC; ++r) {
+              if ((uint32_t)r < c && key < best[h][r]) {
+                const unsigned long long tmp = best[h][r];
+                best[h][r] = key;
+                key = tmp;
+              }
+            }
+          }
+        }
+      }
+      // ---- the four threads that share a row merge their heads: round r takes the smallest head, its owner pops
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const uint32_t r = r0 + h, x = h ? x1 : x0;
+        const uint32_t q = q0 + r;
+        const bool is_in = q < nin;
+        const uint64_t rbase = is_in ? ((uint64_t)a.pair_off[i] + q) * c : (total_in + (uint64_t)i * R + (q - nin)) * c;
+        for (uint32_t round = 0; round < c; ++round) {
+          unsigned long long m = best[h][0];
+          m = min(m, __shfl_xor_sync(FULL, m, 1));
+          m = min(m, __shfl_xor_sync(FULL, m, 2));
+          if (m != kKeyMax && best[h][0] == m) {  // keys are distinct (one id per candidate): exactly one owner
+#pragma unroll
+            for (int rr = 0; rr + 1 < kTileMaxC; ++rr) best[h][rr] = best[h][rr + 1];
+            best[h][kTileMaxC - 1] = kKeyMax;
+          }
+          if (cg == 0 && r < M) {
+            if (x == kInvalid || m == kKeyMax) {
+              a.req_tgt[rbase + round] = kInvalid;
+            } else if (is_in) {
+              a.req_tgt[rbase + round] = x;
+              a.req_key[rbase + round] = m;
+            } else {
+              a.req_tgt[rbase + round] = key_id(m);
+              a.req_key[rbase + round] = (m & 0xFFFFFFFF00000000ull) | x;
+            }
+          }
+        }
+        if (cg == 0 && r < M && x != kInvalid) {
+          npair += nc;
+          ++nrows;  // x's row, fetched once per pair
+        }
+      }
+    }
+  }
+  if (npair) atomicAdd(&a.state->counters[CTR_PAIR], npair);
+  if (nrows) atomicAdd(&a.state->counters[CTR_PK_BYTES], nrows * row_bytes);
+}
+
+// Which pick kernel serves this index: 3 = register tiles (fp32 rows up to 384 bytes, c <= 4), 2 = tensor-core tiles
+// (integer rows up to 256 bytes, k_repair <= 56), 1 = candidate rows staged in shared memory, 0 = rows straight from L2.
 template <typename T>
 static int picks_variant(const DeleteArgs& a) {
+#ifndef GRAND_NO_TILE_PICKS
+  if (sizeof(T) == 4 && a.lay.G <= 4 && a.c <= (uint32_t)kTileMaxC && a.lay.metric == kMetricL2) return 3;
+#endif
   if (sizeof(T) == 1 && a.k_repair <= (uint32_t)kMmaNTiles * 8u && a.lay.row_bytes <= 256u) return 2;
   const size_t stage = (size_t)a.k_repair * ((a.lay.nchunk | 1u) * 16u);
   return stage <= 64 * 1024 ? 1 : 0;
@@ -597,7 +785,7 @@ static cudaError_t launch_delete_picks_prepare_t(const DeleteArgs& a, uint64_t t
   if (variant == 0) return cudaGetLastError();
   const uint64_t cap16 = (uint64_t)sm_count() * 16u;
   const unsigned ub = (unsigned)((a.n + 256) / 256 > cap16 ? cap16 : (a.n + 256) / 256);
-  delete_units_kernel<<<ub, 256, 0, s>>>(a, variant == 2 ? kMmaUnitPairs : kUnitPairs);
+  delete_units_kernel<<<ub, 256, 0, s>>>(a, variant == 3 ? kTileUnitPairs : variant == 2 ? kMmaUnitPairs : kUnitPairs);
   count_launches(1);
   return launch_exclusive_scan(a.in_cnt, a.unit_off, a.n + 1, a.scan_tmp, s);
 }
@@ -618,6 +806,20 @@ static cudaError_t launch_delete_picks_t(const DeleteArgs& a, uint64_t total_in,
       uint64_t blocks = (total + kMmaUnitPairs - 1) / kMmaUnitPairs + a.n;  // upper bound on the number of units
       if (blocks > sms * 8u) blocks = sms * 8u;
       kern<<<(unsigned)blocks, kMmaWarps * 32, smem, s>>>(a, total_in);
+      count_launches(1);
+      return cudaGetLastError();
+    }
+  }
+  if constexpr (sizeof(T) == 4 && G <= 4) {
+    if (variant == 3) {
+      const size_t smem = delete_picks_tile_smem(a.lay.nchunk, a.k_repair);
+      auto kern = delete_picks_tile_kernel<G, CPL>;
+      static SmemOptIn optin{};
+      cudaError_t e = allow_full_dynamic_smem((const void*)kern, &optin);
+      if (e != cudaSuccess) return e;
+      uint64_t blocks = (total + kTileUnitPairs - 1) / kTileUnitPairs + a.n;  // upper bound on the number of units
+      if (blocks > sms * 8u) blocks = sms * 8u;
+      kern<<<(unsigned)blocks, kTileWarps * 32, smem, s>>>(a, total_in);
       count_launches(1);
       return cudaGetLastError();
     }
