@@ -36,8 +36,17 @@ static size_t rebuild_smem_per_warp(uint32_t R, uint32_t P) {
   return (b + 15) / 16 * 16;
 }
 
+// Resident blocks per SM the register allocation must leave room for.  On rows of at most 512 bytes the kernel waits
+// on memory with few warps to hide it (103 registers allowed only 4 blocks on 128-byte rows, 93 only 5 on 384-byte
+// rows): 7 blocks (6 for the 6-chunk layout, where 7 starts to spill) took 7% off the launch on 384-byte rows and 4%
+// on 128-byte rows; 8 spills and is slower.  Whole-warp teams keep their registers (no gain measured there).
+template <int G, int CPL>
+constexpr int rebuild_min_blocks() {
+  return G == 32 ? 1 : (CPL >= 6 ? 6 : 7);
+}
+
 template <typename T, int METRIC, int G, int CPL>
-__global__ void __launch_bounds__(kRebuildWarps * 32) rebuild_kernel(const RebuildArgs a, const uint32_t per_warp_bytes) {
+__global__ void __launch_bounds__(kRebuildWarps * 32, rebuild_min_blocks<G, CPL>()) rebuild_kernel(const RebuildArgs a, const uint32_t per_warp_bytes) {
   using Dist = typename Elem<T>::Dist;
   constexpr unsigned FULL = 0xFFFFFFFFu;
   constexpr int NT = 32 / G;
