@@ -423,13 +423,27 @@ def run_workload(args, torch, gb, dev, dist, rank, world, name, scale, K, W, Kp,
     #      profiled steps, on the launching stream) against the measured HBM copy bandwidth
     peak, peak_kind = read_peaks()
 
-    def roof(kernel, nbytes, ms, launches_, what):
+    # fp32 FFMA peak for the kernels that are dense blocks of pair distances rather than gathers: SMs x 128 lanes x 2 flop
+    # x the maximum SM clock.  A squared-L2 term is a subtract and a fused multiply-add (3 flop in 2 issue slots), so
+    # 0.75 of this figure is the most such a kernel can show.
+    props = torch.cuda.get_device_properties(dev)
+    fp32_peak = props.multi_processor_count * 128 * 2 * 1.965e9 / 1e12
+
+    def roof(kernel, nbytes, ms, launches_, what, pairs=None):
         if not launches_ or ms <= 0:
             return None
         ach = nbytes / (ms * 1e-3) / 1e9
-        return {"bound": "hbm", "kernel": kernel, "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
-                "peak_kind": peak_kind, "traffic": None, "algorithmic_bytes_per_launch": nbytes / launches_,
-                "launches": launches_, "avg_launch_ms": ms / launches_, "bytes_counted": what}
+        r = {"bound": "hbm", "kernel": kernel, "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
+             "peak_kind": peak_kind, "traffic": None, "algorithmic_bytes_per_launch": nbytes / launches_,
+             "launches": launches_, "avg_launch_ms": ms / launches_, "bytes_counted": what}
+        if pairs:
+            r["pair_distances_per_sec"] = pairs / (ms * 1e-3)
+            if is_f32:
+                tf = 3.0 * cfg["dim"] * pairs / (ms * 1e-3) / 1e12
+                r["alu"] = {"bound": "alu", "achieved": tf, "peak": fp32_peak, "unit": "TFLOP/s", "frac": tf / fp32_peak,
+                            "flops_counted": "3 x dim per pair distance (subtract, multiply, add)",
+                            "peak_kind": "nominal: SMs x 128 fp32 lanes x 2 x 1.965 GHz"}
+        return r
 
     search_bytes = stats["expansions"] * (cfg["R"] * 4 + 4) + stats["dist_evals"] * row_bytes
     rooflines = {
@@ -438,9 +452,10 @@ def run_workload(args, torch, gb, dev, dist, rank, world, name, scale, K, W, Kp,
         "rebuild": roof("rebuild_kernel", stats["rebuild_bytes"], stats["ms_rebuild"], stats["n_rebuild_launches"],
                         "per rebuilt row: row read + write (2 x R x 4), request tuples (12 each), and one vector per candidate when a prune runs"),
         "delete_picks": roof("delete_picks_*_kernel", stats["picks_bytes"], stats["ms_picks"], stats["n_picks_launches"],
-                             "one vector per (deleted node, surviving in-/out-neighbour) pair + the repair candidates' vectors per deleted node"),
+                             "one vector per (deleted node, surviving in-/out-neighbour) pair + the repair candidates' vectors per deleted node",
+                             pairs=stats["picks_pair_dists"]),
         "forward_prune": roof("forward_prune_*_kernel", stats["prune_bytes"], stats["ms_prune"], stats["n_prune_launches"],
-                              "one vector per candidate the prune looks at"),
+                              "one vector per candidate the prune looks at", pairs=stats["prune_pair_dists"]),
         "reverse_graph": roof("transpose_hist/scatter_kernel", stats["n_transpose_launches"] * 2 * (cap * 4 + live_edges * 4),
                               stats["ms_transpose"], stats["n_transpose_launches"],
                               "two passes over the degrees and the live adjacency entries (scan and scatter of the batch's rows not counted)"),

@@ -124,6 +124,8 @@ typedef struct {
   uint64_t n_rebuild_launches;
   uint64_t n_picks_launches;
   uint64_t n_transpose_launches;
+  uint64_t picks_pair_dists; /* node-to-node distances evaluated by the repair picks alone ... */
+  uint64_t prune_pair_dists; /* ... and by the forward RobustPrune alone (both are part of pair_dists) */
 } grand_stats;
 
 /* Index life cycle (problem statement of Sec. 3-4: capacity fixed at initialisation, ids in

@@ -42,7 +42,8 @@ class GrandStats(C.Structure):
                 ("ms_search", C.c_double), ("ms_prune", C.c_double), ("ms_group", C.c_double),
                 ("ms_rebuild", C.c_double), ("ms_transpose", C.c_double), ("ms_picks", C.c_double),
                 ("ms_other", C.c_double), ("n_search_launches", C.c_uint64), ("n_prune_launches", C.c_uint64),
-                ("n_rebuild_launches", C.c_uint64), ("n_picks_launches", C.c_uint64), ("n_transpose_launches", C.c_uint64)]
+                ("n_rebuild_launches", C.c_uint64), ("n_picks_launches", C.c_uint64), ("n_transpose_launches", C.c_uint64),
+                ("picks_pair_dists", C.c_uint64), ("prune_pair_dists", C.c_uint64)]
 
     def as_dict(self):
         return {k: getattr(self, k) for k, _ in self._fields_}

@@ -982,6 +982,8 @@ int grand_get_stats(const grand_index* cidx, grand_stats* out) {
   idx->stats.picks_bytes = st.counters[CTR_PK_BYTES];
   idx->stats.prune_bytes = st.counters[CTR_FP_BYTES];
   idx->stats.rebuild_prunes = st.counters[CTR_RB_PRUNED];
+  idx->stats.picks_pair_dists = st.counters[CTR_PK_PAIRS];
+  idx->stats.prune_pair_dists = st.counters[CTR_FP_PAIRS];
   idx->stats.kernel_launches = idx->launches;
   *out = idx->stats;
   return GRAND_OK;

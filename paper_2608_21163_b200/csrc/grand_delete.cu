@@ -206,7 +206,10 @@ __global__ void __launch_bounds__(kPickWarps * 32) delete_picks_kernel(const Del
       __syncwarp();
     }
   }
-  if (npair) atomicAdd(&a.state->counters[CTR_PAIR], npair);
+  if (npair) {
+    atomicAdd(&a.state->counters[CTR_PAIR], npair);
+    atomicAdd(&a.state->counters[CTR_PK_PAIRS], npair);
+  }
   if (nrows) atomicAdd(&a.state->counters[CTR_PK_BYTES], nrows * row_bytes);
 }
 // Every surviving in-neighbour of a deleted node is dirty even if it receives no candidate.
@@ -416,7 +419,10 @@ __global__ void __launch_bounds__(kPickWarps * 32) delete_picks_staged_kernel(co
       }
     }
   }
-  if (npair) atomicAdd(&a.state->counters[CTR_PAIR], npair);
+  if (npair) {
+    atomicAdd(&a.state->counters[CTR_PAIR], npair);
+    atomicAdd(&a.state->counters[CTR_PK_PAIRS], npair);
+  }
   if (nrows) atomicAdd(&a.state->counters[CTR_PK_BYTES], nrows * row_bytes);
 }
 
@@ -570,7 +576,10 @@ __global__ void __launch_bounds__(kMmaWarps * 32) delete_picks_mma_kernel(const 
       }
     }
   }
-  if (npair) atomicAdd(&a.state->counters[CTR_PAIR], npair);
+  if (npair) {
+    atomicAdd(&a.state->counters[CTR_PAIR], npair);
+    atomicAdd(&a.state->counters[CTR_PK_PAIRS], npair);
+  }
   if (nrows) atomicAdd(&a.state->counters[CTR_PK_BYTES], nrows * row_bytes);
 }
 
@@ -755,7 +764,10 @@ __global__ void __launch_bounds__(kTileWarps * 32) delete_picks_tile_kernel(cons
       }
     }
   }
-  if (npair) atomicAdd(&a.state->counters[CTR_PAIR], npair);
+  if (npair) {
+    atomicAdd(&a.state->counters[CTR_PAIR], npair);
+    atomicAdd(&a.state->counters[CTR_PK_PAIRS], npair);
+  }
   if (nrows) atomicAdd(&a.state->counters[CTR_PK_BYTES], nrows * row_bytes);
 }
 

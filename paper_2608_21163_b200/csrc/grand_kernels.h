@@ -54,7 +54,7 @@ struct DevState {
 // bytes the method itself has to move in the rebuild, repair-pick and forward-prune kernels (what each kernel
 // counts is stated where it counts), and the rebuilt rows that went through a prune
 enum { CTR_EXP = 0, CTR_DIST = 1, CTR_PAIR = 2, CTR_DIRTY = 3, CTR_PRUNE = 4, CTR_REQ = 5, CTR_RB_BYTES = 6, CTR_PK_BYTES = 7,
-       CTR_FP_BYTES = 8, CTR_RB_PRUNED = 9 };
+       CTR_FP_BYTES = 8, CTR_RB_PRUNED = 9, CTR_PK_PAIRS = 10, CTR_FP_PAIRS = 11 };  // + pair distances of the picks / forward prune alone
 
 struct GraphView {
   const uint8_t* store;

@@ -119,7 +119,10 @@ __global__ void __launch_bounds__(kPruneThreads) forward_prune_kernel(const Prun
     }
     __syncthreads();
   }
-  if (npair) atomicAdd(&a.state->counters[CTR_PAIR], npair);
+  if (npair) {
+    atomicAdd(&a.state->counters[CTR_PAIR], npair);
+    atomicAdd(&a.state->counters[CTR_FP_PAIRS], npair);
+  }
   if (tid == 0 && nprune) atomicAdd(&a.state->counters[CTR_PRUNE], (unsigned long long)nprune);
   if (tid == 0 && nrows) atomicAdd(&a.state->counters[CTR_FP_BYTES], nrows * a.lay.row_bytes);
 }
@@ -215,7 +218,10 @@ __global__ void __launch_bounds__(kWarpPruneWarps * 32) forward_prune_warp_kerne
     }
     __syncwarp();
   }
-  if (npair) atomicAdd(&a.state->counters[CTR_PAIR], npair);
+  if (npair) {
+    atomicAdd(&a.state->counters[CTR_PAIR], npair);
+    atomicAdd(&a.state->counters[CTR_FP_PAIRS], npair);
+  }
   if (lane == 0 && nprune) atomicAdd(&a.state->counters[CTR_PRUNE], (unsigned long long)nprune);
   if (lane == 0 && nrows) atomicAdd(&a.state->counters[CTR_FP_BYTES], nrows * row_bytes);
 }
@@ -422,7 +428,10 @@ __global__ void __launch_bounds__(kMmaPruneWarps * 32) forward_prune_mma_kernel(
     }
     __syncwarp();
   }
-  if (npair) atomicAdd(&a.state->counters[CTR_PAIR], npair);
+  if (npair) {
+    atomicAdd(&a.state->counters[CTR_PAIR], npair);
+    atomicAdd(&a.state->counters[CTR_FP_PAIRS], npair);
+  }
   if (lane == 0 && nprune) atomicAdd(&a.state->counters[CTR_PRUNE], (unsigned long long)nprune);
   if (lane == 0 && nrows) atomicAdd(&a.state->counters[CTR_FP_BYTES], nrows * row_bytes);
 }

@@ -143,8 +143,55 @@ __global__ void __launch_bounds__(kRebuildWarps * 32, rebuild_min_blocks<G, CPL>
       }
     }
     __syncwarp();
-    bitonic_sort_any(seg, cntu, (uint32_t)lane, 32u, wsync);
     uint32_t ns = 0;
+    if (cntu > kSegSmem) {
+      // A hub can be the target of a large part of a batch's requests (hundreds of thousands on data with strong
+      // hubness), and only the P smallest distinct keys are wanted: the segment is streamed once against a sorted
+      // list of the best P so far instead of being sorted.  After the first few chunks almost every key fails the
+      // comparison with the list's last entry.  Same list as sort + drop repeats + cut at P.
+      for (uint32_t jb0 = 0; jb0 < cntu; jb0 += 128) {
+       unsigned long long k4[4];  // four chunks requested together: the stream is a chain of dependent steps otherwise
+#pragma unroll
+       for (int q = 0; q < 4; ++q) k4[q] = jb0 + q * 32 + lane < cntu ? seg[jb0 + q * 32 + lane] : kKeyMax;
+#pragma unroll
+       for (int q = 0; q < 4; ++q) {
+        const unsigned long long kk = k4[q];
+        const unsigned long long thr = ns == P ? scratch[P - 1] : kKeyMax;
+        unsigned bal = __ballot_sync(FULL, kk < thr);
+        while (bal) {  // (uniform)
+          const int srcl = __ffs(bal) - 1;
+          bal &= bal - 1u;
+          const unsigned long long key = ((unsigned long long)__shfl_sync(FULL, (uint32_t)(kk >> 32), srcl) << 32) |
+                                         __shfl_sync(FULL, (uint32_t)kk, srcl);
+          if (ns == P && !(key < scratch[P - 1])) continue;  // the list has tightened since the ballot
+          uint32_t pos = 0;
+          unsigned dup = 0;
+          for (uint32_t cb = 0; cb < ns; cb += 32) {
+            const uint32_t i = cb + lane;
+            const unsigned long long e = i < ns ? scratch[i] : kKeyMax;
+            pos += __popc(__ballot_sync(FULL, e < key));
+            dup |= __ballot_sync(FULL, e == key);
+          }
+          if (dup) continue;
+          const uint32_t last = min(ns, P - 1u);  // entries [pos, last) move up by one; a full list drops its last entry
+          if (last > pos) {
+            for (int ch = (int)((last - 1u) >> 5); ch >= (int)(pos >> 5); --ch) {
+              const uint32_t i = (uint32_t)ch * 32u + lane;
+              const bool mv = i >= pos && i < last;
+              const unsigned long long e = mv ? scratch[i] : 0ull;
+              __syncwarp();
+              if (mv) scratch[i + 1] = e;
+            }
+          }
+          __syncwarp();
+          if (lane == 0) scratch[pos] = key;
+          __syncwarp();
+          ns = min(ns + 1u, P);
+        }
+       }
+      }
+    } else {
+    bitonic_sort_any(seg, cntu, (uint32_t)lane, 32u, wsync);
     for (uint32_t jb = 0; jb < cntu && ns < P; jb += 32) {
       const uint32_t j = jb + lane;
       bool ok = j < cntu;
@@ -159,6 +206,7 @@ __global__ void __launch_bounds__(kRebuildWarps * 32, rebuild_min_blocks<G, CPL>
       ns += __popc(bal);
     }
     ns = min(ns, P);
+    }
     // ---- keep = N_out(u) \ B, stable; kp = how many kept entries come from the pruned prefix
     uint32_t nk = 0, kp = 0;
 #pragma unroll
