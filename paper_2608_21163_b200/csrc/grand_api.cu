@@ -741,7 +741,7 @@ int grand_delete_batch(grand_index* idx, const uint32_t* ids, uint64_t n, grand_
   if (fixed) {
     PhaseTimer pt(idx, s, PH_REBUILD);
     FixedDeleteArgs f{};
-    f.g = g; f.ids = ids; f.n = n; f.delmap = idx->mark; f.off = d.off; f.src = d.src; f.pair_off = idx->pair_off;
+    f.g = g; f.ids = ids; f.n = n; f.delmap = idx->mark; f.off = d.off; f.src = (uint32_t*)idx->t_src.p; f.pair_off = idx->pair_off;
     f.flag = idx->flag; f.dirty = (uint32_t*)idx->dirty.p; f.state = idx->d_state;
     CKB(launch_fixed_delete(f, total_in, s));
   } else {

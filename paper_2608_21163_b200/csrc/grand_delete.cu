@@ -879,12 +879,53 @@ __global__ void fixed_delete_mark_kernel(const FixedDeleteArgs a, const uint64_t
     if (!bit_test(a.delmap, u) && atomicExch(&a.flag[u], 1u) == 0u) a.dirty[atomicAdd(&a.state->ndirty, 1u)] = u;
   }
 }
+// In-neighbour rows come out of the scatter in no particular order.  The rank of u in such a row is
+// counted directly while the row is short; long rows (hubs: in-degrees are heavy-tailed, and every
+// in-neighbour of a deleted hub asks for its own rank) are sorted once, so that the rank is a
+// binary search instead of a pass over the row per in-neighbour.
+constexpr uint32_t kRankLinear = 256;
+constexpr uint32_t kSortRowSmem = 48 * 1024;  // entries of a long row sorted in shared memory
+__global__ void __launch_bounds__(1024) fixed_delete_sort_rows_kernel(const FixedDeleteArgs a) {
+  extern __shared__ uint32_t sort_sh[];  // kSortRowSmem entries, then the list of long rows and its length
+  uint32_t* longrow = sort_sh + kSortRowSmem;
+  uint32_t& nlong = sort_sh[kSortRowSmem + 1024];
+  auto sync = [] { __syncthreads(); };
+  const uint32_t tid = threadIdx.x;
+  for (uint64_t base = (uint64_t)blockIdx.x * 1024u; base < a.n; base += (uint64_t)gridDim.x * 1024u) {
+    if (tid == 0) nlong = 0;
+    __syncthreads();
+    if (base + tid < a.n) {
+      const uint32_t p = a.ids[base + tid];
+      if (a.off[p + 1] - a.off[p] > kRankLinear) longrow[atomicAdd(&nlong, 1u)] = p;
+    }
+    __syncthreads();
+    const uint32_t nl = nlong;
+    for (uint32_t r = 0; r < nl; ++r) {
+      const uint32_t p = longrow[r];
+      const uint32_t b = a.off[p], n = a.off[p + 1] - b;
+      if (n <= kSortRowSmem) {
+        for (uint32_t j = tid; j < n; j += 1024u) sort_sh[j] = a.src[b + j];
+        __syncthreads();
+        bitonic_sort_any(sort_sh, n, tid, 1024u, sync);
+        for (uint32_t j = tid; j < n; j += 1024u) a.src[b + j] = sort_sh[j];
+      } else {
+        bitonic_sort_any(a.src + b, n, tid, 1024u, sync);
+      }
+      __syncthreads();
+    }
+  }
+}
+// The deleted slots of a row are found with one parallel bitmap test per 32 slots, and a deleted
+// neighbour's row is staged once with its own parallel test, so that a dirty node costs a handful
+// of dependent memory round trips instead of one per slot and per candidate.
 __global__ void __launch_bounds__(128) fixed_delete_rewire_kernel(const FixedDeleteArgs a) {
   constexpr unsigned FULL = 0xFFFFFFFFu;
   constexpr uint32_t kMaxR = 128;
   __shared__ uint32_t rows[4][kMaxR];
+  __shared__ uint32_t prows[4][kMaxR];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   uint32_t* row = rows[warp];
+  uint32_t* prow = prows[warp];
   const uint32_t R = a.g.R;
   const uint32_t nd = a.state->ndirty;
   const uint64_t wglobal = (uint64_t)blockIdx.x * 4 + warp, wtotal = (uint64_t)gridDim.x * 4;
@@ -892,44 +933,81 @@ __global__ void __launch_bounds__(128) fixed_delete_rewire_kernel(const FixedDel
   for (uint64_t k = wglobal; k < nd; k += wtotal) {
     const uint32_t u = a.dirty[k];
     const uint32_t du = min(a.g.deg[u], R);
-    for (uint32_t s = lane; s < du; s += 32) row[s] = a.g.adj[(size_t)u * R + s];
+    uint32_t delw = 0;  // lane w: word w of the set of slots that hold a deleted neighbour
+    for (uint32_t sb = 0; sb < du; sb += 32) {
+      const uint32_t s = sb + lane;
+      uint32_t v = kInvalid;
+      if (s < du) {
+        v = a.g.adj[(size_t)u * R + s];
+        row[s] = v;
+      }
+      const unsigned bal = __ballot_sync(FULL, v != kInvalid && bit_test(a.delmap, v));
+      if ((uint32_t)lane == (sb >> 5)) delw = bal;
+    }
     __syncwarp();
-    for (uint32_t s = 0; s < du; ++s) {
-      const uint32_t p = row[s];
-      if (p == kInvalid || !bit_test(a.delmap, p)) continue;  // warp-uniform
-      // round-robin offset: rank of u among the in-neighbours of p
-      const uint32_t b = a.off[p], e = a.off[p + 1];
-      uint32_t rank = 0;
-      for (uint32_t jb = b; jb < e; jb += 32) {
-        const uint32_t j = jb + lane;
-        rank += __popc(__ballot_sync(FULL, j < e && a.src[j] < u));
+    for (uint32_t w = 0; w * 32 < du; ++w) {
+      uint32_t m = __shfl_sync(FULL, delw, w);
+      while (m) {
+        const uint32_t s = w * 32 + (uint32_t)__ffs(m) - 1u;
+        m &= m - 1;
+        const uint32_t p = row[s];
+        // round-robin offset: rank of u among the in-neighbours of p
+        const uint32_t b = a.off[p], e = a.off[p + 1];
+        uint32_t rank = 0;
+        if (e - b > kRankLinear) {  // sorted by fixed_delete_sort_rows_kernel
+          uint32_t lo = b, hi = e;
+          while (lo < hi) {
+            const uint32_t mid = lo + ((hi - lo) >> 1);
+            if (a.src[mid] < u) lo = mid + 1; else hi = mid;
+          }
+          rank = lo - b;
+        } else {
+          for (uint32_t jb = b; jb < e; jb += 32) {
+            const uint32_t j = jb + lane;
+            rank += __popc(__ballot_sync(FULL, j < e && a.src[j] < u));
+          }
+        }
+        const uint32_t np = min(a.g.deg[p], R);
+        uint32_t okw = 0;  // lane x: word x of the set of p's neighbours that are alive and not u itself
+        for (uint32_t ib = 0; ib < np; ib += 32) {
+          const uint32_t i = ib + lane;
+          bool ok = false;
+          if (i < np) {
+            const uint32_t c = a.g.adj[(size_t)p * R + i];
+            prow[i] = c;
+            ok = c != u && !bit_test(a.delmap, c);
+          }
+          const unsigned bal = __ballot_sync(FULL, ok);
+          if ((uint32_t)lane == (ib >> 5)) okw = bal;
+        }
+        __syncwarp();
+        uint32_t chosen = kInvalid;
+        for (uint32_t tt = 0; tt < np && chosen == kInvalid; ++tt) {
+          const uint32_t i = (rank + tt) % np;
+          if (!((__shfl_sync(FULL, okw, i >> 5) >> (i & 31)) & 1u)) continue;
+          const uint32_t cand = prow[i];
+          bool inrow = false;
+          for (uint32_t sb = 0; sb < du; sb += 32) inrow |= __any_sync(FULL, sb + lane < du && row[sb + lane] == cand);
+          if (!inrow) chosen = cand;
+        }
+        __syncwarp();
+        if (lane == 0) row[s] = chosen;
+        __syncwarp();
       }
-      const uint32_t np = min(a.g.deg[p], R);
-      uint32_t chosen = kInvalid;
-      for (uint32_t tt = 0; tt < np && chosen == kInvalid; ++tt) {
-        const uint32_t cand = a.g.adj[(size_t)p * R + (rank + tt) % np];
-        if (bit_test(a.delmap, cand) || cand == u) continue;
-        bool inrow = false;
-        for (uint32_t sb = 0; sb < du; sb += 32) inrow |= __any_sync(FULL, sb + lane < du && row[sb + lane] == cand);
-        if (!inrow) chosen = cand;
-      }
-      __syncwarp();
-      if (lane == 0) row[s] = chosen;
-      __syncwarp();
     }
     // stable compaction of the surviving slots
-    uint32_t w = 0;
+    uint32_t wr = 0;
     for (uint32_t sb = 0; sb < R; sb += 32) {
       const uint32_t s = sb + lane;
       const uint32_t v = s < du ? row[s] : kInvalid;
       const bool ok = v != kInvalid;
       const unsigned bal = __ballot_sync(FULL, ok);
-      if (ok) a.g.adj[(size_t)u * R + w + __popc(bal & ((1u << lane) - 1u))] = v;
-      w += __popc(bal);
+      if (ok) a.g.adj[(size_t)u * R + wr + __popc(bal & ((1u << lane) - 1u))] = v;
+      wr += __popc(bal);
     }
-    for (uint32_t s = w + lane; s < R; s += 32) a.g.adj[(size_t)u * R + s] = kInvalid;
+    for (uint32_t s = wr + lane; s < R; s += 32) a.g.adj[(size_t)u * R + s] = kInvalid;
     if (lane == 0) {
-      a.g.deg[u] = w;
+      a.g.deg[u] = wr;
       a.flag[u] = 0;
       ++ndone;
     }
@@ -942,6 +1020,16 @@ cudaError_t launch_fixed_delete(const FixedDeleteArgs& a, uint64_t total_in, cud
     uint64_t blocks = (total_in + 255) / 256;
     if (blocks > (uint64_t)sm_count() * 32u) blocks = (uint64_t)sm_count() * 32u;
     fixed_delete_mark_kernel<<<(unsigned)blocks, 256, 0, s>>>(a, total_in);
+    count_launches(1);
+  }
+  if (total_in > kRankLinear) {  // otherwise no row is long
+    auto kern = fixed_delete_sort_rows_kernel;
+    static SmemOptIn optin{};
+    cudaError_t e = allow_full_dynamic_smem((const void*)kern, &optin);
+    if (e != cudaSuccess) return e;
+    uint64_t blocks = (a.n + 1023) / 1024;
+    if (blocks > (uint64_t)sm_count()) blocks = (uint64_t)sm_count();
+    kern<<<(unsigned)blocks, 1024, (kSortRowSmem + 1024 + 1) * sizeof(uint32_t), s>>>(a);
     count_launches(1);
   }
   fixed_delete_rewire_kernel<<<(unsigned)sm_count() * 8u, 128, 0, s>>>(a);

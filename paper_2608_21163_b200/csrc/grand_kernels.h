@@ -222,7 +222,7 @@ struct FixedDeleteArgs {
   GraphView g;
   const uint32_t* ids; uint64_t n;
   const uint32_t* delmap;
-  const uint32_t* off; const uint32_t* src;
+  const uint32_t* off; uint32_t* src;  // in-neighbour rows of the batch (long rows are sorted in place)
   const uint32_t* pair_off;  // n+1 prefix of in-degrees
   uint32_t* flag; uint32_t* dirty;
   DevState* state;

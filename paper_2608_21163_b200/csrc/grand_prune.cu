@@ -8,7 +8,6 @@ namespace grand {
 
 constexpr int kPruneThreads = 128;
 constexpr uint32_t kMaxCand = 1024;  // >= vmax limit
-constexpr uint32_t kSegCap = 1024;   // request segment sorted in shared memory up to this length
 constexpr uint32_t kMaxR = 128;
 
 // GrANDRobustPrune (Alg. 4) over candidate keys sorted ascending in shared memory.  The whole
@@ -474,98 +473,94 @@ cudaError_t launch_forward_prune(const PruneArgs& a, cudaStream_t s) {
   return cudaErrorInvalidValue;
 }
 
-// Sort one target's request segment by (dist, id) and return the pointer to the sorted keys
-// (shared memory copy for short segments, in place in global memory for long ones).
-__device__ __forceinline__ unsigned long long* sort_segment(unsigned long long* seg_global, uint32_t n,
-                                                            unsigned long long* seg_smem) {
-  const uint32_t tid = threadIdx.x, nthreads = blockDim.x;
-  auto sync = [] { __syncthreads(); };
-  unsigned long long* seg = seg_global;
-  if (n <= kSegCap) {
-    for (uint32_t j = tid; j < n; j += nthreads) seg_smem[j] = seg_global[j];
-    seg = seg_smem;
-  }
-  __syncthreads();
-  bitonic_sort_any(seg, n, tid, nthreads, sync);
-  return seg;
-}
-
-
 // Fixed-degree backward edges (Alg. 7): the owner of target q takes its requests in (dist, id)
 // order; a request from new node p appends while deg(q) < R, else replaces the highest-index slot
 // of N_out(q) that also occurs in N_out(p) and was not replaced earlier in this batch.
+// One warp owns one target: almost every target of a batch receives a single request, so a
+// block per target would leave three of its four warps at the barrier.  Short segments are
+// sorted in the warp's shared-memory slice, long ones in place in global memory.
+constexpr uint32_t kFixedSegWarp = 64;
 __global__ void __launch_bounds__(kPruneThreads) fixed_reverse_kernel(const FixedReverseArgs a) {
   constexpr unsigned FULL = 0xFFFFFFFFu;
-  __shared__ unsigned long long seg_smem[kSegCap];
-  __shared__ uint32_t row[kMaxR];
-  __shared__ uint32_t replaced[kMaxR];
-  const uint32_t tid = threadIdx.x;
-  const int lane = tid & 31, warp = tid >> 5;
+  constexpr int kWarps = kPruneThreads / 32;
+  __shared__ unsigned long long seg_s[kWarps][kFixedSegWarp];
+  __shared__ uint32_t row_s[kWarps][kMaxR];
+  __shared__ uint32_t prow_s[kWarps][kMaxR];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint32_t* row = row_s[warp];
+  uint32_t* prow = prow_s[warp];
+  auto wsync = [] { __syncwarp(); };
   const uint32_t R = a.g.R;
   uint32_t ndone = 0;
   const uint32_t ndirty = a.state->ndirty;
-  for (uint32_t k = blockIdx.x; k < ndirty; k += gridDim.x) {
+  const uint64_t wglobal = (uint64_t)blockIdx.x * kWarps + warp, wtotal = (uint64_t)gridDim.x * kWarps;
+  for (uint64_t k = wglobal; k < ndirty; k += wtotal) {
     const uint32_t q = a.dirty[k];
     const uint32_t cntq = a.cnt[q];
-    unsigned long long* seg = sort_segment(a.seg_keys + a.start[q], cntq, seg_smem);
-    for (uint32_t s = tid; s < R; s += blockDim.x) {
-      row[s] = a.g.adj[(size_t)q * R + s];
-      replaced[s] = 0;
+    unsigned long long* seg = a.seg_keys + a.start[q];
+    if (cntq <= kFixedSegWarp) {
+      for (uint32_t j = lane; j < cntq; j += 32) seg_s[warp][j] = seg[j];
+      seg = seg_s[warp];
     }
-    __syncthreads();
-    if (warp == 0) {
-      uint32_t dq = min(a.g.deg[q], R);
-      unsigned long long prev = kKeyMax;
-      for (uint32_t j = 0; j < cntq; ++j) {
-        const unsigned long long kk = seg[j];
-        if (kk == prev) continue;
-        prev = kk;
-        const uint32_t p = key_id(kk);
-        // already linked?
-        bool present = false;
-        for (uint32_t sb = 0; sb < dq; sb += 32) {
-          const uint32_t s = sb + lane;
-          present |= __any_sync(FULL, s < dq && row[s] == p);
-        }
-        if (present) continue;
-        if (dq < R) {
-          if (lane == 0) row[dq] = p;
-          ++dq;
-          __syncwarp();
-          continue;
-        }
-        const uint32_t* prow = a.fwd_rows + (size_t)a.slot_of[p] * R;
-        int pick = -1;
-        for (uint32_t sb = 0; sb < dq; sb += 32) {
-          const uint32_t s = sb + lane;
-          bool hit = false;
-          if (s < dq && !replaced[s]) {
-            const uint32_t x = row[s];
-            for (uint32_t y = 0; y < R; ++y) hit |= prow[y] == x;   // INVALID padding never equals a live id
-          }
-          const unsigned bal = __ballot_sync(FULL, hit);
-          if (bal) pick = (int)sb + 31 - __clz(bal);
-        }
-        if (pick >= 0) {
-          if (lane == 0) {
-            row[pick] = p;
-            replaced[pick] = 1;
-          }
-          __syncwarp();
-        }
+    for (uint32_t s = lane; s < R; s += 32) row[s] = a.g.adj[(size_t)q * R + s];
+    __syncwarp();
+    bitonic_sort_any(seg, cntq, (uint32_t)lane, 32u, wsync);
+    uint32_t repl = 0;  // lane w: word w of the set of slots replaced in this batch
+    uint32_t nrepl = 0;
+    uint32_t dq = min(a.g.deg[q], R);
+    unsigned long long prev = kKeyMax;
+    for (uint32_t j = 0; j < cntq; ++j) {
+      if (nrepl == R) break;  // every slot already replaced once: no later request can change the row
+      const unsigned long long kk = seg[j];
+      if (kk == prev) continue;
+      prev = kk;
+      const uint32_t p = key_id(kk);
+      // already linked?
+      bool present = false;
+      for (uint32_t sb = 0; sb < dq; sb += 32) {
+        const uint32_t s = sb + lane;
+        present |= __any_sync(FULL, s < dq && row[s] == p);
       }
-      for (uint32_t s = lane; s < R; s += 32) a.g.adj[(size_t)q * R + s] = s < dq ? row[s] : kInvalid;
-      if (lane == 0) {
-        a.g.deg[q] = dq;
-        a.cnt[q] = 0;
-        a.fill[q] = 0;
-        a.flag[q] = 0;
-        ++ndone;
+      if (present) continue;
+      if (dq < R) {
+        if (lane == 0) row[dq] = p;
+        ++dq;
+        __syncwarp();
+        continue;
       }
+      const uint32_t* pg = a.fwd_rows + (size_t)a.slot_of[p] * R;
+      for (uint32_t y = lane; y < R; y += 32) prow[y] = pg[y];
+      __syncwarp();
+      int pick = -1;
+      for (uint32_t sb = 0; sb < dq; sb += 32) {
+        const uint32_t s = sb + lane;
+        const uint32_t rw = __shfl_sync(FULL, repl, sb >> 5);
+        bool hit = false;
+        if (s < dq && !((rw >> lane) & 1u)) {
+          const uint32_t x = row[s];
+          for (uint32_t y = 0; y < R; ++y) hit |= prow[y] == x;   // INVALID padding never equals a live id
+        }
+        const unsigned bal = __ballot_sync(FULL, hit);
+        if (bal) pick = (int)sb + 31 - __clz(bal);
+      }
+      if (pick >= 0) {
+        if (lane == 0) row[pick] = p;
+        if (lane == (pick >> 5)) repl |= 1u << (pick & 31);
+        ++nrepl;
+      }
+      __syncwarp();
     }
-    __syncthreads();
+    for (uint32_t s = lane; s < R; s += 32) a.g.adj[(size_t)q * R + s] = s < dq ? row[s] : kInvalid;
+    if (lane == 0) {
+      a.g.deg[q] = dq;
+      a.cnt[q] = 0;
+      a.fill[q] = 0;
+      a.flag[q] = 0;
+      ++ndone;
+    }
+    __syncwarp();
   }
-  if (tid == 0 && ndone) atomicAdd(&a.state->counters[CTR_DIRTY], (unsigned long long)ndone);
+  if (lane == 0 && ndone) atomicAdd(&a.state->counters[CTR_DIRTY], (unsigned long long)ndone);
 }
 
 cudaError_t launch_fixed_reverse(const FixedReverseArgs& a, cudaStream_t s) {

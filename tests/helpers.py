@@ -14,6 +14,7 @@ def oracle_opts(opts):
     if "visited_set_delete" in o:
         o["approx_delete"] = o.pop("visited_set_delete")
     o.pop("snapshot_search", None)     # a property of the library's memory management, not of the method
+    o.pop("max_delete_edges", None)    # workspace sizing of the library
     return o
 
 

@@ -318,6 +318,43 @@ def test_fixed_degree_mode_bit_exact_on_bytes():
     check_search(o, g, wl, cfg2)
 
 
+def test_fixed_degree_delete_of_hubs_bit_exact():
+    """Alg. 8 on a graph whose deleted nodes have very long in-neighbour rows: the round-robin
+    offset (rank of u among the in-neighbours) is then taken from a sorted row, in shared memory
+    (node 1: a few thousand in-neighbours) or in place in global memory (node 0: more than 49,152)."""
+    torch = torch_()
+    n, R, dim = 60000, 6, 8
+    rng = np.random.default_rng(11)
+    vecs = synth.uniform_u8(9, "hubgraph", 0, n, dim)
+    adj = np.full((n, R), INV, np.uint32)
+    adj[2:, 0] = 0                                           # everyone names hub 0 ...
+    some = rng.permutation(np.arange(2, n))[:3000]
+    adj[some, 1] = 1                                         # ... 3000 nodes name hub 1 ...
+    for s in range(2, R):                                    # ... and the rest is a seeded random graph
+        cand = rng.integers(2, n, size=n).astype(np.uint32)
+        adj[:, s] = cand
+    adj[some[:10], 2] = 40                                   # a short row as well
+    # rows must not name a node twice, nor the node itself: repair by blanking, then pack to the front
+    for s in range(1, R):
+        dup = np.zeros(n, bool)
+        for t in range(s):
+            dup |= adj[:, s] == adj[:, t]
+        dup |= adj[:, s] == np.arange(n)
+        adj[dup, s] = INV
+    order = np.argsort(adj == INV, axis=1, kind="stable")
+    adj = np.take_along_axis(adj, order, axis=1)
+    deg = (adj != INV).sum(1).astype(np.uint32)
+    live = go.pack_bitmap(np.ones(n, bool))
+    cfg = dict(dim=dim, dtype=go.U8, metric=go.L2, R=R, L=16, alpha=1.2, mode=go.FIXED_DEGREE, max_build_batch=64, ins=1, dele=64)
+    o, g = make_pair(cfg, n, max_delete_edges=n * R)
+    o.import_graph(adj, deg, live, 5, vecs)
+    g.import_graph(torch.from_numpy(adj), torch.from_numpy(deg), torch.from_numpy(live), 5, torch.from_numpy(vecs))
+    assert_same_graph(o, g, "imported")
+    ids = np.array([0, 1, 40, 41, 77], np.uint32)
+    o.delete_batch(ids); g.delete_batch(torch.from_numpy(ids))
+    assert_same_graph(o, g, "hubs deleted")
+
+
 # ------------------------------------------------------------------ fp32 streams: tolerance + recall
 # Sizes: the largest shrinks whose oracle build finishes in about a minute on the test box's host cores
 # (Deep-shaped 100,000 points, GIST-shaped 30,000, embedding-shaped 165,000).
