@@ -41,7 +41,7 @@ from paper_2608_21163_b200 import synth  # noqa: E402
 METRIC = "update_vectors_per_sec"
 UNIT = "vectors/s"
 WORKLOAD = "deep_f32_d96"
-PER_CONFIG = ["sift_u8_d128", "gist_f32_d960", "embed_f32_d768_ip"]
+PER_CONFIG = ["sift_u8_d128", "gist_f32_d960", "embed_f32_d768_ip", "deep_f32_d96_isotropic"]
 SWEEP_L = (10, 16, 24, 32, 48, 64, 96, 128, 192, 256, 384, 512)
 # DRAM bytes of one beam-search launch divided by the launch's algorithmic bytes, from one-pass ncu captures
 # (dram__bytes_read.sum + dram__bytes_write.sum); each ratio is valid for its workload at the named scale only.
@@ -508,6 +508,7 @@ def run_workload(args, torch, gb, dev, dist, rank, world, name, scale, K, W, Kp,
            "config": {"workload": name, "scale": scale, "built_on": cfg["build"], "dim": cfg["dim"], "R": cfg["R"],
                       "L": cfg["L"], "alpha": cfg["alpha"], "mode": "fixed-degree" if cfg["mode"] else "vamana",
                       "metric": "ip" if cfg["metric"] else "l2",
+                      "generator": {"name": cfg["gen"], **cfg.get("gen_args", {})},
                       "step": f"insert {cfg['ins']} + delete {cfg['dele']} + search {cfg['nq']} (k=10)",
                       "l2": "index (vectors + adjacency) larger than L2, and a 256 MiB flush between steps",
                       "delete": "visited-set (Alg. 6 as printed)" if args.visited_set_delete else "exact in-neighbours",

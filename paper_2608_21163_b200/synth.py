@@ -118,6 +118,40 @@ def aniso_unit_f32(seed, stream, start, n, dim):
     return _rowwise(gen, start, n, dim, np.float32)
 
 
+def _manifold(seed, stream, start, n, dim, latent, n_centres, spread, noise):
+    """Rows near a `latent`-dimensional linear image of a Gaussian mixture, plus isotropic noise:
+    descriptor and embedding sets have an intrinsic dimension far below their coordinate count,
+    and it is that, not the coordinate count, which decides how a proximity graph behaves.
+    The linear map and the mixture centres depend on (seed, dim, latent) only, so base vectors
+    and queries come from the same distribution.  Sums run in a fixed order (no BLAS)."""
+    tag = f"manifold/{dim}/{latent}"
+    W = _normal(seed, tag + "/map", 0, latent, dim) / np.sqrt(float(latent))
+    C = _normal(seed, tag + "/centres", 0, n_centres, latent)
+    which = (hash_u64(seed, stream + "/centre", np.arange(start, start + n, dtype=np.uint64)) % np.uint64(n_centres)).astype(np.int64)
+    z = C[which] + spread * _normal(seed, stream + "/latent", start, n, latent)
+    x = noise * _normal(seed, stream, start, n, dim)
+    for k in range(latent):
+        x += z[:, k:k + 1] * W[k][None, :]
+    return x
+
+
+def manifold_unit_f32(seed, stream, start, n, dim, latent=32, spread=1.0, noise=0.5, n_centres=4096):
+    """Deep- and embedding-shaped floats: a `latent`-dimensional mixture mapped into `dim`
+    coordinates, isotropic noise on top, unit-normalised."""
+    def gen(s, m):
+        x = _manifold(seed, stream, s, m, dim, latent, n_centres, spread, noise)
+        x /= np.linalg.norm(x, axis=1, keepdims=True)
+        return x.astype(np.float32)
+
+    return _rowwise(gen, start, n, dim, np.float32)
+
+
+def manifold_abs_f32(seed, stream, start, n, dim, latent=48, spread=1.0, noise=0.2, n_centres=4096, scale=0.1):
+    """GIST-shaped floats: non-negative coordinates, |mixture image + noise| * scale."""
+    return _rowwise(lambda s, m: (np.abs(_manifold(seed, stream, s, m, dim, latent, n_centres, spread, noise)) * scale).astype(np.float32),
+                    start, n, dim, np.float32)
+
+
 def choose_ids(seed, stream, population, k):
     """k ids drawn uniformly without replacement from `population` (a uint32 array): the k ids with
     the smallest hash, returned in hash order."""
@@ -133,6 +167,8 @@ GENERATORS = {
     "gaussian_unit_f32": gaussian_unit_f32,
     "halfnormal_f32": halfnormal_f32,
     "aniso_unit_f32": aniso_unit_f32,
+    "manifold_unit_f32": manifold_unit_f32,
+    "manifold_abs_f32": manifold_abs_f32,
 }
 
 # dtype / metric / mode codes match include/grand.h
@@ -140,7 +176,7 @@ U8, I8, F32 = 0, 1, 2
 L2, IP = 0, 1
 VAMANA, FIXED_DEGREE = 0, 1
 
-# The five workload shapes.  n = vectors generated, build = size of the initial index, rounds of
+# The workload shapes.  n = vectors generated, build = size of the initial index, rounds of
 # (insert, delete) batch sizes, nq queries.  `scale` shrinks n/build/batches/queries together for
 # parity tests and CPU timing.
 CONFIGS = {
@@ -150,16 +186,24 @@ CONFIGS = {
     "sift_u8_d128": dict(gen="mixture_u8", dim=128, dtype=U8, metric=L2, mode=VAMANA, R=64, L=128, alpha=1.2,
                          n=1_000_000, build=900_000, first_batch=1_000, max_build_batch=10_000,
                          rounds=10, ins=10_000, dele=10_000, nq=10_000, reuse_ids=False),
-    "deep_f32_d96": dict(gen="gaussian_unit_f32", dim=96, dtype=F32, metric=L2, mode=VAMANA, R=64, L=128, alpha=1.2,
+    "deep_f32_d96": dict(gen="manifold_unit_f32", gen_args=dict(latent=32, spread=1.0, noise=0.5),
+                         dim=96, dtype=F32, metric=L2, mode=VAMANA, R=64, L=128, alpha=1.2,
                          n=10_000_000, build=8_000_000, first_batch=1_000, max_build_batch=100_000,
                          rounds=20, ins=100_000, dele=100_000, nq=10_000, reuse_ids=False, delete_oldest=True),
-    "gist_f32_d960": dict(gen="halfnormal_f32", dim=960, dtype=F32, metric=L2, mode=VAMANA, R=64, L=128, alpha=1.2,
+    "gist_f32_d960": dict(gen="manifold_abs_f32", gen_args=dict(latent=48, spread=1.0, noise=0.2),
+                          dim=960, dtype=F32, metric=L2, mode=VAMANA, R=64, L=128, alpha=1.2,
                           n=1_200_000, build=1_000_000, first_batch=1_000, max_build_batch=20_000,
                           rounds=10, ins=20_000, dele=50_000, nq=1_000, reuse_ids=True, delete_first=True),
-    "embed_f32_d768_ip": dict(gen="aniso_unit_f32", dim=768, dtype=F32, metric=IP, mode=FIXED_DEGREE, R=64, L=128,
+    "embed_f32_d768_ip": dict(gen="manifold_unit_f32", gen_args=dict(latent=48, spread=1.0, noise=0.3),
+                              dim=768, dtype=F32, metric=IP, mode=FIXED_DEGREE, R=64, L=128,
                               alpha=1.2, n=5_500_000, build=5_000_000, first_batch=1_000, max_build_batch=50_000,
                               rounds=10, ins=50_000, dele=50_000, nq=10_000, reuse_ids=False),
 }
+# Stress case: the Deep-shaped sizes on isotropic Gaussian directions, whose intrinsic dimension
+# equals the coordinate count.  No descriptor set looks like this (a proximity graph barely helps:
+# recall@10 stays near 0.1 at L = 128), but every search expands into rows it has never seen and
+# every reverse edge forces a full prune, which makes it the heaviest load per inserted vector.
+CONFIGS["deep_f32_d96_isotropic"] = dict(CONFIGS["deep_f32_d96"], gen="gaussian_unit_f32", gen_args={})
 
 
 def scaled(cfg, factor):
@@ -190,12 +234,13 @@ class Workload:
     def __init__(self, cfg, seed=0):
         self.cfg, self.seed = cfg, seed
         self.gen = GENERATORS[cfg["gen"]]
+        self.gen_args = cfg.get("gen_args", {})
 
     def vectors(self, start, n):
-        return self.gen(self.seed, "base", start, n, self.cfg["dim"])
+        return self.gen(self.seed, "base", start, n, self.cfg["dim"], **self.gen_args)
 
     def queries(self):
-        return self.gen(self.seed, "query", 0, self.cfg["nq"], self.cfg["dim"])
+        return self.gen(self.seed, "query", 0, self.cfg["nq"], self.cfg["dim"], **self.gen_args)
 
     def capacity(self):
         c = self.cfg
