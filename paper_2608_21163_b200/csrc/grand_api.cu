@@ -738,6 +738,7 @@ int grand_delete_batch(grand_index* idx, const uint32_t* ids, uint64_t n, grand_
                          "delete batch touches " + std::to_string(total_in) + " in-neighbour entries; the workspace holds " +
                              std::to_string(idx->max_delete_edges) + " (option max_delete_edges)");
   d.req_tgt = (uint32_t*)idx->req_tgt.p; d.req_key = (unsigned long long*)idx->req_key.p; d.dirty = (uint32_t*)idx->dirty.p;
+  d.unit_owner = (uint32_t*)idx->seg_keys.p;  // the grouped-request buffer is idle until the picks have been written
   if (fixed) {
     PhaseTimer pt(idx, s, PH_REBUILD);
     FixedDeleteArgs f{};

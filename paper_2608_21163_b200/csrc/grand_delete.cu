@@ -771,12 +771,198 @@ __global__ void __launch_bounds__(kTileWarps * 32) delete_picks_tile_kernel(cons
   if (nrows) atomicAdd(&a.state->counters[CTR_PK_BYTES], nrows * row_bytes);
 }
 
-// Which pick kernel serves this index: 3 = register tiles (fp32 rows up to 384 bytes, c <= 4), 2 = tensor-core tiles
+// unit_owner[u] = the batch member whose rows unit u covers (largest i with unit_off[i] <= u)
+__global__ void delete_unit_owner_kernel(const DeleteArgs a) {
+  const uint32_t nunits = a.unit_off[a.n];
+  for (uint32_t u = blockIdx.x * blockDim.x + threadIdx.x; u < nunits; u += gridDim.x * blockDim.x) {
+    uint32_t lo = 0, hi = (uint32_t)a.n;
+    while (hi - lo > 1) {
+      const uint32_t mid = (lo + hi) >> 1;
+      if (a.unit_off[mid] <= u) lo = mid; else hi = mid;
+    }
+    a.unit_owner[u] = lo;
+  }
+}
+
+// ---- register-tiled variant for wide fp32 rows (teams of 32 lanes: a warp is one team).  Neither the candidate
+// rows nor a useful number of x rows fit shared memory at 2 to 4 KB a row, and a team per pair re-reads a candidate
+// row from L2 for every pair.  Here a warp owns a tile of 8 x rows by 8 candidates: lane t walks its chunks t, t + 32,
+// ... of all sixteen rows (coalesced 512-byte slices straight from L2) and carries 64 partial sums, so a row slice is
+// loaded once per eight pairs.  The 64 per-lane partials then fold across the lanes in the order a team uses (offsets
+// 16, 8, 4, 2, 1): at each step a lane keeps the half of the sums that its bit selects and trades the other half, which
+// gives every lane the same bits the butterfly gives it, for two of the 64 pairs, in 62 shuffles instead of 320.
+// The c smallest keys per x row are kept per lane and merged over the four lanes that share a row.
+constexpr uint32_t kWideRows = 8;
+constexpr int kWideCands = 8;
+template <int CPL>
+__global__ void __launch_bounds__(kPickWarps * 32, 3) delete_picks_wide_kernel(const DeleteArgs a, const uint64_t total_in) {
+  constexpr unsigned FULL = 0xFFFFFFFFu;
+  constexpr int XT = (int)kWideRows, CT = kWideCands;
+  __shared__ uint32_t xid_s[kPickWarps][XT];
+  __shared__ unsigned long long ck_s[kPickWarps][kMaxKRepair];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const uint32_t R = a.g.R, c = a.c, kr = a.k_repair;
+  const uint32_t row_bytes = a.lay.row_bytes, nchunk = a.lay.nchunk;
+  const uint32_t nunits = a.unit_off[a.n];
+  unsigned long long npair = 0, nrows = 0;
+  // Neighbouring warps take neighbouring units, i.e. tiles of the same deleted node: its candidate rows are then in
+  // use by many warps at once and stay in L2 (a contiguous run of units per warp was measured: every warp then
+  // works on another node, the candidate rows of all of them exceed L2, and the kernel is 1.4x slower).  The owner
+  // of each unit comes from a table written by delete_unit_owner_kernel: a binary search over the prefix here is
+  // a chain of dependent loads half as long as a unit's arithmetic.
+  for (uint32_t unit = blockIdx.x * kPickWarps + warp; unit < nunits; unit += gridDim.x * kPickWarps) {
+    const uint32_t i = a.unit_owner[unit];
+    const uint32_t p = a.ids[i];
+    const uint32_t nin = a.pair_off[i + 1] - a.pair_off[i];
+    const uint32_t q0 = (unit - a.unit_off[i]) * kWideRows, q1 = min(nin + R, q0 + kWideRows);
+    const uint32_t M = q1 - q0, nc = min(a.Ci_n[i], kr);
+    __syncwarp();  // the previous unit's readers are done with the warp's lists
+    if (lane < XT) {
+      const uint32_t q = q0 + lane;
+      uint32_t x = kInvalid;
+      if ((uint32_t)lane < M) {
+        if (q < nin) {
+          x = a.src[in_base(a, i) + q];
+        } else if (q - nin < a.g.deg[p]) {
+          x = a.g.adj[(size_t)p * R + (q - nin)];
+        }
+        if (x != kInvalid && (bit_test(a.delmap, x) || (a.livemap && !bit_test(a.livemap, x)))) x = kInvalid;
+      }
+      xid_s[warp][lane] = x;
+    }
+    const uint32_t ncp = (nc + CT - 1) / CT * CT;
+    for (uint32_t j = lane; j < ncp; j += 32) ck_s[warp][j] = j < nc ? a.Ci[(size_t)i * kr + j] : kKeyMax;
+    __syncwarp();
+    // (row ids rather than pointers are carried: 16 registers instead of 32, and the address is one multiply-add)
+    uint32_t xi[XT];
+#pragma unroll
+    for (int h = 0; h < XT; ++h) xi[h] = xid_s[warp][h];
+    const int myrow = lane >> 2, cg = lane & 3;
+    const uint32_t myx = xid_s[warp][myrow];
+    unsigned long long best[kTileMaxC];
+#pragma unroll
+    for (int r = 0; r < kTileMaxC; ++r) best[r] = kKeyMax;
+    const uint4 zero4 = make_uint4(0, 0, 0, 0);
+    for (uint32_t cb = 0; cb < nc; cb += CT) {
+      float acc[XT * CT];
+#pragma unroll
+      for (int e = 0; e < XT * CT; ++e) acc[e] = 0.0f;
+      uint32_t yi[CT];
+#pragma unroll
+      for (int j = 0; j < CT; ++j) {
+        const unsigned long long kc = ck_s[warp][cb + j];
+        yi[j] = kc != kKeyMax ? key_id(kc) : kInvalid;
+      }
+#pragma unroll 1
+      for (int cc = 0; cc < CPL; ++cc) {
+        const uint32_t ch = (uint32_t)lane + 32u * (uint32_t)cc;
+        const bool inb = ch < nchunk;
+        // all sixteen slices are requested before the first is used: one round trip to L2 per step, not nine
+        uint4 xv[XT], yv[CT];
+#pragma unroll
+        for (int h = 0; h < XT; ++h)
+          xv[h] = inb && xi[h] != kInvalid ? __ldg(reinterpret_cast<const uint4*>(a.g.store + (size_t)xi[h] * row_bytes) + ch) : zero4;
+#pragma unroll
+        for (int j = 0; j < CT; ++j)
+          yv[j] = inb && yi[j] != kInvalid ? __ldg(reinterpret_cast<const uint4*>(a.g.store + (size_t)yi[j] * row_bytes) + ch) : zero4;
+#pragma unroll
+        for (int j = 0; j < CT; ++j)
+#pragma unroll
+          for (int h = 0; h < XT; ++h) acc_chunk<float, kMetricL2>(xv[h], yv[j], acc[h * CT + j]);
+      }
+      // ---- fold over the lanes; afterwards this lane holds the sums of pairs 2 * lane and 2 * lane + 1
+      //      (pair e = row * 8 + candidate: row lane / 4, candidates 2 * (lane % 4) and + 1)
+      float r32[32], r16[16], r8[8], r4[4], r2[2];
+      {
+        const bool up = lane & 16;
+#pragma unroll
+        for (int k = 0; k < 32; ++k) r32[k] = (up ? acc[k + 32] : acc[k]) + __shfl_xor_sync(FULL, up ? acc[k] : acc[k + 32], 16);
+      }
+      {
+        const bool up = lane & 8;
+#pragma unroll
+        for (int k = 0; k < 16; ++k) r16[k] = (up ? r32[k + 16] : r32[k]) + __shfl_xor_sync(FULL, up ? r32[k] : r32[k + 16], 8);
+      }
+      {
+        const bool up = lane & 4;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) r8[k] = (up ? r16[k + 8] : r16[k]) + __shfl_xor_sync(FULL, up ? r16[k] : r16[k + 8], 4);
+      }
+      {
+        const bool up = lane & 2;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) r4[k] = (up ? r8[k + 4] : r8[k]) + __shfl_xor_sync(FULL, up ? r8[k] : r8[k + 4], 2);
+      }
+      {
+        const bool up = lane & 1;
+#pragma unroll
+        for (int k = 0; k < 2; ++k) r2[k] = (up ? r4[k + 2] : r4[k]) + __shfl_xor_sync(FULL, up ? r4[k] : r4[k + 2], 1);
+      }
+#pragma unroll
+      for (int k = 0; k < 2; ++k) {
+        const unsigned long long kc = ck_s[warp][cb + 2 * cg + k];
+        const uint32_t y = key_id(kc);
+        unsigned long long key = (kc != kKeyMax && y != myx) ? make_key(r2[k], y) : kKeyMax;
+#pragma unroll
+        for (int r = 0; r < kTileMaxC; ++r) {
+          if ((uint32_t)r < c && key < best[r]) {
+            const unsigned long long tmp = best[r];
+            best[r] = key;
+            key = tmp;
+          }
+        }
+      }
+    }
+    // ---- the four lanes that share a row merge their heads: round r takes the smallest head, its owner pops
+    {
+      const uint32_t r = (uint32_t)myrow, x = myx;
+      const uint32_t q = q0 + r;
+      const bool is_in = q < nin;
+      const uint64_t rbase = is_in ? ((uint64_t)a.pair_off[i] + q) * c : (total_in + (uint64_t)i * R + (q - nin)) * c;
+      for (uint32_t round = 0; round < c; ++round) {
+        unsigned long long m = best[0];
+        m = min(m, __shfl_xor_sync(FULL, m, 1));
+        m = min(m, __shfl_xor_sync(FULL, m, 2));
+        if (m != kKeyMax && best[0] == m) {  // keys are distinct (one id per candidate): exactly one owner
+#pragma unroll
+          for (int rr = 0; rr + 1 < kTileMaxC; ++rr) best[rr] = best[rr + 1];
+          best[kTileMaxC - 1] = kKeyMax;
+        }
+        if (cg == 0 && r < M) {
+          if (x == kInvalid || m == kKeyMax) {
+            a.req_tgt[rbase + round] = kInvalid;
+          } else if (is_in) {
+            a.req_tgt[rbase + round] = x;
+            a.req_key[rbase + round] = m;
+          } else {
+            a.req_tgt[rbase + round] = key_id(m);
+            a.req_key[rbase + round] = (m & 0xFFFFFFFF00000000ull) | x;
+          }
+        }
+      }
+      if (cg == 0 && r < M && x != kInvalid) {
+        npair += nc;
+        ++nrows;  // x's row, fetched once per pair
+      }
+    }
+  }
+  if (npair) {
+    atomicAdd(&a.state->counters[CTR_PAIR], npair);
+    atomicAdd(&a.state->counters[CTR_PK_PAIRS], npair);
+  }
+  if (nrows) atomicAdd(&a.state->counters[CTR_PK_BYTES], nrows * row_bytes);
+}
+
+// Which pick kernel serves this index: 4 = warp tiles straight from L2 (fp32 rows above 512 bytes, c <= 4),
+// 3 = register tiles (fp32 rows up to 384 bytes, c <= 4), 2 = tensor-core tiles
 // (integer rows up to 256 bytes, k_repair <= 56), 1 = candidate rows staged in shared memory, 0 = rows straight from L2.
 template <typename T>
 static int picks_variant(const DeleteArgs& a) {
 #ifndef GRAND_NO_TILE_PICKS
   if (sizeof(T) == 4 && a.lay.G <= 4 && a.c <= (uint32_t)kTileMaxC && a.lay.metric == kMetricL2) return 3;
+#endif
+#ifndef GRAND_NO_WIDE_PICKS
+  if (sizeof(T) == 4 && a.lay.G == 32 && a.c <= (uint32_t)kTileMaxC && a.k_repair <= kMaxKRepair && a.lay.metric == kMetricL2) return 4;
 #endif
   if (sizeof(T) == 1 && a.k_repair <= (uint32_t)kMmaNTiles * 8u && a.lay.row_bytes <= 256u) return 2;
   const size_t stage = (size_t)a.k_repair * ((a.lay.nchunk | 1u) * 16u);
@@ -797,9 +983,13 @@ static cudaError_t launch_delete_picks_prepare_t(const DeleteArgs& a, uint64_t t
   if (variant == 0) return cudaGetLastError();
   const uint64_t cap16 = (uint64_t)sm_count() * 16u;
   const unsigned ub = (unsigned)((a.n + 256) / 256 > cap16 ? cap16 : (a.n + 256) / 256);
-  delete_units_kernel<<<ub, 256, 0, s>>>(a, variant == 3 ? kTileUnitPairs : variant == 2 ? kMmaUnitPairs : kUnitPairs);
+  delete_units_kernel<<<ub, 256, 0, s>>>(a, variant == 4 ? kWideRows : variant == 3 ? kTileUnitPairs : variant == 2 ? kMmaUnitPairs : kUnitPairs);
   count_launches(1);
-  return launch_exclusive_scan(a.in_cnt, a.unit_off, a.n + 1, a.scan_tmp, s);
+  cudaError_t e = launch_exclusive_scan(a.in_cnt, a.unit_off, a.n + 1, a.scan_tmp, s);
+  if (e != cudaSuccess || variant != 4) return e;
+  delete_unit_owner_kernel<<<(unsigned)sm_count() * 8u, 256, 0, s>>>(a);
+  count_launches(1);
+  return cudaGetLastError();
 }
 
 template <typename T, int METRIC, int G, int CPL>
@@ -832,6 +1022,15 @@ static cudaError_t launch_delete_picks_t(const DeleteArgs& a, uint64_t total_in,
       uint64_t blocks = (total + kTileUnitPairs - 1) / kTileUnitPairs + a.n;  // upper bound on the number of units
       if (blocks > sms * 8u) blocks = sms * 8u;
       kern<<<(unsigned)blocks, kTileWarps * 32, smem, s>>>(a, total_in);
+      count_launches(1);
+      return cudaGetLastError();
+    }
+  }
+  if constexpr (sizeof(T) == 4 && G == 32) {
+    if (variant == 4) {
+      uint64_t blocks = ((total + kWideRows - 1) / kWideRows + a.n + kPickWarps - 1) / kPickWarps;  // upper bound on the units
+      if (blocks > sms * 3u) blocks = sms * 3u;
+      delete_picks_wide_kernel<CPL><<<(unsigned)blocks, kPickWarps * 32, 0, s>>>(a, total_in);
       count_launches(1);
       return cudaGetLastError();
     }

@@ -206,6 +206,7 @@ struct DeleteArgs {
   const unsigned long long* vis; const uint32_t* vis_n; uint32_t vis_stride;  // visited lists of the per-deleted searches
   uint32_t* in_cnt; uint32_t* pair_off;       // n+1
   uint32_t* unit_off;                         // n+1: work units (chunks of pairs) per deleted node, prefix
+  uint32_t* unit_owner;                       // per unit: its batch member (wide-row picks only; at most (total_in + n*R) / 8 + n entries)
   uint32_t* scan_tmp;
   uint32_t* req_tgt; unsigned long long* req_key;   // (total_in + n*R) * c
   uint32_t* flag; uint32_t* dirty;
