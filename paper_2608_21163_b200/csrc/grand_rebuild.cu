@@ -38,11 +38,12 @@ static size_t rebuild_smem_per_warp(uint32_t R, uint32_t P) {
 
 // Resident blocks per SM the register allocation must leave room for.  On rows of at most 512 bytes the kernel waits
 // on memory with few warps to hide it (103 registers allowed only 4 blocks on 128-byte rows, 93 only 5 on 384-byte
-// rows): 7 blocks (6 for the 6-chunk layout, where 7 starts to spill) took 7% off the launch on 384-byte rows and 4%
-// on 128-byte rows; 8 spills and is slower.  Whole-warp teams keep their registers (no gain measured there).
+// rows): 7 blocks took 7% off the launch on 384-byte rows and 4% on 128-byte rows (on 384-byte rows 5 / 6 / 7 / 8
+// blocks measure 56.5 / 52.5 / 50.6 / 59.9 ms per step on the Deep-shaped stream); 8 spills and is slower.
+// Whole-warp teams keep their registers (no gain measured there).
 template <int G, int CPL>
 constexpr int rebuild_min_blocks() {
-  return G == 32 ? 1 : (CPL >= 6 ? 6 : 7);
+  return G == 32 ? 1 : 7;
 }
 
 template <typename T, int METRIC, int G, int CPL>
