@@ -504,6 +504,7 @@ static cudaError_t launch_beam_search_t(const SearchArgs& a, cudaStream_t s) {
   // short rows (teams of at most 8 lanes) with the usual parameter pairs take the unrolled instantiations
   if constexpr (G <= 8) {
     if (a.g.R == 64 && a.L == 128) return launch_beam_search_rl<T, METRIC, G, CPL, 64, 128>(a, s);
+    if (a.g.R == 64 && a.L == 32) return launch_beam_search_rl<T, METRIC, G, CPL, 64, 32>(a, s);  // query searches at a small L
     if (a.g.R == 32 && a.L == 64) return launch_beam_search_rl<T, METRIC, G, CPL, 32, 64>(a, s);
   }
   return launch_beam_search_rl<T, METRIC, G, CPL, 0, 0>(a, s);
