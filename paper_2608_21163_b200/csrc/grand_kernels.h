@@ -94,6 +94,7 @@ struct SearchArgs {
   const uint32_t* boot_ids;  // bootstrap: scan these ids (all batch-mates) instead of walking the graph
   uint32_t boot_n;
   uint32_t hash_bits;
+  uint32_t cache_ways;  // tags per bucket of the visited cache: 8 or 12 (set by the launcher)
   uint32_t* work_ctr;  // zeroed by the caller before the launch; nullptr = static striding
   uint32_t check_live; // 1: skip neighbours that are not live (rows may hold dangling edges)
   uint32_t mips;       // 1: rows are MIPS -> L2 augmented; reported distances go back to negated inner products
@@ -101,7 +102,7 @@ struct SearchArgs {
   DevState* state;
 };
 cudaError_t launch_beam_search(const SearchArgs& a, cudaStream_t s);
-size_t beam_search_smem_per_warp(uint32_t L, uint32_t R, uint32_t hash_bits);
+size_t beam_search_smem_per_warp(uint32_t L, uint32_t R, uint32_t hash_bits, uint32_t cache_ways);
 
 struct PruneArgs {
   Layout lay;
