@@ -66,7 +66,8 @@ typedef struct {
   uint32_t vmax;      /* expansion cap of update searches; default 2*L; <= 1024 */
   uint32_t mode;      /* grand_mode; default GRAND_MODE_VAMANA.  GRAND_MODE_FIXED_DEGREE needs R <= L (Alg. 7 keeps
                          the R closest entries of a search result of L entries); else GRAND_ERR_INVALID_ARG */
-  uint32_t hash_bits; /* log2 of the per-query visited cache in 4-byte words; default 10; 8..13, and 4 << hash_bits >= padded row bytes */
+  uint32_t hash_bits; /* log2 of the per-query visited cache in 4-byte words; 8..13, and 4 << hash_bits >= padded row bytes;
+                         0 = default: 10, and on rows above 512 bytes up to three times that where shared memory is left over */
   uint32_t full_transpose; /* 1: every delete batch builds the whole reverse graph; default 0: only the rows of the
                               batch's nodes (the only rows the repair reads; identical result) */
   float mips_max_norm;     /* > 0: Vamana mode accepts the IP metric on fp32 vectors through the MIPS -> L2

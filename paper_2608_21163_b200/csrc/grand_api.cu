@@ -85,6 +85,7 @@ struct Buf {
 struct grand_index {
   Layout lay;
   uint32_t R, L, P, c, k_repair, vmax, mode, hash_bits, full_transpose;
+  uint32_t auto_cache = 0;  // hash_bits was left at its default
   bool approx = false; // visited-set delete mode (Alg. 6 as printed): rows may hold dangling edges
   unsigned long long* vis_keys = nullptr;  // max_batch x vmax visited lists of the per-deleted searches (that mode only)
   uint32_t *vis_n = nullptr, *vis_in = nullptr;
@@ -282,6 +283,7 @@ SearchArgs search_args(grand_index* idx, cudaStream_t s, bool work, int slot = -
   a.g = view(idx, work);
   a.entry = idx->entry;
   a.hash_bits = idx->hash_bits;
+  a.auto_cache = idx->auto_cache;
   a.check_live = idx->approx ? 1u : 0u;
   a.mips = idx->mips ? 1u : 0u;
   a.mips_M2 = (float)idx->mips_M2;
@@ -403,6 +405,7 @@ int grand_create_ex(uint32_t dim, uint32_t dtype, uint32_t metric, uint32_t R, u
   idx->vmax = o->vmax ? o->vmax : 2 * L;
   idx->mode = o->mode;
   idx->hash_bits = o->hash_bits ? o->hash_bits : 10;
+  idx->auto_cache = o->hash_bits == 0;
   idx->full_transpose = o->full_transpose;
   idx->approx = o->visited_set_delete != 0 && o->mode == GRAND_MODE_VAMANA;
   idx->snap = o->snapshot_search != 0;

@@ -95,6 +95,7 @@ struct SearchArgs {
   uint32_t boot_n;
   uint32_t hash_bits;
   uint32_t cache_ways;  // tags per bucket of the visited cache: 8 or 12 (set by the launcher)
+  uint32_t auto_cache;  // the caller left hash_bits at its default: the launcher may enlarge the cache
   uint32_t* work_ctr;  // zeroed by the caller before the launch; nullptr = static striding
   uint32_t check_live; // 1: skip neighbours that are not live (rows may hold dangling edges)
   uint32_t mips;       // 1: rows are MIPS -> L2 augmented; reported distances go back to negated inner products

@@ -513,18 +513,27 @@ static cudaError_t launch_beam_search_rl(const SearchArgs& a0, cudaStream_t s) {
   cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, kSearchWarps * 32, smem);
   if (occ < 1) occ = 1;
   if constexpr (G == 32) {
-    // rows above 512 bytes: the kernel is bound by HBM traffic, registers limit the resident blocks to a few, and
-    // the larger buckets fit the shared memory those blocks leave over.  (Not on 384-byte rows: six resident
-    // blocks with the larger cache take 210 KB of the SM's 256 KB, what is left as L1 no longer holds the loads in
-    // flight, and the search slows from 84.7 to 112.5 ms per step although it gathers 5% fewer bytes.)
+    // Rows above 512 bytes: the kernel is bound by HBM traffic, a re-evaluated node costs a whole row of it, and
+    // registers limit the resident blocks to a few - so the visited cache takes what shared memory those blocks
+    // leave over: buckets of twelve tags, and twice the buckets when the caller left the size to the library.
+    // (Not on 384-byte rows: six resident blocks with the larger cache take 210 KB of the SM's 256 KB, what is left
+    // as L1 no longer holds the loads in flight, and the search slows from 84.7 to 112.5 ms per step although it
+    // gathers 5% fewer bytes.)
 #ifndef GRAND_NO_WAYS12
-    const size_t per_warp12 = beam_search_smem_per_warp(a.L, a.g.R, a.hash_bits, 12);
-    int occ12 = 0;
-    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ12, kern, kSearchWarps * 32, per_warp12 * kSearchWarps);
-    if (occ12 >= occ && a.g.cap <= (1ull << (a.hash_bits + 14))) {
-      a.cache_ways = 12;
-      per_warp = per_warp12;
-      smem = per_warp * kSearchWarps;
+    const uint32_t hb0 = a.hash_bits;
+    const uint32_t try_hb[4] = {hb0 + 1, hb0 + 1, hb0, hb0}, try_ways[4] = {12, 8, 12, 8};
+    for (int k = a.auto_cache ? 0 : 2; k < 3; ++k) {
+      if (try_hb[k] > 13 || a.g.cap > (1ull << (try_hb[k] + 14))) continue;  // (the tag layout must hold every id)
+      const size_t pw = beam_search_smem_per_warp(a.L, a.g.R, try_hb[k], try_ways[k]);
+      int o2 = 0;
+      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o2, kern, kSearchWarps * 32, pw * kSearchWarps);
+      if (o2 >= occ) {
+        a.hash_bits = try_hb[k];
+        a.cache_ways = try_ways[k];
+        per_warp = pw;
+        smem = per_warp * kSearchWarps;
+        break;
+      }
     }
 #endif
   }
