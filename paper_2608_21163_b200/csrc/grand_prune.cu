@@ -126,9 +126,11 @@ __global__ void __launch_bounds__(kPruneThreads) forward_prune_kernel(const Prun
   if (tid == 0 && nrows) atomicAdd(&a.state->counters[CTR_FP_BYTES], nrows * a.lay.row_bytes);
 }
 
-// The same candidate-ordered prune with one WARP per node, for rows of at most 512 bytes: such a row keeps only a
-// few lanes busy per test, the tests of one candidate are few, and a block would spend its time in barriers
-// (measured on 384-byte rows: 12.8 -> 7.6 ms per 100,000 nodes against the block-per-node kernel).
+// The same candidate-ordered prune with one WARP per node: a short row keeps only a few lanes busy per test, the
+// tests of one candidate are few, and a block would spend its time in barriers (measured on 384-byte rows:
+// 12.8 -> 7.6 ms per 100,000 nodes against the block-per-node kernel; on 3,840-byte rows, where a warp is a single
+// team, 28.7 -> 26.0 ms per 20,000 nodes with a tenth fewer tests - a block tests four members at once and the
+// first hit wastes the others).  The block-per-node kernel keeps the candidate lists longer than 256.
 constexpr uint32_t kWarpPruneCand = 256;  // candidates per node this kernel accepts (shared memory per warp)
 constexpr int kWarpPruneWarps = 4;
 
@@ -453,7 +455,7 @@ static cudaError_t launch_forward_prune_t(const PruneArgs& a, cudaStream_t s) {
       return cudaGetLastError();
     }
   }
-  if constexpr (G * CPL <= 32) {
+  {
     if (!a.fixed_mode && a.cand_stride <= kWarpPruneCand) {
       const uint64_t want = (a.n + kWarpPruneWarps - 1) / kWarpPruneWarps, most = (uint64_t)sm_count() * 16u;
       const unsigned blocks = (unsigned)(want < most ? want : most);
