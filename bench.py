@@ -456,9 +456,9 @@ def run_workload(args, torch, gb, dev, dist, rank, world, name, scale, K, W, Kp,
                              pairs=stats["picks_pair_dists"]),
         "forward_prune": roof("forward_prune_*_kernel", stats["prune_bytes"], stats["ms_prune"], stats["n_prune_launches"],
                               "one vector per candidate the prune looks at", pairs=stats["prune_pair_dists"]),
-        "reverse_graph": roof("transpose_hist/scatter_kernel", stats["n_transpose_launches"] * 2 * (cap * 4 + live_edges * 4),
+        "reverse_graph": roof("transpose_hist_pairs/scatter_pairs_kernel", stats["n_transpose_launches"] * (cap * 4 + live_edges * 4),
                               stats["ms_transpose"], stats["n_transpose_launches"],
-                              "two passes over the degrees and the live adjacency entries (scan and scatter of the batch's rows not counted)"),
+                              "one pass over the degrees and the live adjacency entries (the scan, and the list and scatter of the batch's rows, not counted)"),
     }
     tr = NCU_TRAFFIC.get((name, float(scale)))
     if tr and rooflines["beam_search"]:

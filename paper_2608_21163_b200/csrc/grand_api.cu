@@ -127,6 +127,7 @@ struct grand_index {
   uint32_t wk_stride = 0;
   unsigned long long* Ci = nullptr;
   uint32_t *Ci_n = nullptr, *in_cnt = nullptr, *pair_off = nullptr, *unit_off = nullptr, *scan_tmp = nullptr;
+  uint32_t* pair_count = nullptr;  // length of the marked-edge list of a delete batch's reverse graph
   uint8_t* mean_row = nullptr;
   // Work counters of the search launches.  Slot 0 serves the searches inside update calls (each such call ends
   // with a stream synchronisation, so its launch is over before the next one starts).  grand_search is
@@ -464,6 +465,7 @@ int grand_create_ex(uint32_t dim, uint32_t dtype, uint32_t metric, uint32_t R, u
   A(alloc_dev(idx, &idx->unit_off, mb + 1, true));
   A(alloc_dev(idx, &idx->scan_tmp, (cap + 1) / 2048 + mb / 2048 + 8, true));
   A(alloc_dev(idx, &idx->mean_row, lay.row_bytes, true));
+  A(alloc_dev(idx, &idx->pair_count, 1, true));
   if (idx->approx) {
     A(alloc_dev(idx, &idx->vis_keys, (size_t)mb * idx->vmax, false));
     A(alloc_dev(idx, &idx->vis_n, mb, true));
@@ -670,6 +672,10 @@ static int build_reverse(grand_index* idx, bool sort_rows, const uint32_t* heads
   t.indeg = (uint32_t*)indeg->p; t.off = (uint32_t*)off->p; t.fillc = (uint32_t*)fillc->p;
   t.src = (uint32_t*)src->p; t.scan_tmp = idx->scan_tmp; t.sort_rows = sort_rows; t.heads = heads;
   t.src_capacity = src->bytes / 4;
+  if (!introspection && heads && !sort_rows) {
+    // the request buffer is idle until the picks are written: it holds the batch's marked edges meanwhile
+    t.pairs = (unsigned long long*)idx->req_key.p; t.pairs_capacity = idx->req_key.bytes / 8; t.pair_count = idx->pair_count;
+  }
   CK(launch_transpose(t, s));
   return GRAND_OK;
 }

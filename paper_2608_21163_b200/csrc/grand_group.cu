@@ -198,17 +198,65 @@ __device__ __forceinline__ void for_each_marked_edge(const GraphView& g, const u
         if (bad && z[k] != 0xFFFFFFFFu && z[k] >= g.cap) *bad = 1u;
       }
 #pragma unroll
-      for (int k = 0; k < kTransposeRows; ++k)
-        if (hit[k]) f(z[k], (uint32_t)(v0 + k * wtotal));
+      for (int k = 0; k < kTransposeRows; ++k) f(hit[k], z[k], (uint32_t)(v0 + k * wtotal));  // (all lanes, converged)
     }
   }
 }
 __global__ void transpose_hist_kernel(const GraphView g, uint32_t* indeg, const uint32_t* heads, uint32_t* bad) {
-  for_each_marked_edge(g, heads, bad, [&](uint32_t z, uint32_t) { atomicAdd(&indeg[z], 1u); });
+  for_each_marked_edge(g, heads, bad, [&](bool hit, uint32_t z, uint32_t) {
+    if (hit) atomicAdd(&indeg[z], 1u);
+  });
+}
+// The same pass, which also writes the marked edges out as (head, tail) pairs: the heads of a delete batch catch a
+// percent or so of the edges, and scattering them from the list spares the second pass over the adjacency.
+// Pairs collect in a per-warp buffer and leave in runs (one bump of the list's counter per run, not per edge);
+// pairs beyond the list's capacity are dropped and still counted, like entries beyond the capacity of `src`.
+constexpr uint32_t kPairRun = 64;
+__global__ void __launch_bounds__(kThreads) transpose_hist_pairs_kernel(const GraphView g, uint32_t* indeg, const uint32_t* heads,
+                                                                        uint32_t* bad, unsigned long long* pairs,
+                                                                        const uint64_t pairs_capacity, uint32_t* pair_count) {
+  constexpr unsigned FULL = 0xFFFFFFFFu;
+  __shared__ unsigned long long buf_s[kThreads / 32][kPairRun + 32];
+  const int lane = threadIdx.x & 31;
+  unsigned long long* buf = buf_s[threadIdx.x >> 5];
+  const uint32_t lt_mask = (1u << lane) - 1u;
+  uint32_t cnt = 0;  // (uniform over the warp)
+  auto flush = [&] {
+    __syncwarp();
+    uint32_t base = 0;
+    if (lane == 0) base = atomicAdd(pair_count, cnt);
+    base = __shfl_sync(FULL, base, 0);
+    for (uint32_t j = lane; j < cnt; j += 32)
+      if ((uint64_t)base + j < pairs_capacity) pairs[(uint64_t)base + j] = buf[j];
+    __syncwarp();
+    cnt = 0;
+  };
+  for_each_marked_edge(g, heads, bad, [&](bool hit, uint32_t z, uint32_t v) {
+    const unsigned bal = __ballot_sync(FULL, hit);
+    if (!bal) return;
+    if (hit) {
+      atomicAdd(&indeg[z], 1u);
+      buf[cnt + __popc(bal & lt_mask)] = ((unsigned long long)z << 32) | v;
+    }
+    cnt += __popc(bal);
+    if (cnt >= kPairRun) flush();
+  });
+  if (cnt) flush();
+}
+__global__ void transpose_scatter_pairs_kernel(const unsigned long long* pairs, const uint64_t pairs_capacity, const uint32_t* pair_count,
+                                               const uint32_t* off, uint32_t* fillc, uint32_t* src, const uint64_t src_capacity) {
+  const uint64_t n = min((uint64_t)*pair_count, pairs_capacity);
+  for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < n; i += (uint64_t)gridDim.x * blockDim.x) {
+    const unsigned long long pr = pairs[i];
+    const uint32_t z = (uint32_t)(pr >> 32);
+    const uint64_t at = (uint64_t)off[z] + atomicAdd(&fillc[z], 1u);
+    if (at < src_capacity) src[at] = (uint32_t)pr;
+  }
 }
 __global__ void transpose_scatter_kernel(const GraphView g, const uint32_t* off, uint32_t* fillc, uint32_t* src, const uint32_t* heads,
                                          const uint64_t src_capacity) {
-  for_each_marked_edge(g, heads, nullptr, [&](uint32_t z, uint32_t v) {
+  for_each_marked_edge(g, heads, nullptr, [&](bool hit, uint32_t z, uint32_t v) {
+    if (!hit) return;
     const uint64_t at = (uint64_t)off[z] + atomicAdd(&fillc[z], 1u);
     if (at < src_capacity) src[at] = v;
   });
@@ -235,10 +283,23 @@ __global__ void __launch_bounds__(128) transpose_sort_rows_kernel(uint64_t cap, 
 cudaError_t launch_transpose(const TransposeArgs& a, cudaStream_t s) {
   const uint64_t cap = a.g.cap;
   cudaMemsetAsync(a.indeg, 0, (cap + 1) * 4, s);
-  transpose_hist_kernel<<<grid_for(cap * 32), kThreads, 0, s>>>(a.g, a.indeg, a.heads, a.bad);
+  const bool listed = a.heads && a.src && a.pairs && a.pair_count && !a.sort_rows;
+  if (listed) {
+    cudaMemsetAsync(a.pair_count, 0, 4, s);
+    transpose_hist_pairs_kernel<<<grid_for(cap * 32), kThreads, 0, s>>>(a.g, a.indeg, a.heads, a.bad, a.pairs, a.pairs_capacity, a.pair_count);
+  } else {
+    transpose_hist_kernel<<<grid_for(cap * 32), kThreads, 0, s>>>(a.g, a.indeg, a.heads, a.bad);
+  }
   count_launches(1);
   cudaError_t e = launch_exclusive_scan(a.indeg, a.off, cap + 1, a.scan_tmp, s);
   if (e != cudaSuccess) return e;
+  if (listed) {
+    cudaMemsetAsync(a.fillc, 0, cap * 4, s);
+    transpose_scatter_pairs_kernel<<<(unsigned)sm_count() * 8u, kThreads, 0, s>>>(a.pairs, a.pairs_capacity, a.pair_count, a.off, a.fillc,
+                                                                              a.src, a.src_capacity);
+    count_launches(1);
+    return cudaGetLastError();
+  }
   if (a.src) {
     cudaMemsetAsync(a.fillc, 0, cap * 4, s);
     transpose_scatter_kernel<<<grid_for(cap * 32), kThreads, 0, s>>>(a.g, a.off, a.fillc, a.src, a.heads, a.src_capacity);

@@ -189,6 +189,9 @@ struct TransposeArgs {
   const uint32_t* heads;  // optional bitmap: build only the rows of these nodes
   uint64_t src_capacity;  // entries `src` can hold; edges beyond it are dropped (the caller compares the total)
   uint32_t* bad;          // optional: set to 1 when a row names a neighbour id >= cap (such an edge is skipped)
+  // optional (with `heads`, unsorted rows): list of the marked edges as (head << 32 | tail), its capacity in pairs
+  // and a device word for its length; the rows are then scattered from the list instead of a second adjacency pass
+  unsigned long long* pairs; uint64_t pairs_capacity; uint32_t* pair_count;
 };
 cudaError_t launch_transpose(const TransposeArgs& a, cudaStream_t s);
 cudaError_t launch_exclusive_scan(const uint32_t* in, uint32_t* out, uint64_t n, uint32_t* tmp, cudaStream_t s);
