@@ -48,8 +48,8 @@ SWEEP_L = (10, 16, 24, 32, 48, 64, 96, 128, 192, 256, 384, 512)
 NCU_TRAFFIC = {
     ("deep_f32_d96", 1.0): (0.945, "profiles/beam_search_dram_deep_f32_d96_full.txt"),
     ("sift_u8_d128", 1.0): (0.379, "profiles/beam_search_dram_sift_u8_d128_full.txt"),
-    ("gist_f32_d960", 1.0): (0.655, "profiles/beam_search_dram_gist_f32_d960_full.txt"),
-    ("embed_f32_d768_ip", 1.0): (0.975, "profiles/beam_search_dram_embed_f32_d768_ip_full.txt"),
+    ("gist_f32_d960", 1.0): (0.680, "profiles/beam_search_dram_gist_f32_d960_full.txt"),
+    ("embed_f32_d768_ip", 1.0): (0.971, "profiles/beam_search_dram_embed_f32_d768_ip_full.txt"),
 }
 
 
