@@ -46,6 +46,135 @@ constexpr int rebuild_min_blocks() {
   return G == 32 ? 1 : 7;
 }
 
+// The P smallest distinct keys of a long request segment, ascending, into `best` (shared memory); returns how many.
+// Kept out of line: a rare path whose code would otherwise sit in the middle of the per-node loop.
+__device__ __forceinline__ uint32_t stream_best_keys_impl(const unsigned long long* seg, uint32_t cntu, unsigned long long* scratch,
+                                                          uint32_t P, int lane) {
+  constexpr unsigned FULL = 0xFFFFFFFFu;
+  uint32_t ns = 0;
+      for (uint32_t jb0 = 0; jb0 < cntu; jb0 += 128) {
+       unsigned long long k4[4];  // four chunks requested together: the stream is a chain of dependent steps otherwise
+#pragma unroll
+       for (int q = 0; q < 4; ++q) k4[q] = jb0 + q * 32 + lane < cntu ? seg[jb0 + q * 32 + lane] : kKeyMax;
+#pragma unroll
+       for (int q = 0; q < 4; ++q) {
+        const unsigned long long kk = k4[q];
+        const unsigned long long thr = ns == P ? scratch[P - 1] : kKeyMax;
+        unsigned bal = __ballot_sync(FULL, kk < thr);
+        while (bal) {  // (uniform)
+          const int srcl = __ffs(bal) - 1;
+          bal &= bal - 1u;
+          const unsigned long long key = ((unsigned long long)__shfl_sync(FULL, (uint32_t)(kk >> 32), srcl) << 32) |
+                                         __shfl_sync(FULL, (uint32_t)kk, srcl);
+          if (ns == P && !(key < scratch[P - 1])) continue;  // the list has tightened since the ballot
+          uint32_t pos = 0;
+          unsigned dup = 0;
+          for (uint32_t cb = 0; cb < ns; cb += 32) {
+            const uint32_t i = cb + lane;
+            const unsigned long long e = i < ns ? scratch[i] : kKeyMax;
+            pos += __popc(__ballot_sync(FULL, e < key));
+            dup |= __ballot_sync(FULL, e == key);
+          }
+          if (dup) continue;
+          const uint32_t last = min(ns, P - 1u);  // entries [pos, last) move up by one; a full list drops its last entry
+          if (last > pos) {
+            for (int ch = (int)((last - 1u) >> 5); ch >= (int)(pos >> 5); --ch) {
+              const uint32_t i = (uint32_t)ch * 32u + lane;
+              const bool mv = i >= pos && i < last;
+              const unsigned long long e = mv ? scratch[i] : 0ull;
+              __syncwarp();
+              if (mv) scratch[i + 1] = e;
+            }
+          }
+          __syncwarp();
+          if (lane == 0) scratch[pos] = key;
+          __syncwarp();
+          ns = min(ns + 1u, P);
+        }
+       }
+      }
+  return ns;
+}
+__device__ __noinline__ uint32_t stream_best_keys_ool(const unsigned long long* seg, uint32_t cntu, unsigned long long* scratch,
+                                                      uint32_t P, int lane) {
+  return stream_best_keys_impl(seg, cntu, scratch, P, lane);
+}
+// Whether the two rare paths of the rebuild sit out of line.  Out of line they shorten the per-node loop (128-byte
+// rows: rebuild 1.79 -> 1.60 ms per step, alternating runs of both builds on one GPU); the calls cost the 6-chunk
+// layout, which runs at its register bound, a few more spills (53.3 against 51.8 ms per step), so that layout keeps
+// them inline.
+template <int G, int CPL>
+constexpr bool rebuild_cold_paths_out_of_line() { return !(G == 4 && CPL == 6); }
+
+// Fallback of the prune for candidate lists without a trusted run: every test alpha * dist(c_i, c_j) <= D_u[c_j],
+// i < j, goes into a bit matrix (row i, bit j = "c_i prunes c_j"), and the sequential selection is replayed on
+// masks.  Lane w holds word w of the set of still-valid candidates; the updated word is returned.  Out of line: rare.
+template <typename T, int G, int CPL>
+__device__ __forceinline__ uint32_t prune_all_pairs_impl(const uint8_t* __restrict__ store, uint32_t row_bytes, uint32_t nchunk,
+                                                         const unsigned long long* cs, uint32_t nC, uint32_t W, uint32_t* prune, uint32_t* hasp,
+                                                         AlphaParam ap, uint32_t valid, unsigned long long& npair, int lane) {
+  using Dist = typename Elem<T>::Dist;
+  constexpr unsigned FULL = 0xFFFFFFFFu;
+  constexpr int NT = 32 / G;
+  const int t = lane % G, team = lane / G;
+  for (uint32_t w = lane; w < nC * W; w += 32) prune[w] = 0u;
+  __syncwarp();
+  uint32_t jprev = kInvalid;
+  uint4 rj[CPL];
+#pragma unroll
+  for (int c = 0; c < CPL; ++c) rj[c] = make_uint4(0, 0, 0, 0);
+  const uint32_t npairs = nC * (nC - 1) / 2;
+  for (uint32_t pb = 0; pb < npairs; pb += NT) {
+    const uint32_t p = pb + team;
+    const bool act = p < npairs;
+    uint32_t i = 0, j = 1;
+    if (act) {
+      j = (uint32_t)((1.0f + sqrtf(1.0f + 8.0f * (float)p)) * 0.5f);
+      while (j * (j - 1) / 2 > p) --j;
+      while ((j + 1) * j / 2 <= p) ++j;
+      i = p - j * (j - 1) / 2;
+    }
+    uint4 ri[CPL];
+    if (act) {
+      if (j != jprev) {
+        load_row<G, CPL>(store + (size_t)key_id(cs[j]) * row_bytes, nchunk, t, rj);
+        jprev = j;
+      }
+      load_row<G, CPL>(store + (size_t)key_id(cs[i]) * row_bytes, nchunk, t, ri);
+    } else {
+#pragma unroll
+      for (int c = 0; c < CPL; ++c) ri[c] = make_uint4(0, 0, 0, 0);
+    }
+    const Dist d = team_dist_regs<T, kMetricL2, G, CPL>(ri, rj);
+    if (act && t == 0) {
+      ++npair;
+      if (alpha_test(ap, d, key_dist<Dist>(cs[j]))) {
+        atomicOr(&prune[i * W + (j >> 5)], 1u << (j & 31));
+        atomicOr(&hasp[i >> 5], 1u << (i & 31));
+      }
+    }
+  }
+  __syncwarp();
+  // the valid set only changes when a still-valid candidate with a non-zero matrix row is reached, so only those
+  // candidates are visited, in ascending order; everything valid in between is selected
+  for (uint32_t w = 0; w < W; ++w) {
+    uint32_t hw = hasp[w];
+    while (hw) {
+      const uint32_t b = __ffs(hw) - 1;
+      hw &= hw - 1;
+      const uint32_t vw = __shfl_sync(FULL, valid, w);
+      if (((vw >> b) & 1u) && (uint32_t)lane < W) valid &= ~prune[(w * 32 + b) * W + lane];
+    }
+  }
+  return valid;
+}
+template <typename T, int G, int CPL>
+__device__ __noinline__ uint32_t prune_all_pairs_ool(const uint8_t* __restrict__ store, uint32_t row_bytes, uint32_t nchunk,
+                                                     const unsigned long long* cs, uint32_t nC, uint32_t W, uint32_t* prune, uint32_t* hasp,
+                                                     AlphaParam ap, uint32_t valid, unsigned long long& npair, int lane) {
+  return prune_all_pairs_impl<T, G, CPL>(store, row_bytes, nchunk, cs, nC, W, prune, hasp, ap, valid, npair, lane);
+}
+
 template <typename T, int METRIC, int G, int CPL>
 __global__ void __launch_bounds__(kRebuildWarps * 32, rebuild_min_blocks<G, CPL>()) rebuild_kernel(const RebuildArgs a, const uint32_t per_warp_bytes) {
   using Dist = typename Elem<T>::Dist;
@@ -74,29 +203,6 @@ __global__ void __launch_bounds__(kRebuildWarps * 32, rebuild_min_blocks<G, CPL>
   unsigned long long npair = 0, nbytes = 0;  // nbytes: what the method has to move for the rows this warp rebuilds
   uint32_t nprune = 0, ndone = 0;
   const uint32_t ndirty = a.split ? a.state->nheavy : a.state->ndirty;  // (split: the front of the work list)
-
-  // one prune test: rows of candidates i < j (sorted positions), result into the bit matrix
-  auto pair_test = [&](bool act, uint32_t i, uint32_t j, uint32_t& jprev, uint4 (&rj)[CPL]) {
-    uint4 ri[CPL];
-    if (act) {
-      if (j != jprev) {
-        load_row<G, CPL>(store + (size_t)key_id(cs[j]) * row_bytes, nchunk, t, rj);
-        jprev = j;
-      }
-      load_row<G, CPL>(store + (size_t)key_id(cs[i]) * row_bytes, nchunk, t, ri);
-    } else {
-#pragma unroll
-      for (int c = 0; c < CPL; ++c) ri[c] = make_uint4(0, 0, 0, 0);
-    }
-    const Dist d = team_dist_regs<T, kMetricL2, G, CPL>(ri, rj);
-    if (act && t == 0) {
-      ++npair;
-      if (alpha_test(ap, d, key_dist<Dist>(cs[j]))) {
-        atomicOr(&prune[i * W + (j >> 5)], 1u << (j & 31));
-        atomicOr(&hasp[i >> 5], 1u << (i & 31));
-      }
-    }
-  };
 
   // One counter serves every warp of the grid.  The ticket for the node after this one is drawn while this one
   // is processed, so the atomic's round trip is never waited for.
@@ -150,47 +256,8 @@ __global__ void __launch_bounds__(kRebuildWarps * 32, rebuild_min_blocks<G, CPL>
       // hubness), and only the P smallest distinct keys are wanted: the segment is streamed once against a sorted
       // list of the best P so far instead of being sorted.  After the first few chunks almost every key fails the
       // comparison with the list's last entry.  Same list as sort + drop repeats + cut at P.
-      for (uint32_t jb0 = 0; jb0 < cntu; jb0 += 128) {
-       unsigned long long k4[4];  // four chunks requested together: the stream is a chain of dependent steps otherwise
-#pragma unroll
-       for (int q = 0; q < 4; ++q) k4[q] = jb0 + q * 32 + lane < cntu ? seg[jb0 + q * 32 + lane] : kKeyMax;
-#pragma unroll
-       for (int q = 0; q < 4; ++q) {
-        const unsigned long long kk = k4[q];
-        const unsigned long long thr = ns == P ? scratch[P - 1] : kKeyMax;
-        unsigned bal = __ballot_sync(FULL, kk < thr);
-        while (bal) {  // (uniform)
-          const int srcl = __ffs(bal) - 1;
-          bal &= bal - 1u;
-          const unsigned long long key = ((unsigned long long)__shfl_sync(FULL, (uint32_t)(kk >> 32), srcl) << 32) |
-                                         __shfl_sync(FULL, (uint32_t)kk, srcl);
-          if (ns == P && !(key < scratch[P - 1])) continue;  // the list has tightened since the ballot
-          uint32_t pos = 0;
-          unsigned dup = 0;
-          for (uint32_t cb = 0; cb < ns; cb += 32) {
-            const uint32_t i = cb + lane;
-            const unsigned long long e = i < ns ? scratch[i] : kKeyMax;
-            pos += __popc(__ballot_sync(FULL, e < key));
-            dup |= __ballot_sync(FULL, e == key);
-          }
-          if (dup) continue;
-          const uint32_t last = min(ns, P - 1u);  // entries [pos, last) move up by one; a full list drops its last entry
-          if (last > pos) {
-            for (int ch = (int)((last - 1u) >> 5); ch >= (int)(pos >> 5); --ch) {
-              const uint32_t i = (uint32_t)ch * 32u + lane;
-              const bool mv = i >= pos && i < last;
-              const unsigned long long e = mv ? scratch[i] : 0ull;
-              __syncwarp();
-              if (mv) scratch[i + 1] = e;
-            }
-          }
-          __syncwarp();
-          if (lane == 0) scratch[pos] = key;
-          __syncwarp();
-          ns = min(ns + 1u, P);
-        }
-       }
-      }
+      if constexpr (rebuild_cold_paths_out_of_line<G, CPL>()) ns = stream_best_keys_ool(seg, cntu, scratch, P, lane);
+      else ns = stream_best_keys_impl(seg, cntu, scratch, P, lane);
     } else {
     bitonic_sort_any(seg, cntu, (uint32_t)lane, 32u, wsync);
     for (uint32_t jb = 0; jb < cntu && ns < P; jb += 32) {
@@ -428,10 +495,6 @@ __global__ void __launch_bounds__(kRebuildWarps * 32, rebuild_min_blocks<G, CPL>
         valid = nC >= lo + 32 ? 0xFFFFFFFFu : (nC > lo ? (1u << (nC - lo)) - 1u : 0u);
       }
       const uint32_t nu = nC - kpe;
-      uint32_t jprev = kInvalid;
-      uint4 rj[CPL];
-#pragma unroll
-      for (int c = 0; c < CPL; ++c) rj[c] = make_uint4(0, 0, 0, 0);
       if (nu <= 2 * P && kpe == kp) {  // (the list of uncertain positions holds 2P entries; the tags must be trusted)
         // ---- few uncertain members among a pruned run.  Members of the run never prune each other, so the
         //      sequential prune only ever changes at an uncertain member f, and those are taken in key order:
@@ -508,33 +571,12 @@ __global__ void __launch_bounds__(kRebuildWarps * 32, rebuild_min_blocks<G, CPL>
           __syncwarp();
         }
       } else {
-        for (uint32_t w = lane; w < nC * W; w += 32) prune[w] = 0u;
-        __syncwarp();
-        const uint32_t npairs = nC * (nC - 1) / 2;
-        for (uint32_t pb = 0; pb < npairs; pb += NT) {
-          const uint32_t p = pb + team;
-          const bool act = p < npairs;
-          uint32_t i = 0, j = 1;
-          if (act) {
-            j = (uint32_t)((1.0f + sqrtf(1.0f + 8.0f * (float)p)) * 0.5f);
-            while (j * (j - 1) / 2 > p) --j;
-            while ((j + 1) * j / 2 <= p) ++j;
-            i = p - j * (j - 1) / 2;
-          }
-          pair_test(act, i, j, jprev, rj);
-        }
-        __syncwarp();
-        // ---- sequential selection replayed on bit masks.  The valid set only changes when a still-valid
-        //      candidate with a non-zero matrix row is reached, so only those candidates are visited, in
-        //      ascending order; everything valid in between is selected.
-        for (uint32_t w = 0; w < W; ++w) {
-          uint32_t hw = hasp[w];
-          while (hw) {
-            const uint32_t b = __ffs(hw) - 1;
-            hw &= hw - 1;
-            const uint32_t vw = __shfl_sync(FULL, valid, w);
-            if (((vw >> b) & 1u) && (uint32_t)lane < W) valid &= ~prune[(w * 32 + b) * W + lane];
-          }
+        if constexpr (rebuild_cold_paths_out_of_line<G, CPL>()) {
+          unsigned long long tested = 0;  // (a local of this branch: the loop's own counter stays in a register)
+          valid = prune_all_pairs_ool<T, G, CPL>(store, row_bytes, nchunk, cs, nC, W, prune, hasp, ap, valid, tested, lane);
+          npair += tested;
+        } else {
+          valid = prune_all_pairs_impl<T, G, CPL>(store, row_bytes, nchunk, cs, nC, W, prune, hasp, ap, valid, npair, lane);
         }
       }
       __syncwarp();
