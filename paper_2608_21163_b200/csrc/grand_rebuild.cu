@@ -175,6 +175,41 @@ __device__ __noinline__ uint32_t prune_all_pairs_ool(const uint8_t* __restrict__
   return prune_all_pairs_impl<T, G, CPL>(store, row_bytes, nchunk, cs, nC, W, prune, hasp, ap, valid, npair, lane);
 }
 
+// D_u for kept neighbours whose distance is not cached in the row (rows of an imported graph, ids that have come
+// back since the row was written): dist(u, keep[j]) into cand[j], tagged uncertain behind the pruned run.
+template <typename T, int G, int CPL>
+__device__ __forceinline__ void fill_uncached_dists_impl(const uint8_t* __restrict__ store, uint32_t row_bytes, uint32_t nchunk, uint32_t u,
+                                                         const uint32_t* keep, const uint32_t* keepd, uint32_t nk, uint32_t kp,
+                                                         unsigned long long* cand, unsigned long long& npair, int lane) {
+  using Dist = typename Elem<T>::Dist;
+  constexpr int NT = 32 / G;
+  const int t = lane % G, team = lane / G;
+  uint4 ur[CPL];
+  load_row<G, CPL>(store + (size_t)u * row_bytes, nchunk, t, ur);
+  for (uint32_t jb = 0; jb < nk; jb += NT) {
+    const uint32_t j = jb + team;
+    const bool act = j < nk && keepd[j] == kInvalid;
+    uint4 v[CPL];
+    if (act) {
+      load_row<G, CPL>(store + (size_t)keep[j] * row_bytes, nchunk, t, v);
+    } else {
+#pragma unroll
+      for (int c = 0; c < CPL; ++c) v[c] = make_uint4(0, 0, 0, 0);
+    }
+    const Dist d = team_dist_regs<T, kMetricL2, G, CPL>(ur, v);
+    if (act && t == 0) {
+      cand[j] = make_key(d, keep[j]) | (j >= kp ? kExpandedBit : 0ull);
+      ++npair;
+    }
+  }
+}
+template <typename T, int G, int CPL>
+__device__ __noinline__ void fill_uncached_dists_ool(const uint8_t* __restrict__ store, uint32_t row_bytes, uint32_t nchunk, uint32_t u,
+                                                     const uint32_t* keep, const uint32_t* keepd, uint32_t nk, uint32_t kp,
+                                                     unsigned long long* cand, unsigned long long& npair, int lane) {
+  fill_uncached_dists_impl<T, G, CPL>(store, row_bytes, nchunk, u, keep, keepd, nk, kp, cand, npair, lane);
+}
+
 template <typename T, int METRIC, int G, int CPL>
 __global__ void __launch_bounds__(kRebuildWarps * 32, rebuild_min_blocks<G, CPL>()) rebuild_kernel(const RebuildArgs a, const uint32_t per_warp_bytes) {
   using Dist = typename Elem<T>::Dist;
@@ -343,23 +378,12 @@ __global__ void __launch_bounds__(kRebuildWarps * 32, rebuild_min_blocks<G, CPL>
         if (__any_sync(FULL, miss)) all_cached = false;
       }
       if (!all_cached) {
-        uint4 ur[CPL];
-        load_row<G, CPL>(store + (size_t)u * row_bytes, nchunk, t, ur);
-        for (uint32_t jb = 0; jb < nk; jb += NT) {
-          const uint32_t j = jb + team;
-          const bool act = j < nk && keepd[j] == kInvalid;
-          uint4 v[CPL];
-          if (act) {
-            load_row<G, CPL>(store + (size_t)keep[j] * row_bytes, nchunk, t, v);
-          } else {
-#pragma unroll
-            for (int c = 0; c < CPL; ++c) v[c] = make_uint4(0, 0, 0, 0);
-          }
-          const Dist d = team_dist_regs<T, kMetricL2, G, CPL>(ur, v);
-          if (act && t == 0) {
-            cand[j] = make_key(d, keep[j]) | (j >= kp ? kExpandedBit : 0ull);
-            ++npair;
-          }
+        if constexpr (rebuild_cold_paths_out_of_line<G, CPL>()) {
+          unsigned long long tested = 0;
+          fill_uncached_dists_ool<T, G, CPL>(store, row_bytes, nchunk, u, keep, keepd, nk, kp, cand, tested, lane);
+          npair += tested;
+        } else {
+          fill_uncached_dists_impl<T, G, CPL>(store, row_bytes, nchunk, u, keep, keepd, nk, kp, cand, npair, lane);
         }
       }
       __syncwarp();
