@@ -264,6 +264,33 @@ def test_delete_repair_bit_exact_across_row_sizes(dim, dtype):
         assert_same_graph(o, g, f"delete {r}")
 
 
+@pytest.mark.parametrize("dim", [16, 96, 100, 300, 960])
+def test_fp32_rows_with_small_integer_coordinates_bit_exact(dim):
+    """fp32 vectors whose coordinates are small integers: every partial sum of a squared distance is exact in
+    fp32, whatever the order, and alpha = 1.25 makes the prune test exact as well - so the fp32 kernels (register
+    and warp tiles of the delete repair, the prunes, the rebuild, the search; one row size per layout class) must
+    reproduce the fp64 oracle bit for bit, not only within the tolerance."""
+    torch = torch_()
+    n = 2400
+    base = (synth.uniform_u8(21, f"intf32/{dim}", 0, n, dim) % 8).astype(np.float32)
+    cfg = dict(dim=dim, dtype=go.F32, metric=go.L2, R=16, L=32, alpha=1.25, mode=go.VAMANA, max_build_batch=600, ins=1, dele=500)
+    o, g = make_pair(cfg, n)
+    for lo in range(0, n, 600):
+        ids = np.arange(lo, lo + 600, dtype=np.uint32)
+        o.insert_batch(ids, base[ids]); g.insert_batch(torch.from_numpy(ids), torch.from_numpy(base[ids]))
+        assert_same_graph(o, g, f"build {lo}")
+    alive = np.ones(n, bool)
+    for r in range(2):
+        dele = synth.choose_ids(dim, f"intdel/{r}", np.flatnonzero(alive).astype(np.uint32), 500)
+        o.delete_batch(dele); g.delete_batch(torch.from_numpy(dele))
+        alive[dele] = False
+        assert_same_graph(o, g, f"delete {r}")
+    q = (synth.uniform_u8(22, f"intq/{dim}", 0, 100, dim) % 8).astype(np.float32)
+    oi, od = o.search(q, 10, 32)
+    gi, gd = gpu_search(g, q, 10, 32)
+    assert (oi == gi).all() and (od == gd.astype(np.float64)).all()
+
+
 def test_hub_segment_longer_than_shared_memory_cap():
     """Every point of a large batch links to the same few hubs: request segments far above the
     in-kernel shared-memory cap take the in-place global-memory sort."""
