@@ -99,12 +99,13 @@ __device__ __noinline__ uint32_t stream_best_keys_ool(const unsigned long long* 
                                                       uint32_t P, int lane) {
   return stream_best_keys_impl(seg, cntu, scratch, P, lane);
 }
-// Whether the two rare paths of the rebuild sit out of line.  Out of line they shorten the per-node loop (128-byte
-// rows: rebuild 1.79 -> 1.60 ms per step, alternating runs of both builds on one GPU); the calls cost the 6-chunk
-// layout, which runs at its register bound, a few more spills (53.3 against 51.8 ms per step), so that layout keeps
-// them inline.
+// Whether the rare paths of the rebuild sit out of line.  Out of line they shorten the per-node loop, which pays on
+// rows of at most 128 bytes, where the kernel is bound by instruction issue and fetch (rebuild 1.79 -> 1.60 ms per
+// step, alternating runs of both builds on one GPU).  Elsewhere they stay inline: the calls cost the 6-chunk layout,
+// which runs at its register bound, a few more spills (53.3 against 51.8 ms per step), and on wide rows with reused
+// ids and strong hubs these paths are not rare at all (GIST-shaped rebuild 41 against 55 ms per step).
 template <int G, int CPL>
-constexpr bool rebuild_cold_paths_out_of_line() { return !(G == 4 && CPL == 6); }
+constexpr bool rebuild_cold_paths_out_of_line() { return G * CPL <= 8; }
 
 // Fallback of the prune for candidate lists without a trusted run: every test alpha * dist(c_i, c_j) <= D_u[c_j],
 // i < j, goes into a bit matrix (row i, bit j = "c_i prunes c_j"), and the sequential selection is replayed on
