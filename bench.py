@@ -50,6 +50,7 @@ NCU_TRAFFIC = {
     ("sift_u8_d128", 1.0): (0.379, "profiles/beam_search_dram_sift_u8_d128_full.txt"),
     ("gist_f32_d960", 1.0): (0.680, "profiles/beam_search_dram_gist_f32_d960_full.txt"),
     ("embed_f32_d768_ip", 1.0): (0.971, "profiles/beam_search_dram_embed_f32_d768_ip_full.txt"),
+    ("deep_f32_d96_isotropic", 1.0): (0.961, "profiles/beam_search_dram_deep_f32_d96_isotropic_full.txt"),
 }
 
 
